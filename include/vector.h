@@ -27,7 +27,8 @@
  *  - Linear maps follow the paper's column convention y = W x: W[c_out][c_in],
  *    row-major, one d x d map per (layer, KV head): index l * n_kv_heads + h.
  *  - Supported: head_dim 64 or 128; dtype fp32 or bf16; n_q_heads % n_kv_heads == 0,
- *    g <= 16; window * g <= 1024; pool_kernel odd, 1..15.
+ *    g <= 8; window * g <= 1024; pool_kernel odd, 1..15; at most 65535 units per call;
+ *    every device pointer 16-byte aligned.
  */
 #ifndef VECTOR_H_
 #define VECTOR_H_
@@ -37,6 +38,12 @@
 
 #ifdef __cplusplus
 extern "C" {
+#endif
+
+#if defined(__GNUC__)
+#define VECTOR_API __attribute__((visibility("default")))
+#else
+#define VECTOR_API
 #endif
 
 typedef enum {
@@ -93,9 +100,9 @@ typedef struct {
 } vector_cache;
 
 /* Text for a status code (static storage). */
-const char* vector_status_string(vector_status s);
+VECTOR_API const char* vector_status_string(vector_status s);
 /* The raw cudaError_t of the last VECTOR_ERR_CUDA on this thread (0 if none). */
-int vector_last_cuda_error(void);
+VECTOR_API int vector_last_cuda_error(void);
 
 /*
  * Tier sizes, host only (paper Section 3.2 proportions and Eq. (1)).
@@ -103,10 +110,10 @@ int vector_last_cuda_error(void);
  * taken as 0: n_a = min(floor((N - Bp)/2), floor(Bp/2)); otherwise n_a is used
  * as given.  Derived: n_pool = Bp + n_a, n_apx = 2 n_a, n_ret = Bp - n_a, so
  * n_pool keys + n_ret values cost exactly Bp pairs.  Errors: VECTOR_ERR_BUDGET
- * if Bp > N, 2 n_a > Bp, n_pool > N, window > N or n_pool < window (the base
+ * if Bp > N, n_a > Bp, n_pool > N, window > N or n_pool < window (the base
  * scorer always keeps its observation window).
  */
-vector_status vector_plan_budget(int64_t n_tokens, int64_t n_budget_pairs, int64_t n_a,
+VECTOR_API vector_status vector_plan_budget(int64_t n_tokens, int64_t n_budget_pairs, int64_t n_a,
                                  int32_t window, vector_budget* out /* host */);
 
 /*
@@ -117,11 +124,11 @@ vector_status vector_plan_budget(int64_t n_tokens, int64_t n_budget_pairs, int64
  * 1 - sum||v - W k||^2 / sum||v - mean(v)||^2.  VECTOR_ERR_SINGULAR if the
  * regularised Gram matrix is not positive definite.
  */
-vector_status vector_calibrate(const void* K, const void* V, int64_t n, int32_t d_k, int32_t d_v,
+VECTOR_API vector_status vector_calibrate(const void* K, const void* V, int64_t n, int32_t d_k, int32_t d_v,
                                int32_t dt, double lambda, float* W_out, double* r2_out);
 
 /* Bytes of device workspace that suffice for every device call with this shape and budget. */
-size_t vector_workspace_bytes(const vector_shape* shape, const vector_budget* budget);
+VECTOR_API size_t vector_workspace_bytes(const vector_shape* shape, const vector_budget* budget);
 
 /*
  * Base importance score (Step 1's scorer, SnapKV-style).  For each unit the last
@@ -133,14 +140,14 @@ size_t vector_workspace_bytes(const vector_shape* shape, const vector_budget* bu
  * Q_obs: device [U][g][w][d]; K: device [U][N][d]; scores: device fp32 [U][N];
  * raw_out (nullable): device fp32 [U][N], the un-pooled sums.
  */
-vector_status vector_score(const vector_shape* shape, const void* Q_obs, const void* K, int64_t N,
+VECTOR_API vector_status vector_score(const vector_shape* shape, const void* Q_obs, const void* K, int64_t N,
                            float* scores, float* raw_out, void* ws, size_t ws_bytes, void* stream);
 
 /*
  * Step 1, budget relaxation: per unit the n_pool largest scores, ties to the
  * lower index.  scores: device fp32 [U][N]; pool_idx: device [U][n_pool] ascending.
  */
-vector_status vector_pool_select(const vector_shape* shape, const vector_budget* budget,
+VECTOR_API vector_status vector_pool_select(const vector_shape* shape, const vector_budget* budget,
                                  const float* scores, int32_t* pool_idx,
                                  void* ws, size_t ws_bytes, void* stream);
 
@@ -150,7 +157,7 @@ vector_status vector_pool_select(const vector_shape* shape, const vector_budget*
  * K, V: device [U][N][d]; W: device [L*Hkv][d][d] of shape->dtype;
  * idx: device [U][n_idx]; eps: device fp32 [U][n_idx].
  */
-vector_status vector_residual(const vector_shape* shape, const void* K, const void* V, const void* W,
+VECTOR_API vector_status vector_residual(const vector_shape* shape, const void* K, const void* V, const void* W,
                               int64_t N, const int32_t* idx, int64_t n_idx, float* eps, void* stream);
 
 /*
@@ -160,7 +167,7 @@ vector_status vector_residual(const vector_shape* shape, const void* K, const vo
  * tier: device [U][N], 0 evicted / 1 approximated / 2 retained;
  * ret_idx: device [U][n_ret], apx_idx: device [U][n_apx], both ascending.
  */
-vector_status vector_truncate(const vector_shape* shape, const vector_budget* budget,
+VECTOR_API vector_status vector_truncate(const vector_shape* shape, const vector_budget* budget,
                               const float* eps, const int32_t* pool_idx,
                               uint8_t* tier, int32_t* ret_idx, int32_t* apx_idx,
                               void* ws, size_t ws_bytes, void* stream);
@@ -170,7 +177,7 @@ vector_status vector_truncate(const vector_shape* shape, const vector_budget* bu
  * Arguments as in the three calls above; eps_out (nullable): device fp32
  * [U][n_pool]; pool_idx_out (nullable): device [U][n_pool].
  */
-vector_status vector_route(const vector_shape* shape, const vector_budget* budget,
+VECTOR_API vector_status vector_route(const vector_shape* shape, const vector_budget* budget,
                            const float* scores, const void* K, const void* V, const void* W,
                            uint8_t* tier, int32_t* ret_idx, int32_t* apx_idx,
                            float* eps_out, int32_t* pool_idx_out,
@@ -182,7 +189,7 @@ vector_status vector_route(const vector_shape* shape, const vector_budget* budge
  * indices to ret_pos / apx_pos.  Requires cache->n_ret == budget->n_ret,
  * cache->n_apx == budget->n_apx, capacities >= counts (VECTOR_ERR_SHAPE).
  */
-vector_status vector_compact(const vector_shape* shape, const vector_budget* budget,
+VECTOR_API vector_status vector_compact(const vector_shape* shape, const vector_budget* budget,
                              const void* K, const void* V,
                              const int32_t* ret_idx, const int32_t* apx_idx,
                              const vector_cache* cache, void* stream);
@@ -195,7 +202,7 @@ vector_status vector_compact(const vector_shape* shape, const vector_budget* bud
  *   mode 1 (per tile):  o = sum_R p_i v_i + sum_A p_i (W k~_i)
  * q: device [U][g][d] of shape->dtype; out: device [U][g][d] of out_dtype.
  */
-vector_status vector_decode_attn(const vector_shape* shape, const void* q, const vector_cache* cache,
+VECTOR_API vector_status vector_decode_attn(const vector_shape* shape, const void* q, const vector_cache* cache,
                                  const void* W, void* out, int32_t out_dtype, int32_t mode,
                                  void* ws, size_t ws_bytes, void* stream);
 

@@ -61,8 +61,9 @@ int oracle_plan_budget(int64_t n_tokens, int64_t n_budget_pairs, int64_t n_a,
         int64_t b = n_budget_pairs / 2;
         n_a = a < b ? a : b;
     }
-    /* the approximation tier may not outgrow half the budget, nor the evictable tokens */
-    if (2 * n_a > n_budget_pairs) return ORACLE_ERR_BUDGET;
+    /* an explicit n_a may empty the retention tier (the sensitivity sweep of Section 5.3
+       reaches p_a = 0.5 at p_c = 0.5) but not make it negative, nor outgrow the context */
+    if (n_a > n_budget_pairs) return ORACLE_ERR_BUDGET;
     if (n_budget_pairs + n_a > n_tokens) return ORACLE_ERR_BUDGET;
     out->n_tokens = n_tokens;
     out->n_budget_pairs = n_budget_pairs;

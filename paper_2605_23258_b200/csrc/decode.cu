@@ -1,0 +1,216 @@
+// Generation-time attention over the mixed cache (paper Section 3.2, Step 3):
+// one softmax over the exact keys of the retained and the key-only pool; a
+// retained token contributes its stored value, an approximated token W k.
+// Factored form: o = sum_R p_i v_i + W (sum_A p_i k_i), so the kernel streams
+// both pools once, accumulating p-weighted values and p-weighted keys, and the
+// d x d map is applied once per query head in the merge step.
+//
+//   split  grid (n_splits, U): online softmax over a slice of the logical key
+//          range [0, n_ret + n_apx); emits (m, l, acc_v[d], acc_k[d]) per head
+//   merge  grid (U): combines the splits, applies W to acc_k, normalises
+#include "common.cuh"
+#include "internal.h"
+
+namespace vec {
+
+template <typename T, int EPL> struct RowLoad;
+template <> struct RowLoad<float, 4> {
+    static __device__ __forceinline__ void load(const float* p, int lane, float (&o)[4]) {
+        float4 v = reinterpret_cast<const float4*>(p)[lane];
+        o[0] = v.x; o[1] = v.y; o[2] = v.z; o[3] = v.w;
+    }
+};
+template <> struct RowLoad<float, 2> {
+    static __device__ __forceinline__ void load(const float* p, int lane, float (&o)[2]) {
+        float2 v = reinterpret_cast<const float2*>(p)[lane];
+        o[0] = v.x; o[1] = v.y;
+    }
+};
+template <> struct RowLoad<__nv_bfloat16, 4> {
+    static __device__ __forceinline__ void load(const __nv_bfloat16* p, int lane, float (&o)[4]) {
+        uint2 v = reinterpret_cast<const uint2*>(p)[lane];
+        o[0] = __uint_as_float(v.x << 16); o[1] = __uint_as_float(v.x & 0xffff0000u);
+        o[2] = __uint_as_float(v.y << 16); o[3] = __uint_as_float(v.y & 0xffff0000u);
+    }
+};
+template <> struct RowLoad<__nv_bfloat16, 2> {
+    static __device__ __forceinline__ void load(const __nv_bfloat16* p, int lane, float (&o)[2]) {
+        uint32_t v = reinterpret_cast<const uint32_t*>(p)[lane];
+        o[0] = __uint_as_float(v << 16); o[1] = __uint_as_float(v & 0xffff0000u);
+    }
+};
+
+// Partial record per (unit, split, head): [m, l, acc_v[D], acc_k[D]]
+template <int D> struct Rec { static constexpr int floats = 2 + 2 * D; };
+
+template <typename T, int D, int G>
+__global__ void __launch_bounds__(128)
+decode_split_generic(const T* __restrict__ q, const T* __restrict__ ret_k, const T* __restrict__ ret_v,
+                     const T* __restrict__ apx_k, int64_t cap_ret, int64_t cap_apx, int n_ret, int n_apx,
+                     int g, float scale, float* __restrict__ partial) {
+    constexpr int EPL = D / 32;
+    constexpr int REC = Rec<D>::floats;
+    __shared__ float sm[4][G][REC];
+    const int u = blockIdx.y, split = blockIdx.x, n_splits = gridDim.x;
+    const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
+    const int total = n_ret + n_apx;
+    const int per = (total + n_splits - 1) / n_splits;
+    const int lo = split * per, hi = min(total, lo + per);
+
+    float qr[G][EPL], av[G][EPL], ak[G][EPL], m[G], l[G];
+#pragma unroll
+    for (int a = 0; a < G; ++a) {
+        m[a] = -INFINITY;
+        l[a] = 0.f;
+#pragma unroll
+        for (int e = 0; e < EPL; ++e) { av[a][e] = 0.f; ak[a][e] = 0.f; qr[a][e] = 0.f; }
+        if (a < g) {
+            RowLoad<T, EPL>::load(q + ((size_t)u * g + a) * D, lane, qr[a]);
+#pragma unroll
+            for (int e = 0; e < EPL; ++e) qr[a][e] *= scale;
+        }
+    }
+    for (int i = lo + wid; i < hi; i += 4) {
+        const bool retained = i < n_ret;
+        const T* kp = retained ? ret_k + ((size_t)u * cap_ret + i) * D
+                               : apx_k + ((size_t)u * cap_apx + (i - n_ret)) * D;
+        float kx[EPL], vx[EPL];
+        RowLoad<T, EPL>::load(kp, lane, kx);
+        if (retained) RowLoad<T, EPL>::load(ret_v + ((size_t)u * cap_ret + i) * D, lane, vx);
+#pragma unroll
+        for (int a = 0; a < G; ++a) {
+            if (a < g) {
+                float s = 0.f;
+#pragma unroll
+                for (int e = 0; e < EPL; ++e) s = fmaf(qr[a][e], kx[e], s);
+                s = warp_sum(s);
+                float mn = fmaxf(m[a], s);
+                float corr = __expf(m[a] - mn);     // first row: exp(-inf) = 0
+                float p = __expf(s - mn);
+                m[a] = mn;
+                l[a] = l[a] * corr + p;
+#pragma unroll
+                for (int e = 0; e < EPL; ++e) {
+                    av[a][e] *= corr;
+                    ak[a][e] *= corr;
+                    if (retained) av[a][e] = fmaf(p, vx[e], av[a][e]);
+                    else          ak[a][e] = fmaf(p, kx[e], ak[a][e]);
+                }
+            }
+        }
+    }
+#pragma unroll
+    for (int a = 0; a < G; ++a) {
+        if (a < g) {
+            if (lane == 0) { sm[wid][a][0] = m[a]; sm[wid][a][1] = l[a]; }
+#pragma unroll
+            for (int e = 0; e < EPL; ++e) {
+                sm[wid][a][2 + lane * EPL + e] = av[a][e];
+                sm[wid][a][2 + D + lane * EPL + e] = ak[a][e];
+            }
+        }
+    }
+    __syncthreads();
+    float* out = partial + ((size_t)u * n_splits + split) * g * REC;
+    for (int a = 0; a < g; ++a) {
+        float M = fmaxf(fmaxf(sm[0][a][0], sm[1][a][0]), fmaxf(sm[2][a][0], sm[3][a][0]));
+        float f[4];
+#pragma unroll
+        for (int wv = 0; wv < 4; ++wv) f[wv] = sm[wv][a][0] > -INFINITY ? __expf(sm[wv][a][0] - M) : 0.f;
+        for (int c = threadIdx.x; c < REC; c += 128) {
+            float v;
+            if (c == 0) v = M;
+            else v = f[0] * sm[0][a][c] + f[1] * sm[1][a][c] + f[2] * sm[2][a][c] + f[3] * sm[3][a][c];
+            out[a * REC + c] = v;
+        }
+    }
+}
+
+// grid (U), D threads.
+template <typename T, typename TO, int D>
+__global__ void __launch_bounds__(D)
+decode_merge_generic(const float* __restrict__ partial, const T* __restrict__ W, int LH, int g, int n_splits,
+                     TO* __restrict__ out) {
+    constexpr int REC = Rec<D>::floats;
+    __shared__ float aks[D];
+    const int u = blockIdx.x, c = threadIdx.x;
+    const T* Wu = W + (size_t)(u % LH) * D * D;
+    for (int a = 0; a < g; ++a) {
+        const float* rec = partial + ((size_t)u * n_splits * g + a) * REC;
+        const size_t stride = (size_t)g * REC;
+        float M = -INFINITY;
+        for (int s = 0; s < n_splits; ++s) M = fmaxf(M, rec[s * stride]);
+        float L = 0.f, accv = 0.f, acck = 0.f;
+        for (int s = 0; s < n_splits; ++s) {
+            const float* r = rec + s * stride;
+            float f = r[0] > -INFINITY ? __expf(r[0] - M) : 0.f;
+            L += f * r[1];
+            accv += f * r[2 + c];
+            acck += f * r[2 + D + c];
+        }
+        __syncthreads();
+        aks[c] = acck;
+        __syncthreads();
+        float proj = 0.f;
+#pragma unroll 8
+        for (int c2 = 0; c2 < D; ++c2) proj = fmaf(to_f32(Wu[(size_t)c * D + c2]), aks[c2], proj);
+        store_out(out + ((size_t)u * g + a) * D + c, (accv + proj) / L);
+    }
+}
+
+template <typename T, int D, int G>
+static vector_status launch_decode(const Dims& dm, const void* q, const vector_cache* ch, const void* W, void* out,
+                                   int out_dtype, float* partial, cudaStream_t st) {
+    const int n_splits = decode_num_splits(dm.U, ch->n_ret + ch->n_apx);
+    dim3 grid(n_splits, dm.U);
+    decode_split_generic<T, D, G><<<grid, 128, 0, st>>>((const T*)q, (const T*)ch->ret_k, (const T*)ch->ret_v,
+                                                        (const T*)ch->apx_k, ch->cap_ret, ch->cap_apx,
+                                                        (int)ch->n_ret, (int)ch->n_apx, dm.g, dm.scale, partial);
+    VEC_LAUNCH_CHECK();
+    if (out_dtype == VECTOR_F32)
+        decode_merge_generic<T, float, D><<<dm.U, D, 0, st>>>(partial, (const T*)W, dm.LH, dm.g, n_splits,
+                                                             (float*)out);
+    else
+        decode_merge_generic<T, __nv_bfloat16, D><<<dm.U, D, 0, st>>>(partial, (const T*)W, dm.LH, dm.g, n_splits,
+                                                                     (__nv_bfloat16*)out);
+    VEC_LAUNCH_CHECK();
+    return VECTOR_OK;
+}
+
+template <typename T, int D>
+static vector_status launch_decode_g(const Dims& dm, const void* q, const vector_cache* ch, const void* W,
+                                     void* out, int out_dtype, float* partial, cudaStream_t st) {
+    if (dm.g <= 2) return launch_decode<T, D, 2>(dm, q, ch, W, out, out_dtype, partial, st);
+    if (dm.g <= 4) return launch_decode<T, D, 4>(dm, q, ch, W, out, out_dtype, partial, st);
+    return launch_decode<T, D, 8>(dm, q, ch, W, out, out_dtype, partial, st);
+}
+
+}  // namespace vec
+
+using namespace vec;
+
+extern "C" vector_status vector_decode_attn(const vector_shape* shape, const void* q, const vector_cache* cache,
+                                            const void* W, void* out, int32_t out_dtype, int32_t mode, void* ws,
+                                            size_t ws_bytes, void* stream) {
+    Dims dm;
+    vector_status rc = check_shape(shape, &dm);
+    if (rc != VECTOR_OK) return rc;
+    if (!q || !cache || !W || !out) return VECTOR_ERR_NULL;
+    if (out_dtype != VECTOR_F32 && out_dtype != VECTOR_BF16) return VECTOR_ERR_DTYPE;
+    if (mode != 0 && mode != 1) return VECTOR_ERR_SHAPE;
+    if (cache->n_ret < 0 || cache->n_apx < 0 || cache->n_ret + cache->n_apx <= 0 ||
+        cache->n_ret + cache->n_apx > (int64_t(1) << 30) || cache->cap_ret < cache->n_ret ||
+        cache->cap_apx < cache->n_apx)
+        return VECTOR_ERR_SHAPE;
+    if (cache->n_ret > 0 && (!cache->ret_k || !cache->ret_v)) return VECTOR_ERR_NULL;
+    if (cache->n_apx > 0 && !cache->apx_k) return VECTOR_ERR_NULL;
+    if (!ws || ((uintptr_t)ws & 255) || ws_bytes < decode_ws_bytes(dm)) return VECTOR_ERR_WORKSPACE;
+    if (mode == 1 || dm.rope) return VECTOR_ERR_UNSUPPORTED;
+    cudaStream_t st = (cudaStream_t)stream;
+    float* partial = (float*)ws;
+    if (dm.dtype == VECTOR_F32)
+        return dm.d == 64 ? launch_decode_g<float, 64>(dm, q, cache, W, out, out_dtype, partial, st)
+                          : launch_decode_g<float, 128>(dm, q, cache, W, out, out_dtype, partial, st);
+    return dm.d == 64 ? launch_decode_g<__nv_bfloat16, 64>(dm, q, cache, W, out, out_dtype, partial, st)
+                      : launch_decode_g<__nv_bfloat16, 128>(dm, q, cache, W, out, out_dtype, partial, st);
+}

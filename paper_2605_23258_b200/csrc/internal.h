@@ -1,0 +1,59 @@
+// Internal declarations shared by the translation units of libvector (host side).
+#ifndef VECTOR_INTERNAL_H_
+#define VECTOR_INTERNAL_H_
+
+#include <cstddef>
+#include <cstdint>
+
+#include "vector.h"
+
+namespace vec {
+
+// Geometry derived from a validated vector_shape.
+struct Dims {
+    int U;        // units = batch * n_layers * n_kv_heads
+    int LH;       // maps  = n_layers * n_kv_heads
+    int g;        // query heads per KV head
+    int d;        // head_dim
+    int w;        // observation window
+    int R;        // score rows per unit = g * w
+    int pool_kernel;
+    int dtype;
+    int esize;    // bytes per element
+    float scale;
+    int rope;
+    float theta;
+};
+
+// Checks a shape against what the kernels support and fills Dims.
+vector_status check_shape(const vector_shape* s, Dims* out);
+// Checks internal consistency of tier sizes (the identities of the planner).
+vector_status check_budget(const vector_budget* b, int window);
+
+void set_last_cuda_error(int e);
+
+// ---- workspace layout (bytes, each region 256-byte aligned) ----
+// Number of key chunks the first score pass splits a unit's keys into.
+int score_num_chunks(int U, int R, int64_t N);
+size_t score_ws_bytes(const Dims& D, int64_t N, bool need_raw);
+size_t select_ws_bytes(const Dims& D, const vector_budget& b);
+// Number of key splits of one unit in decode attention for `rows` logical keys.
+int decode_num_splits(int U, int64_t rows);
+size_t decode_ws_bytes(const Dims& D);
+
+inline size_t align256(size_t x) { return (x + 255) & ~size_t(255); }
+
+}  // namespace vec
+
+#define VEC_CUDA_CHECK(expr)                                  \
+    do {                                                      \
+        cudaError_t e__ = (expr);                             \
+        if (e__ != cudaSuccess) {                             \
+            vec::set_last_cuda_error((int)e__);               \
+            return VECTOR_ERR_CUDA;                           \
+        }                                                     \
+    } while (0)
+
+#define VEC_LAUNCH_CHECK() VEC_CUDA_CHECK(cudaPeekAtLastError())
+
+#endif  // VECTOR_INTERNAL_H_

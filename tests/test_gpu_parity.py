@@ -1,0 +1,311 @@
+"""Parity of the CUDA path (through the C-ABI) with the CPU oracle on the same seeded inputs.
+
+Tolerances:
+  scores          |g - o| <= 1e-3 * max(|o|, 1e-6 * g*w)     (g*w = total attention mass of a unit)
+  selections      bit-exact when both sides are fed identical fp32 scores / residuals
+  residual eps    relative 2e-5 (fp32 accumulation of exact products, d <= 128 terms, vs fp64)
+  end-to-end      >= 99.9 % of tokens routed alike; each disagreement sits within 1e-3 (relative)
+                  of the oracle's own selection threshold
+  decode output   |o_gpu - o_oracle| <= 2e-2 with fp32 output; bf16 output adds 2^-8 |o|
+"""
+import numpy as np
+import pytest
+import torch
+
+import paper_2605_23258_b200 as vec
+from paper_2605_23258_b200 import synth
+from paper_2605_23258_b200.pipeline import Compressor
+
+from helpers import budget_of, calibrated_maps, oracle_scores, score_close, shape_of
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda"
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _lib():
+    assert torch.cuda.is_available(), "these tests need the B200"
+    vec.load_library()          # fails loudly if the CUDA library has not been built
+
+
+SCORE_CASES = [
+    # (base workload, overrides)
+    (0, {}),                                                    # config 0 as given: fp32, d=64, N=1024
+    (0, {"N": 333, "window": 16, "pool_kernel": 5}),            # ragged tail, fp32
+    (1, {"N": 1000, "n_kv_heads": 2, "n_q_heads": 8}),          # bf16 d=128, N not a tile multiple
+    (1, {"N": 4096 + 77, "n_kv_heads": 1, "n_q_heads": 4}),
+    (4, {"N": 2048 + 5, "n_layers": 1, "n_kv_heads": 1, "n_q_heads": 8, "window": 128}),   # g=8, 1024 rows
+    (1, {"N": 64, "n_kv_heads": 1, "n_q_heads": 4}),            # N == window: every token is a window token
+    (1, {"N": 70, "n_kv_heads": 1, "n_q_heads": 1, "window": 3, "pool_kernel": 1}),        # g=1, tiny window
+    (0, {"N": 640, "head_dim": 128, "dtype": "bf16"}),
+    (1, {"N": 900, "head_dim": 64, "n_kv_heads": 1, "n_q_heads": 2}),                      # bf16 d=64
+]
+
+
+@pytest.mark.parametrize("base,over", SCORE_CASES)
+def test_score_parity(oracle, base, over):
+    wl = synth.shrink(synth.WORKLOADS[base], **over)
+    K, V, Q = synth.context(wl, DEV)
+    sh = shape_of(wl)
+    b = vec.vector_plan_budget(wl.N, wl.N, 0, wl.window)
+    ws = vec.alloc_workspace(sh, b)
+    scores = torch.empty(wl.units, wl.N, dtype=torch.float32, device=DEV)
+    raw = torch.empty_like(scores)
+    vec.vector_score(sh, Q, K, wl.N, scores, raw, ws)
+    scores2 = torch.empty_like(scores)
+    vec.vector_score(sh, Q, K, wl.N, scores2, None, ws)        # raw kept in the workspace
+    torch.cuda.synchronize()
+    assert torch.equal(scores, scores2)
+    raw_o, sc_o = oracle_scores(oracle, wl, Q.cpu(), K.cpu())
+    mass = wl.group * wl.window
+    ok, worst = score_close(scores.cpu().numpy(), sc_o, mass)
+    assert ok, f"score off by {worst:.3g} x tolerance"
+    ok, worst = score_close(raw.cpu().numpy(), raw_o, mass)
+    assert ok, f"raw off by {worst:.3g} x tolerance"
+    # the mass every unit distributes is g*w
+    assert np.allclose(raw.double().sum(1).cpu().numpy(), mass, rtol=1e-4)
+
+
+def _selection_inputs(U, N, seed, ties):
+    g = torch.Generator().manual_seed(seed)
+    s = torch.rand(U, N, generator=g)
+    if ties:
+        s = torch.round(s * 16) / 16                    # many exact ties
+    s[:, -8:] = float("inf")
+    s[0, : N // 3] = 0.0
+    return s
+
+
+@pytest.mark.parametrize("N,n_pool,ties", [(1000, 300, False), (1000, 300, True), (5000, 4999, True),
+                                           (4096, 8, True), (70000, 20000, True), (2048, 2048, False),
+                                           (131072, 9829, False)])
+def test_pool_select_bit_exact(oracle, N, n_pool, ties):
+    U = 3
+    s = _selection_inputs(U, N, N + n_pool, ties)
+    wl = synth.shrink(synth.WORKLOADS[0], N=N, window=8, n_kv_heads=U, n_q_heads=U)
+    sh = shape_of(wl)
+    b = vec.Budget(N, n_pool, 0, n_pool, 0, n_pool, N - n_pool)
+    out = torch.empty(U, n_pool, dtype=torch.int32, device=DEV)
+    vec.vector_pool_select(sh, b, s.to(DEV), out)
+    got = out.cpu().numpy()
+    for u in range(U):
+        assert np.array_equal(got[u], oracle.pool_select(s[u].numpy(), n_pool)), u
+
+
+@pytest.mark.parametrize("base,over,n_idx", [(0, {}, 384), (1, {"N": 3000, "n_kv_heads": 2, "n_q_heads": 8}, 1001),
+                                             (1, {"N": 500, "head_dim": 64, "n_kv_heads": 1, "n_q_heads": 2}, 77),
+                                             (0, {"N": 300, "head_dim": 128}, 300)])
+def test_residual_parity(oracle, base, over, n_idx):
+    wl = synth.shrink(synth.WORKLOADS[base], n_calib=1024, **over)
+    K, V, _ = synth.context(wl, DEV)
+    W = calibrated_maps(wl).to(DEV)
+    g = torch.Generator().manual_seed(5)
+    idx = torch.stack([torch.randperm(wl.N, generator=g)[:n_idx].sort().values for _ in range(wl.units)])
+    idx = idx.to(torch.int32).to(DEV)
+    eps = torch.empty(wl.units, n_idx, dtype=torch.float32, device=DEV)
+    vec.vector_residual(shape_of(wl), K, V, W, wl.N, idx, n_idx, eps)
+    got = eps.cpu().numpy()
+    for u in range(wl.units):
+        want = oracle.residual(K[u].cpu(), V[u].cpu(), W[u % W.shape[0]].cpu(), idx[u].cpu().numpy())
+        assert np.allclose(got[u], want, rtol=2e-5, atol=1e-30), u
+
+
+@pytest.mark.parametrize("N,n_pool,n_apx,ties", [(1024, 384, 256, False), (1024, 384, 256, True),
+                                                 (4000, 1501, 0, True), (4000, 1500, 1500, True),
+                                                 (131072, 9829, 6552, False), (50, 20, 2, True)])
+def test_truncate_bit_exact(oracle, N, n_pool, n_apx, ties):
+    U = 3
+    g = torch.Generator().manual_seed(N + n_apx)
+    pool = torch.stack([torch.randperm(N, generator=g)[:n_pool].sort().values for _ in range(U)]).to(torch.int32)
+    eps = torch.rand(U, n_pool, generator=g) * 3
+    if ties:
+        eps = torch.round(eps * 8) / 8
+    wl = synth.shrink(synth.WORKLOADS[0], N=N, window=1, n_kv_heads=U, n_q_heads=U)
+    n_a = n_apx // 2
+    b = vec.Budget(N, n_pool - n_a, n_a, n_pool, n_apx, n_pool - n_apx, N - n_pool)
+    tier = torch.empty(U, N, dtype=torch.uint8, device=DEV)
+    ret = torch.empty(U, max(n_pool - n_apx, 1), dtype=torch.int32, device=DEV)
+    apx = torch.empty(U, max(n_apx, 1), dtype=torch.int32, device=DEV)
+    vec.vector_truncate(shape_of(wl), b, eps.to(DEV), pool.to(DEV), tier, ret, apx)
+    for u in range(U):
+        t, r, a = oracle.truncate(eps[u].numpy(), pool[u].numpy(), n_apx, N)
+        assert np.array_equal(tier[u].cpu().numpy(), t)
+        assert np.array_equal(ret[u, : n_pool - n_apx].cpu().numpy(), r)
+        assert np.array_equal(apx[u, :n_apx].cpu().numpy(), a)
+
+
+def _oracle_route_unit(oracle, wl, b, score_f32, K, V, W):
+    return oracle.route(score_f32, K, V, W, b.n_pool, b.n_apx)
+
+
+def _assert_routing_agrees(oracle, wl, b, comp, K, V, W, sc_oracle, units):
+    """End-to-end agreement of the device routing (fed by device scores) with the oracle's."""
+    tier = comp.tier.cpu().numpy()
+    total = mism = 0
+    for j, u in enumerate(units):
+        s32 = sc_oracle[j].astype(np.float32)
+        r = _oracle_route_unit(oracle, wl, b, s32, K[j].cpu(), V[j].cpu(), W[u % W.shape[0]].cpu())
+        bad = np.nonzero(tier[j] != r["tier"])[0]
+        total += wl.N
+        mism += len(bad)
+        if len(bad) == 0:
+            continue
+        # thresholds of the oracle's own two selections
+        pool = r["pool_idx"]
+        in_pool = np.zeros(wl.N, bool)
+        in_pool[pool] = True
+        fin = np.isfinite(sc_oracle[j])
+        thr_s = np.min(sc_oracle[j][in_pool & fin]) if b.n_evict > 0 and np.any(in_pool & fin) else None
+        eps_all = oracle.residual(K[j].cpu(), V[j].cpu(), W[u % W.shape[0]].cpu(), np.arange(wl.N, dtype=np.int32))
+        is_apx = r["tier"] == 1
+        thr_e = np.max(eps_all[is_apx]) if b.n_apx > 0 else None
+        for i in bad:
+            near_s = thr_s is not None and abs(sc_oracle[j][i] - thr_s) <= 1e-3 * max(abs(thr_s), 1e-6 * wl.group * wl.window)
+            near_e = thr_e is not None and abs(eps_all[i] - thr_e) <= 1e-3 * abs(thr_e)
+            assert near_s or near_e, f"unit {u} token {i}: routed differently away from any threshold"
+    assert mism <= 1e-3 * total, f"{mism} of {total} tokens routed differently"
+
+
+def _run_pipeline_case(oracle, wl, percent, units=None, decode_steps=2, n_a=-1):
+    """Device pipeline on the given units, compared step by step with the oracle."""
+    units = list(range(wl.units)) if units is None else units
+    K, V, Q = synth.context(wl, DEV, units)
+    Wfull = calibrated_maps(wl)
+    LH = wl.n_layers * wl.n_kv_heads
+    # the device call indexes maps by u % LH; give it one map per listed unit in that layout
+    W = torch.stack([Wfull[u % LH] for u in units]).to(DEV)
+    sub = synth.shrink(wl, batch=1, n_layers=1, n_kv_heads=len(units), n_q_heads=len(units) * wl.group)
+    sh = shape_of(sub)
+    b = budget_of(wl, percent, n_a)
+    comp = Compressor(sh, b, extra_rows=decode_steps, keep_eps=True)
+    comp.compress(Q, K, V, W)
+    torch.cuda.synchronize()
+    raw_o, sc_o = oracle_scores(oracle, wl, Q.cpu(), K.cpu())
+    ok, worst = score_close(comp.scores.cpu().numpy(), sc_o, wl.group * wl.window)
+    assert ok, f"score off by {worst:.3g} x tolerance"
+    # routing fed by the oracle's scores must be bit-exact in Step 1, and in Step 3 given equal residuals
+    sc32 = torch.from_numpy(sc_o.astype(np.float32)).to(DEV)
+    tier = torch.empty_like(comp.tier)
+    ret = torch.empty_like(comp.ret_idx)
+    apx = torch.empty_like(comp.apx_idx)
+    eps = torch.empty(len(units), b.n_pool, dtype=torch.float32, device=DEV)
+    pool = torch.empty(len(units), b.n_pool, dtype=torch.int32, device=DEV)
+    vec.vector_route(sh, b, sc32, K, V, W, tier, ret, apx, eps, pool, comp.ws)
+    torch.cuda.synchronize()
+    for j, u in enumerate(units):
+        r = _oracle_route_unit(oracle, wl, b, sc_o[j].astype(np.float32), K[j].cpu(), V[j].cpu(), W[j].cpu())
+        assert np.array_equal(pool[j].cpu().numpy(), r["pool_idx"]), f"unit {u}: pool differs"
+        assert np.allclose(eps[j].cpu().numpy(), r["eps"], rtol=2e-5, atol=1e-30)
+        t2, r2, a2 = oracle.truncate(eps[j].cpu().numpy(), r["pool_idx"], b.n_apx, wl.N)
+        assert np.array_equal(tier[j].cpu().numpy(), t2), f"unit {u}: tiers differ on identical residuals"
+        assert np.array_equal(ret[j].cpu().numpy(), r2) and np.array_equal(apx[j].cpu().numpy(), a2)
+    # end to end (device scores -> device routing) against the oracle end to end
+    _assert_routing_agrees(oracle, sub, b, comp, K, V, W.cpu(), sc_o, list(range(len(units))))
+    # compaction is a pure gather of the device's own index lists
+    c = comp.cache
+    ri, ai = comp.ret_idx.long(), comp.apx_idx.long()
+    for j in range(len(units)):
+        assert torch.equal(c.ret_k[j, : b.n_ret], K[j][ri[j]]) and torch.equal(c.ret_v[j, : b.n_ret], V[j][ri[j]])
+        assert torch.equal(c.apx_k[j, : b.n_apx], K[j][ai[j]])
+        assert torch.equal(c.ret_pos[j, : b.n_ret], comp.ret_idx[j]) and torch.equal(c.apx_pos[j, : b.n_apx], comp.apx_idx[j])
+        assert 2 * b.n_ret + b.n_apx == 2 * b.n_budget_pairs
+    # decode steps over the mixed cache, appending the generated token each step
+    sk, sq, wt = synth.all_head_params(wl, DEV)
+    out = torch.empty(len(units), wl.group, wl.head_dim, dtype=torch.float32, device=DEV)
+    out_bf = torch.empty(len(units), wl.group, wl.head_dim, dtype=torch.bfloat16, device=DEV)
+    scale = 1.0 / np.sqrt(wl.head_dim)
+    for step in range(decode_steps):
+        q = synth.decode_q(wl, step, DEV, sq, units)
+        comp.decode(q, W, out)
+        comp.decode(q, W, out_bf)
+        torch.cuda.synchronize()
+        for j in range(len(units)):
+            o_tok, o_fac = oracle.attend(q[j].cpu(), c.ret_k[j, : c.n_ret].cpu(), c.ret_v[j, : c.n_ret].cpu(),
+                                         c.apx_k[j, : c.n_apx].cpu(), W[j].cpu(), scale)
+            assert np.max(np.abs(o_tok - o_fac)) <= 1e-9 * max(1.0, np.max(np.abs(o_tok)))
+            err = np.max(np.abs(out[j].cpu().double().numpy() - o_fac))
+            assert err <= 2e-2, f"decode step {step} unit {units[j]}: abs err {err}"
+            errb = np.abs(out_bf[j].cpu().double().numpy() - o_fac)
+            assert np.all(errb <= 2e-2 + 2.0 ** -8 * np.abs(o_fac))
+        kn, vn = synth.decode_kv(wl, step, DEV, sk, wt, units)
+        comp.append(kn, vn, wl.N + step)
+
+
+def test_pipeline_config0_all_units(oracle):
+    _run_pipeline_case(oracle, synth.WORKLOADS[0], 25, decode_steps=8)
+
+
+@pytest.mark.parametrize("percent", [10, 20, 40])
+def test_pipeline_config1_all_units(oracle, percent):
+    _run_pipeline_case(oracle, synth.WORKLOADS[1], percent, decode_steps=3)
+
+
+def test_pipeline_eviction_only_and_ragged(oracle):
+    wl = synth.shrink(synth.WORKLOADS[1], N=1531, n_kv_heads=2, n_q_heads=8, n_calib=2048)
+    _run_pipeline_case(oracle, wl, 30, n_a=0)          # no approximation tier: plain eviction
+    _run_pipeline_case(oracle, wl, 30)
+    wl8 = synth.shrink(synth.WORKLOADS[4], N=3000, n_layers=2, n_kv_heads=1, n_q_heads=8, n_calib=2048)
+    _run_pipeline_case(oracle, wl8, 12)                # g = 8, window 128
+
+
+def test_decode_degenerate_pools(oracle):
+    """Only retained rows, only key-only rows, and a single key."""
+    wl = synth.shrink(synth.WORKLOADS[1], N=512, n_kv_heads=2, n_q_heads=8, n_calib=1024)
+    K, V, _ = synth.context(wl, DEV)
+    W = calibrated_maps(wl).to(DEV)
+    sh = shape_of(wl)
+    _, sq, _ = synth.all_head_params(wl, DEV)
+    q = synth.decode_q(wl, 0, DEV, sq)
+    b = budget_of(wl, 50)
+    ws = vec.alloc_workspace(sh, b)
+    out = torch.empty(wl.units, wl.group, wl.head_dim, dtype=torch.float32, device=DEV)
+    scale = 1.0 / np.sqrt(wl.head_dim)
+    ipos = torch.arange(512, dtype=torch.int32, device=DEV).repeat(wl.units, 1).contiguous()
+    for n_ret, n_apx in [(512, 0), (0, 512), (1, 0), (0, 1), (300, 1), (1, 300), (257, 255)]:
+        cache = vec.Cache(K.clone(), V.clone(), K.flip(1).contiguous(), ipos, ipos.clone(), n_ret, n_apx)
+        vec.vector_decode_attn(sh, q, cache, W, out, 0, ws)
+        torch.cuda.synchronize()
+        for u in range(wl.units):
+            _, o = oracle.attend(q[u].cpu(), cache.ret_k[u, :n_ret].cpu(), cache.ret_v[u, :n_ret].cpu(),
+                                 cache.apx_k[u, :n_apx].cpu(), W[u].cpu(), scale)
+            assert np.max(np.abs(out[u].cpu().double().numpy() - o)) <= 2e-2, (n_ret, n_apx, u)
+
+
+def test_full_size_bench_configuration_sampled_units(oracle):
+    """Config 2 at full size in the launch shape the benchmark times; the oracle checks sampled units."""
+    wl = synth.WORKLOADS[2]
+    sample = [0, 131, 255]
+    # device pipeline over ALL 256 units; inputs of non-sampled units are the same law
+    K, V, Q = synth.context(wl, DEV)
+    W = calibrated_maps(wl).to(DEV)
+    sh = shape_of(wl)
+    b = budget_of(wl, 20)
+    comp = Compressor(sh, b, extra_rows=1, keep_eps=True)
+    comp.compress(Q, K, V, W)
+    torch.cuda.synchronize()
+    raw_o, sc_o = oracle_scores(oracle, wl, Q[sample].cpu(), K[sample].cpu())
+    ok, worst = score_close(comp.scores[sample].cpu().numpy(), sc_o, wl.group * wl.window)
+    assert ok, f"score off by {worst:.3g} x tolerance"
+    tier_all = comp.tier
+    # properties that hold at any size, on every unit
+    assert torch.all((tier_all == 1).sum(1) == b.n_apx) and torch.all((tier_all == 2).sum(1) == b.n_ret)
+    assert torch.all(tier_all[:, -wl.window:] > 0)
+    assert torch.all(comp.ret_idx[:, 1:] > comp.ret_idx[:, :-1]) and torch.all(comp.apx_idx[:, 1:] > comp.apx_idx[:, :-1])
+    emax_apx = torch.gather(comp.eps, 1, torch.searchsorted(comp.pool_idx, comp.apx_idx).clamp(max=b.n_pool - 1)).max(1).values
+    emin_ret = torch.gather(comp.eps, 1, torch.searchsorted(comp.pool_idx, comp.ret_idx).clamp(max=b.n_pool - 1)).min(1).values
+    assert torch.all(emax_apx <= emin_ret)
+    # sampled units against the oracle end to end
+    class _View:            # the slice of the compressor state the agreement check reads
+        tier = tier_all[sample]
+    sub = synth.shrink(wl, batch=1, n_layers=1, n_kv_heads=len(sample), n_q_heads=len(sample) * wl.group)
+    _assert_routing_agrees(oracle, sub, b, _View, K[sample], V[sample], W[sample].cpu(), sc_o, list(range(len(sample))))
+    _, sq, _ = synth.all_head_params(wl, DEV)
+    q = synth.decode_q(wl, 0, DEV, sq)
+    out = torch.empty(wl.units, wl.group, wl.head_dim, dtype=torch.float32, device=DEV)
+    comp.decode(q, W, out)
+    torch.cuda.synchronize()
+    c = comp.cache
+    for u in sample:
+        _, o = oracle.attend(q[u].cpu(), c.ret_k[u, : c.n_ret].cpu(), c.ret_v[u, : c.n_ret].cpu(),
+                             c.apx_k[u, : c.n_apx].cpu(), W[u].cpu(), 1.0 / np.sqrt(wl.head_dim))
+        assert np.max(np.abs(out[u].cpu().double().numpy() - o)) <= 2e-2

@@ -81,12 +81,15 @@ def test_plan_rejects_impossible_budgets(oracle):
     with pytest.raises(oracle.OracleError):
         oracle.plan_budget(100, 101, -1, 0)          # more pairs than tokens
     with pytest.raises(oracle.OracleError):
-        oracle.plan_budget(100, 10, 6, 0)            # approximation tier > half the budget
+        oracle.plan_budget(100, 10, 11, 0)           # more approximated pairs than the budget holds
     with pytest.raises(oracle.OracleError):
         oracle.plan_budget(100, 90, 20, 0)           # pool larger than the context
     with pytest.raises(oracle.OracleError):
         oracle.plan_budget(100, 10, -1, 32)          # pool smaller than the window
     assert oracle.plan_budget(100, 10, 0, 8).n_apx == 0
+    # Section 5.3 sweeps p_a up to 0.5 at p_c = 0.5: everything approximated, nothing retained
+    b = oracle.plan_budget(100, 50, 50, 0)
+    assert (b.n_pool, b.n_apx, b.n_ret, b.n_evict) == (100, 100, 0, 0)
 
 
 # ---------------------------------------------------------------------- calibrate
