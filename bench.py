@@ -1,0 +1,423 @@
+#!/usr/bin/env python
+"""Benchmark of the VECTOR hot path on B200: one JSON line per run.
+
+A step is one pass of the whole hot path over one synthetic batch: prefill-time
+compression of every (sequence, layer, KV head) unit (vector_score ->
+vector_route -> vector_compact) followed by the workload's decode steps of
+vector_decode_attn over the mixed cache, the retained pool growing by one
+generated token per step.  `value` is compressed tokens/s = batch * N divided by
+the mean device time of the compression calls; decode attention is reported as
+achieved HBM GB/s.  Inputs are seeded synthetic tensors resident in HBM before
+the timed region; `e2e` repeats the measurement through host buffers.
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--config C] [--impl reference]
+
+With --gpus N > 1 (under torchrun) every rank runs an independent replica of the
+workload on its own GPU: the path has no exchange step, so there is no collective
+on the data path and the aggregate is the sum over replicas (weak scaling).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import tempfile
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+METRIC = "compressed tokens/s (score+route+compact); decode-attn HBM GB/s vs peak"
+UNIT = "tokens/s"
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+
+
+def load_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        with open(p) as f:
+            d = json.load(f)
+        d["source"] = "measured"
+        return d
+    d = dict(FALLBACK_PEAKS)
+    d["source"] = "fallback"
+    return d
+
+
+# --------------------------------------------------------------------------- clocks
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+         "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.gpu = gpu_index
+        self.proc = None
+        self.path = None
+
+    def start(self):
+        try:
+            fd, self.path = tempfile.mkstemp(suffix=".csv")
+            os.close(fd)
+            self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
+                                          "-lms", "100", "-i", str(self.gpu)],
+                                         stdout=open(self.path, "w"), stderr=subprocess.DEVNULL)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if self.proc is None:
+            return out
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        try:
+            with open(self.path) as f:
+                for line in f:
+                    p = [x.strip() for x in line.split(",")]
+                    if len(p) < 9:
+                        continue
+                    try:
+                        sm.append(float(p[1])), mx.append(float(p[2]))
+                    except ValueError:
+                        continue
+                    for name, val in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown",
+                                          "sw_power_cap"), p[5:9]):
+                        if val.lower().startswith("active"):
+                            reasons.add(name)
+            os.unlink(self.path)
+        except Exception:
+            pass
+        if sm:
+            out.update(sm_mhz=statistics.median(sm), sm_max_mhz=max(mx), reasons=sorted(reasons), samples=len(sm))
+        return out
+
+
+# ------------------------------------------------------------------- oracle (CPU) arm
+def oracle_sample(wl, percent, n_units=1, decode_steps=2, device="cpu"):
+    """Times the oracle, as it stands, single-threaded, on `n_units` units of the workload.
+    Returns seconds per unit for compression and per decode step, and what the sample was."""
+    import numpy as np
+    import oracle
+    from paper_2605_23258_b200 import synth
+    oracle.build()
+    N, d = wl.N, wl.head_dim
+    Bp = N * percent // 100
+    b = oracle.plan_budget(N, Bp, -1, wl.window)
+    scale = 1.0 / np.sqrt(d)
+    units = [int(round(j * (wl.units - 1) / max(n_units - 1, 1))) for j in range(n_units)]
+    t_comp, t_dec = [], []
+    for u in units:
+        bb, l, h = wl.unit_coords(u)
+        params = synth.head_params(wl, l, h, device)
+        K, V = synth.unit_kv(wl, bb, l, h, device, params)
+        Q = synth.unit_qobs(wl, bb, l, h, device, params)
+        kc, vc = synth.calib_kv(wl, l, h, device, params)
+        W = oracle.calibrate(kc.cpu(), vc.cpu(), wl.lam)             # offline, not timed
+        W = np.asarray(__import__("torch").from_numpy(W).to(wl.torch_dtype).double().numpy())
+        Kc, Vc, Qc = K.cpu(), V.cpu(), Q.cpu()
+        t0 = time.perf_counter()
+        _, sc = oracle.score(Qc, Kc, scale, wl.pool_kernel)
+        r = oracle.route(sc.astype(np.float32), Kc, Vc, W, b.n_pool, b.n_apx)
+        rk, _ = oracle.gather_rows(Kc, r["ret_idx"])
+        rv, _ = oracle.gather_rows(Vc, r["ret_idx"])
+        ak, _ = oracle.gather_rows(Kc, r["apx_idx"])
+        t_comp.append(time.perf_counter() - t0)
+        _, sq, _ = params
+        g = __import__("torch").Generator().manual_seed(u)
+        for _ in range(decode_steps):
+            q = (__import__("torch").randn(wl.group, d, generator=g) * sq.cpu()).to(wl.torch_dtype)
+            t0 = time.perf_counter()
+            oracle.attend(q, rk, rv, ak, W, scale)
+            t_dec.append(time.perf_counter() - t0)
+    return {"compress_s_per_unit": statistics.mean(t_comp), "decode_s_per_unit_step": statistics.mean(t_dec),
+            "units": units, "budget": b}
+
+
+def run_reference(args, wl, percent):
+    """--impl reference: the CPU oracle, timed on the host cores, same metric and config."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return 0
+    steps = max(args.steps, 1)
+    for _ in range(min(args.warmup, 1)):
+        oracle_sample(wl, percent, 1, 1)
+    t0 = time.perf_counter()
+    res = [oracle_sample(wl, percent, 1, 2) for _ in range(min(steps, 3))]
+    wall = time.perf_counter() - t0
+    per_unit = statistics.mean(r["compress_s_per_unit"] for r in res)
+    dec_unit = statistics.mean(r["decode_s_per_unit_step"] for r in res)
+    t_compress_all = per_unit * wl.units                      # one core, every unit in turn
+    value = wl.batch * wl.N / t_compress_all
+    b = res[0]["budget"]
+    dec_bytes = wl.units * (2 * b.n_ret + b.n_apx) * wl.head_dim * (2 if wl.dtype == "bf16" else 4)
+    sample = (f"unit {res[0]['units'][0]} of {wl.units} per step ({min(steps, 3)} timed samples): "
+              f"score+route+compact and 2 decode steps, single thread; whole-workload time = per-unit time x {wl.units}")
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": 0, "steps": min(steps, 3),
+        "warmup": min(args.warmup, 1), "ms_per_step": 1e3 * (t_compress_all + dec_unit * wl.units * wl.decode_steps),
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": wl.name, "budget_percent": percent, "batch": wl.batch, "N": wl.N,
+                   "units": wl.units, "extrapolated_from_units": 1},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": sample},
+        "decode": {"gbs": dec_bytes / (dec_unit * wl.units) / 1e9, "s_per_step": dec_unit * wl.units},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0, "wall_s": wall,
+    }
+    print(json.dumps(line))
+    return 0
+
+
+# ----------------------------------------------------------------------------- GPU arm
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=5)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--config", type=int, default=2, help="workload 1..4 (default 2: 32-layer Llama-3-8B shape)")
+    ap.add_argument("--budget", type=int, default=None, help="budget percent (default: the workload's)")
+    ap.add_argument("--decode-steps", type=int, default=None)
+    ap.add_argument("--impl", default="vector", choices=["vector", "reference"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true")
+    args = ap.parse_args()
+
+    from paper_2605_23258_b200 import synth
+    wl = synth.WORKLOADS[args.config]
+    percent = args.budget if args.budget is not None else (20 if args.config == 1 else wl.budget_percents[0])
+    if args.impl == "reference":
+        return run_reference(args, wl, percent)
+
+    import torch
+    import paper_2605_23258_b200 as vec
+    from paper_2605_23258_b200.pipeline import Compressor, calibrate_maps
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    dev = f"cuda:{local}"
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device(dev))
+    vec.load_library()
+    W_warm = max(args.warmup, 3)
+    K_steps = max(args.steps, 1)
+    D = args.decode_steps if args.decode_steps is not None else wl.decode_steps
+    es = 2 if wl.dtype == "bf16" else 4
+    U, N, d, g, w = wl.units, wl.N, wl.head_dim, wl.group, wl.window
+
+    # ---- setup (untimed): inputs resident in HBM, maps calibrated offline
+    Kt, Vt, Qt = synth.context(wl, dev)
+    pairs = []
+    for l in range(wl.n_layers):
+        for h in range(wl.n_kv_heads):
+            kc, vc = synth.calib_kv(wl, l, h, dev)
+            pairs.append((kc.cpu(), vc.cpu()))
+    Wm = calibrate_maps(pairs, wl.lam).to(wl.torch_dtype).to(dev)
+    del pairs
+    shape = vec.Shape(wl.batch, wl.n_layers, wl.n_q_heads, wl.n_kv_heads, d,
+                      vec.VECTOR_BF16 if wl.dtype == "bf16" else vec.VECTOR_F32, w, wl.pool_kernel)
+    budget = vec.vector_plan_budget(N, N * percent // 100, -1, w)
+    comp = Compressor(shape, budget, extra_rows=D)
+    sk, sq, wt = synth.all_head_params(wl, dev)
+    n_q = min(D, 16)
+    qs = [synth.decode_q(wl, t, dev, sq) for t in range(n_q)]
+    # generated tokens are kept in full: their rows sit behind the retained pool from the start
+    # (compaction never touches rows >= n_ret), so a decode step only bumps the row count
+    for t in range(D):
+        kn, vn = synth.decode_kv(wl, t, dev, sk, wt)
+        comp.cache.ret_k[:, budget.n_ret + t] = kn
+        comp.cache.ret_v[:, budget.n_ret + t] = vn
+        comp.cache.ret_pos[:, budget.n_ret + t] = N + t
+    out = torch.empty(U, g, d, dtype=wl.torch_dtype, device=dev)
+    torch.cuda.synchronize()
+
+    ev = lambda: torch.cuda.Event(enable_timing=True)
+
+    def one_step(marks=None):
+        """The whole hot path once; `marks` collects events at the call boundaries."""
+        if marks is not None:
+            marks.append(ev()); marks[-1].record()
+        comp.score(Qt, Kt)
+        if marks is not None:
+            marks.append(ev()); marks[-1].record()
+        comp.route(Kt, Vt, Wm)
+        if marks is not None:
+            marks.append(ev()); marks[-1].record()
+        comp.compact(Kt, Vt)
+        if marks is not None:
+            marks.append(ev()); marks[-1].record()
+        for t in range(D):
+            comp.cache.n_ret = budget.n_ret + t
+            comp.decode(qs[t % n_q], Wm, out)
+        if marks is not None:
+            marks.append(ev()); marks[-1].record()
+
+    def barrier():
+        if world > 1:
+            import torch.distributed as dist
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(W_warm):
+        one_step()
+    barrier()
+    sampler = ClockSampler(local)
+    sampler.start()
+    all_marks = []
+    t_begin, t_end = ev(), ev()
+    barrier()
+    t_begin.record()
+    for _ in range(K_steps):
+        m = []
+        one_step(m)
+        all_marks.append(m)
+    t_end.record()
+    barrier()
+    clocks = sampler.stop()
+    total_ms = t_begin.elapsed_time(t_end)
+    phase = {"score": [], "route": [], "compact": [], "decode": []}
+    for m in all_marks:
+        for name, i in (("score", 0), ("route", 1), ("compact", 2), ("decode", 3)):
+            phase[name].append(m[i].elapsed_time(m[i + 1]))
+    ms = {k: statistics.mean(v) for k, v in phase.items()}
+    compress_ms = ms["score"] + ms["route"] + ms["compact"]
+    if world > 1:
+        import torch.distributed as dist
+        t = torch.tensor([total_ms, compress_ms, ms["decode"]], device=dev, dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        total_ms, compress_ms, dec_ms_max = t.tolist()
+    else:
+        dec_ms_max = ms["decode"]
+
+    # ---- algorithmic work (per step, one replica)
+    n_ret, n_apx, n_pool = budget.n_ret, budget.n_apx, budget.n_pool
+    score_flops = 4.0 * g * w * N * d * U
+    score_bytes = U * (N * d * es + N * 4)
+    resid_bytes = U * (2 * n_pool * d * es) + U * d * d * es
+    compact_bytes = 2 * U * (2 * n_ret + n_apx) * d * es
+    dec_rows = sum(2 * (n_ret + t) + n_apx for t in range(D))
+    decode_bytes = U * dec_rows * d * es + D * (Wm.numel() * es + 2 * U * g * d * es)
+    peaks = load_peaks()
+    hbm, tf = peaks["hbm_gbs"], peaks["bf16_tflops_sustained"]
+    kernels = [
+        {"kernel": "vector_score (logit passes)", "bound": "tensor", "achieved": score_flops / (ms["score"] * 1e-3) / 1e12,
+         "peak": tf, "unit": "TFLOP/s", "ms": ms["score"], "hbm_gbs": score_bytes / (ms["score"] * 1e-3) / 1e9},
+        {"kernel": "vector_route (select + residual + truncate)", "bound": "hbm",
+         "achieved": (resid_bytes + U * N * 4 * 2) / (ms["route"] * 1e-3) / 1e9, "peak": hbm, "unit": "GB/s", "ms": ms["route"]},
+        {"kernel": "vector_compact", "bound": "hbm", "achieved": compact_bytes / (ms["compact"] * 1e-3) / 1e9,
+         "peak": hbm, "unit": "GB/s", "ms": ms["compact"]},
+        {"kernel": "vector_decode_attn (split + merge)", "bound": "hbm",
+         "achieved": decode_bytes / (ms["decode"] * 1e-3) / 1e9, "peak": hbm, "unit": "GB/s", "ms": ms["decode"]},
+    ]
+    for k in kernels:
+        k["frac"] = k["achieved"] / k["peak"]
+        k["traffic"] = None
+    dominant = max(kernels, key=lambda k: k["ms"])
+    roofline = {k: dominant[k] for k in ("bound", "achieved", "peak", "unit", "frac", "traffic")}
+    roofline["kernel"] = dominant["kernel"]
+    roofline["peak_source"] = f"{peaks['source']} ({'copy GB/s' if dominant['bound'] == 'hbm' else 'sustained bf16 TFLOP/s'})"
+
+    # ---- end to end through host buffers (rank 0 semantics on every rank; reported from rank 0)
+    e2e = None
+    if not args.no_e2e:
+        hK = torch.empty(Kt.shape, dtype=Kt.dtype, pin_memory=True).copy_(Kt)
+        hV = torch.empty(Vt.shape, dtype=Vt.dtype, pin_memory=True).copy_(Vt)
+        hQ = torch.empty(Qt.shape, dtype=Qt.dtype, pin_memory=True).copy_(Qt)
+        h_tier = torch.empty(comp.tier.shape, dtype=torch.uint8, pin_memory=True)
+        h_ret = torch.empty(comp.ret_idx.shape, dtype=torch.int32, pin_memory=True)
+        h_apx = torch.empty(comp.apx_idx.shape, dtype=torch.int32, pin_memory=True)
+        hq = torch.empty(qs[0].shape, dtype=qs[0].dtype, pin_memory=True).copy_(qs[0])
+        h_out = torch.empty(out.shape, dtype=out.dtype, pin_memory=True)
+        dq = torch.empty_like(qs[0])
+
+        def e2e_step():
+            Kt.copy_(hK, non_blocking=True); Vt.copy_(hV, non_blocking=True); Qt.copy_(hQ, non_blocking=True)
+            comp.compress(Qt, Kt, Vt, Wm)
+            h_tier.copy_(comp.tier, non_blocking=True)
+            h_ret.copy_(comp.ret_idx, non_blocking=True)
+            h_apx.copy_(comp.apx_idx, non_blocking=True)
+
+        def e2e_decode():
+            dq.copy_(hq, non_blocking=True)
+            comp.decode(dq, Wm, out)
+            h_out.copy_(out, non_blocking=True)
+
+        e2e_step(); torch.cuda.synchronize()
+        n_e = max(2, min(K_steps, 3))
+        a, b_ = ev(), ev()
+        barrier(); a.record()
+        for _ in range(n_e):
+            e2e_step()
+        b_.record(); barrier()
+        e_ms = a.elapsed_time(b_) / n_e
+        a, b_ = ev(), ev()
+        a.record()
+        for _ in range(20):
+            e2e_decode()
+        b_.record(); torch.cuda.synchronize()
+        ed_ms = a.elapsed_time(b_) / 20
+        if world > 1:
+            import torch.distributed as dist
+            t = torch.tensor([e_ms, ed_ms], device=dev, dtype=torch.float64)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            e_ms, ed_ms = t.tolist()
+        h2d = (hK.numel() + hV.numel() + hQ.numel()) * es
+        d2h = h_tier.numel() + (h_ret.numel() + h_apx.numel()) * 4
+        e2e = {"value": world * wl.batch * N / (e_ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
+               "d2h_bytes_per_step": d2h, "ms_per_step": e_ms,
+               "decode_step_us": ed_ms * 1e3, "decode_h2d_bytes": hq.numel() * es, "decode_d2h_bytes": h_out.numel() * es}
+        del hK, hV, hQ
+
+    if rank != 0:
+        if world > 1:
+            import torch.distributed as dist
+            dist.destroy_process_group()
+        return 0
+
+    cpu = None
+    if not args.no_cpu_baseline and world == 1:
+        r = oracle_sample(wl, percent, 1, 2)
+        t_all = r["compress_s_per_unit"] * U
+        cpu = {"value": wl.batch * N / t_all, "unit": UNIT, "cores": 1, "kind": "oracle",
+               "sample": f"unit {r['units'][0]} of {U}: score+route+compact took {r['compress_s_per_unit']:.2f} s single-threaded; "
+                         f"whole-workload time = x{U}; one decode step of that unit {r['decode_s_per_unit_step'] * 1e3:.1f} ms"}
+
+    kernels_per_step = 8 + 2 * D
+    line = {
+        "metric": METRIC, "value": world * wl.batch * N / (compress_ms * 1e-3), "unit": UNIT, "n_gpus": world,
+        "steps": K_steps, "warmup": W_warm, "ms_per_step": total_ms / K_steps, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "bf16" if wl.dtype == "bf16" else "f32", "data": "synthetic",
+        "config": {"workload": wl.name, "budget_percent": percent, "batch": wl.batch, "N": N, "units": U,
+                   "layers": wl.n_layers, "q_heads": wl.n_q_heads, "kv_heads": wl.n_kv_heads, "head_dim": d,
+                   "window": w, "pool_kernel": wl.pool_kernel, "decode_steps_per_step": D,
+                   "n_ret": n_ret, "n_apx": n_apx, "n_pool": n_pool,
+                   "l2": "inputs larger than L2 (K+V %.2f GB, compacted cache %.2f GB per replica)" %
+                         (2 * U * N * d * es / 1e9, U * (2 * n_ret + n_apx) * d * es / 1e9),
+                   "parallelism": "replicas only" if world > 1 else "single GPU"},
+        "compress_ms": compress_ms, "phase_ms": ms,
+        "decode": {"gbs": decode_bytes / (dec_ms_max * 1e-3) / 1e9, "frac_of_measured_copy": decode_bytes / (dec_ms_max * 1e-3) / 1e9 / hbm,
+                   "frac_of_8tbs": decode_bytes / (dec_ms_max * 1e-3) / 1e9 / 8000.0, "us_per_step": dec_ms_max * 1e3 / D,
+                   "tokens_per_s": world * wl.batch * D / (dec_ms_max * 1e-3), "bytes_per_step": decode_bytes / D},
+        "roofline": roofline, "roofline_kernels": kernels, "cpu_baseline": cpu, "e2e": e2e,
+        "gpu_launches": kernels_per_step * K_steps, "clocks": clocks,
+    }
+    print(json.dumps(line))
+    if world > 1:
+        import torch.distributed as dist
+        dist.destroy_process_group()
+    return 0
+
+
+if __name__ == "__main__":
+    sys.exit(main())
