@@ -206,6 +206,39 @@ VECTOR_API vector_status vector_decode_attn(const vector_shape* shape, const voi
                                  const void* W, void* out, int32_t out_dtype, int32_t mode,
                                  void* ws, size_t ws_bytes, void* stream);
 
+/*
+ * Allocation-free variant of vector_decode_attn (the paper has no counterpart:
+ * this entry point exists for the integration, not for the method).
+ *
+ * Meant for callers that cannot obtain device memory at the time of the call:
+ * a serving process whose own pool already owns the whole device so that a
+ * later cudaMalloc fails, or a latency-critical decode loop in which the
+ * device-wide stall of a cudaMalloc/cudaFree is not acceptable and no spare
+ * workspace buffer was planned.  The split-KV partial results, which
+ * vector_decode_attn keeps in the caller's workspace, live here in a fixed
+ * array of VECTOR_STATIC_SCRATCH_BYTES inside the library's device image; every
+ * GPU on which the library is loaded holds that much memory until the process
+ * exits.  The call itself performs no cudaMalloc, cudaFree or other allocating
+ * routine.  Inputs and outputs are passed exactly as for vector_decode_attn.
+ *
+ *  - Limit: shapes whose partial results need more than VECTOR_STATIC_SCRATCH_BYTES
+ *    (vector_decode_scratch_bytes(shape) reports the need) are rejected with
+ *    VECTOR_ERR_WORKSPACE; use vector_decode_attn with your own workspace then.
+ *  - The first call on each device looks up the array's device address (with
+ *    that device current).  Make that first call during start-up, before any
+ *    stream capture begins.
+ *  - All calls on a device share the one array, and it keeps whatever the last
+ *    call left there.  Nothing in it has to start at zero: each call overwrites
+ *    every partial record before reading it.  Two calls that overlap on the GPU
+ *    (different streams, no ordering between them) race on the array and give
+ *    undefined results; order them on one stream or with events.
+ */
+#define VECTOR_STATIC_SCRATCH_BYTES (16u << 20)
+VECTOR_API size_t vector_decode_scratch_bytes(const vector_shape* shape);
+VECTOR_API vector_status vector_decode_attn_static(const vector_shape* shape, const void* q,
+                                                   const vector_cache* cache, const void* W, void* out,
+                                                   int32_t out_dtype, int32_t mode, void* stream);
+
 #ifdef __cplusplus
 }
 #endif

@@ -143,6 +143,10 @@ def load_library() -> ctypes.CDLL:
     lib.vector_route.argtypes = [SP, BP, P, P, P, P, P, P, P, P, P, P, SZ, P]
     lib.vector_compact.argtypes = [SP, BP, P, P, P, P, CP, P]
     lib.vector_decode_attn.argtypes = [SP, P, CP, P, P, I32, I32, P, SZ, P]
+    lib.vector_decode_scratch_bytes.restype = SZ
+    lib.vector_decode_scratch_bytes.argtypes = [SP]
+    lib.vector_decode_attn_static.argtypes = [SP, P, CP, P, P, I32, I32, P]
+    lib.vector_decode_attn_static.restype = ctypes.c_int
     for name in ("vector_plan_budget", "vector_calibrate", "vector_score", "vector_pool_select",
                  "vector_residual", "vector_truncate", "vector_route", "vector_compact", "vector_decode_attn"):
         getattr(lib, name).restype = ctypes.c_int
@@ -293,3 +297,30 @@ def vector_decode_attn(shape: Shape, q, cache: Cache, W, out, mode: int = 0, ws=
                                            ctypes.byref(c), _dev(W, shape.torch_dtype, "W"), _dev(out, None, "out"),
                                            out_dt, mode, wp, wn, _stream(stream))
     _check(rc, "vector_decode_attn")
+
+
+VECTOR_STATIC_SCRATCH_BYTES = 16 << 20
+
+
+def vector_decode_scratch_bytes(shape: Shape) -> int:
+    """Bytes of split-KV scratch a decode call of this shape needs (0 for an unsupported shape)."""
+    return int(load_library().vector_decode_scratch_bytes(ctypes.byref(shape._c())))
+
+
+def vector_decode_attn_static(shape: Shape, q, cache: Cache, W, out, mode: int = 0, stream=None):
+    """vector_decode_attn without a workspace argument and without any allocation.
+
+    For callers that cannot get device memory when they call (their own pool owns the
+    device, or a cudaMalloc stall is unacceptable inside the decode loop): the partial
+    results go to a fixed VECTOR_STATIC_SCRATCH_BYTES array inside the library.  Shapes
+    that need more raise VectorError (workspace).  Calls on one device share that array,
+    so calls that overlap on the GPU race; make the first call per device at start-up.
+    """
+    c = cache._c()
+    if out.dtype not in (torch.float32, torch.bfloat16):
+        raise ValueError("out must be fp32 or bf16")
+    out_dt = VECTOR_BF16 if out.dtype == torch.bfloat16 else VECTOR_F32
+    rc = load_library().vector_decode_attn_static(ctypes.byref(shape._c()), _dev(q, shape.torch_dtype, "q"),
+                                                  ctypes.byref(c), _dev(W, shape.torch_dtype, "W"),
+                                                  _dev(out, None, "out"), out_dt, mode, _stream(stream))
+    _check(rc, "vector_decode_attn_static")

@@ -8,6 +8,8 @@
 //   split  grid (n_splits, U): online softmax over a slice of the logical key
 //          range [0, n_ret + n_apx); emits (m, l, acc_v[d], acc_k[d]) per head
 //   merge  grid (U): combines the splits, applies W to acc_k, normalises
+#include <mutex>
+
 #include "common.cuh"
 #include "internal.h"
 
@@ -213,4 +215,53 @@ extern "C" vector_status vector_decode_attn(const vector_shape* shape, const voi
                           : launch_decode_g<float, 128>(dm, q, cache, W, out, out_dtype, partial, st);
     return dm.d == 64 ? launch_decode_g<__nv_bfloat16, 64>(dm, q, cache, W, out, out_dtype, partial, st)
                       : launch_decode_g<__nv_bfloat16, 128>(dm, q, cache, W, out, out_dtype, partial, st);
+}
+
+// ---------------------------------------------------------------------------
+// Allocation-free variant: the split-KV partial records live in a fixed array
+// of the library's device image instead of a caller-provided workspace.
+namespace vec {
+
+static __device__ __align__(256) unsigned char g_decode_scratch[VECTOR_STATIC_SCRATCH_BYTES];
+
+constexpr int kMaxDevices = 64;
+static std::mutex g_scratch_mu;
+static void* g_scratch_addr[kMaxDevices] = {};
+
+// In host code `g_decode_scratch` is only a handle; the address a kernel can use
+// comes from cudaGetSymbolAddress, once per device, with that device current.
+static vector_status static_scratch_address(void** out) {
+    int dev = -1;
+    VEC_CUDA_CHECK(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= kMaxDevices) return VECTOR_ERR_UNSUPPORTED;
+    std::lock_guard<std::mutex> lock(g_scratch_mu);
+    if (!g_scratch_addr[dev]) {
+        void* p = nullptr;
+        VEC_CUDA_CHECK(cudaGetSymbolAddress(&p, g_decode_scratch));
+        if (!p) return VECTOR_ERR_CUDA;
+        g_scratch_addr[dev] = p;
+    }
+    *out = g_scratch_addr[dev];
+    return VECTOR_OK;
+}
+
+}  // namespace vec
+
+extern "C" size_t vector_decode_scratch_bytes(const vector_shape* shape) {
+    Dims dm;
+    if (check_shape(shape, &dm) != VECTOR_OK) return 0;
+    return decode_ws_bytes(dm);
+}
+
+extern "C" vector_status vector_decode_attn_static(const vector_shape* shape, const void* q,
+                                                   const vector_cache* cache, const void* W, void* out,
+                                                   int32_t out_dtype, int32_t mode, void* stream) {
+    Dims dm;
+    vector_status rc = check_shape(shape, &dm);
+    if (rc != VECTOR_OK) return rc;
+    if (decode_ws_bytes(dm) > (size_t)VECTOR_STATIC_SCRATCH_BYTES) return VECTOR_ERR_WORKSPACE;
+    void* scratch = nullptr;
+    if ((rc = static_scratch_address(&scratch)) != VECTOR_OK) return rc;
+    return vector_decode_attn(shape, q, cache, W, out, out_dtype, mode, scratch,
+                              (size_t)VECTOR_STATIC_SCRATCH_BYTES, stream);
 }
