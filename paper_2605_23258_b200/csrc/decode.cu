@@ -11,6 +11,7 @@
 #include <mutex>
 
 #include "common.cuh"
+#include "decode_bf16.cuh"
 #include "internal.h"
 
 namespace vec {
@@ -179,6 +180,31 @@ static vector_status launch_decode(const Dims& dm, const void* q, const vector_c
     return VECTOR_OK;
 }
 
+// bf16, head_dim 128: tensor-core split kernel, generic merge.
+static vector_status launch_decode_bf16_d128(const Dims& dm, const void* q, const vector_cache* ch, const void* W,
+                                             void* out, int out_dtype, float* partial, cudaStream_t st) {
+    using T = __nv_bfloat16;
+    static bool configured = false;
+    if (!configured) {
+        VEC_CUDA_CHECK(cudaFuncSetAttribute(dbf::decode_split_bf16_d128,
+                                            cudaFuncAttributeMaxDynamicSharedMemorySize, dbf::SMEM_BYTES));
+        configured = true;
+    }
+    const int n_splits = decode_num_splits(dm.U, ch->n_ret + ch->n_apx);
+    dim3 grid(n_splits, dm.U);
+    dbf::decode_split_bf16_d128<<<grid, 128, dbf::SMEM_BYTES, st>>>(
+        (const T*)q, (const T*)ch->ret_k, (const T*)ch->ret_v, (const T*)ch->apx_k, ch->cap_ret, ch->cap_apx,
+        (int)ch->n_ret, (int)ch->n_apx, dm.g, dm.scale * 1.4426950408889634f, partial);
+    VEC_LAUNCH_CHECK();
+    if (out_dtype == VECTOR_F32)
+        decode_merge_generic<T, float, 128><<<dm.U, 128, 0, st>>>(partial, (const T*)W, dm.LH, dm.g, n_splits,
+                                                                 (float*)out);
+    else
+        decode_merge_generic<T, T, 128><<<dm.U, 128, 0, st>>>(partial, (const T*)W, dm.LH, dm.g, n_splits, (T*)out);
+    VEC_LAUNCH_CHECK();
+    return VECTOR_OK;
+}
+
 template <typename T, int D>
 static vector_status launch_decode_g(const Dims& dm, const void* q, const vector_cache* ch, const void* W,
                                      void* out, int out_dtype, float* partial, cudaStream_t st) {
@@ -214,7 +240,7 @@ extern "C" vector_status vector_decode_attn(const vector_shape* shape, const voi
         return dm.d == 64 ? launch_decode_g<float, 64>(dm, q, cache, W, out, out_dtype, partial, st)
                           : launch_decode_g<float, 128>(dm, q, cache, W, out, out_dtype, partial, st);
     return dm.d == 64 ? launch_decode_g<__nv_bfloat16, 64>(dm, q, cache, W, out, out_dtype, partial, st)
-                      : launch_decode_g<__nv_bfloat16, 128>(dm, q, cache, W, out, out_dtype, partial, st);
+                      : launch_decode_bf16_d128(dm, q, cache, W, out, out_dtype, partial, st);
 }
 
 // ---------------------------------------------------------------------------

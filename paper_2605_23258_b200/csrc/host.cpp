@@ -78,7 +78,7 @@ size_t select_ws_bytes(const Dims& D, const vector_budget& b) {
 }
 
 int decode_num_splits(int U, int64_t rows) {
-    int64_t want = (4 * 148 + U - 1) / U;
+    int64_t want = (8 * 148 + U - 1) / U;
     int64_t max_by_rows = (rows + 255) / 256;   // at least 256 rows per split
     if (want > max_by_rows) want = max_by_rows;
     if (want > 64) want = 64;
