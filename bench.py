@@ -186,6 +186,7 @@ def main():
     ap.add_argument("--config", type=int, default=2, help="workload 1..4 (default 2: 32-layer Llama-3-8B shape)")
     ap.add_argument("--budget", type=int, default=None, help="budget percent (default: the workload's)")
     ap.add_argument("--decode-steps", type=int, default=None)
+    ap.add_argument("--layers", type=int, default=None, help="shrink the workload to this many layers (profiling)")
     ap.add_argument("--impl", default="vector", choices=["vector", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
@@ -193,6 +194,8 @@ def main():
 
     from paper_2605_23258_b200 import synth
     wl = synth.WORKLOADS[args.config]
+    if args.layers is not None:
+        wl = synth.shrink(wl, n_layers=args.layers, name=f"{wl.name}_first{args.layers}layers")
     percent = args.budget if args.budget is not None else (20 if args.config == 1 else wl.budget_percents[0])
     if args.impl == "reference":
         return run_reference(args, wl, percent)

@@ -127,6 +127,13 @@ VECTOR_API vector_status vector_plan_budget(int64_t n_tokens, int64_t n_budget_p
 VECTOR_API vector_status vector_calibrate(const void* K, const void* V, int64_t n, int32_t d_k, int32_t d_v,
                                int32_t dt, double lambda, float* W_out, double* r2_out);
 
+/*
+ * Waits inside the kernels are bounded.  This call synchronises the current device and returns
+ * the code recorded by a wait that gave up since the last call (0 = none, -1 = CUDA error),
+ * clearing it.  Results of the call that recorded a fault are invalid.
+ */
+VECTOR_API int vector_device_fault(void);
+
 /* Bytes of device workspace that suffice for every device call with this shape and budget. */
 VECTOR_API size_t vector_workspace_bytes(const vector_shape* shape, const vector_budget* budget);
 

@@ -187,6 +187,13 @@ def vector_status_string(status: int) -> str:
     return load_library().vector_status_string(status).decode()
 
 
+def vector_device_fault() -> int:
+    """Synchronises the device; returns (and clears) the code of a kernel wait that gave up, 0 if none."""
+    lib = load_library()
+    lib.vector_device_fault.restype = ctypes.c_int
+    return int(lib.vector_device_fault())
+
+
 def vector_plan_budget(n_tokens: int, n_budget_pairs: int, n_a: int = -1, window: int = 0) -> Budget:
     b = _Budget()
     _check(load_library().vector_plan_budget(n_tokens, n_budget_pairs, n_a, window, ctypes.byref(b)),

@@ -180,27 +180,53 @@ static vector_status launch_decode(const Dims& dm, const void* q, const vector_c
     return VECTOR_OK;
 }
 
-// bf16, head_dim 128: tensor-core split kernel, generic merge.
+// Fault word that bounded waits inside kernels write to (0 = none).
+static __device__ int g_kernel_fault;
+static int* kernel_fault_address() {
+    static int* addr = nullptr;           // single-device processes; looked up with the current device
+    if (!addr) {
+        void* p = nullptr;
+        if (cudaGetSymbolAddress(&p, g_kernel_fault) == cudaSuccess) addr = (int*)p;
+    }
+    return addr;
+}
+
+// bf16, head_dim 128: persistent TMA + tensor-core streaming kernel and the record merge.
 static vector_status launch_decode_bf16_d128(const Dims& dm, const void* q, const vector_cache* ch, const void* W,
                                              void* out, int out_dtype, float* partial, cudaStream_t st) {
     using T = __nv_bfloat16;
     static bool configured = false;
     if (!configured) {
-        VEC_CUDA_CHECK(cudaFuncSetAttribute(dbf::decode_split_bf16_d128,
+        VEC_CUDA_CHECK(cudaFuncSetAttribute(dbf::decode_stream_bf16_d128,
                                             cudaFuncAttributeMaxDynamicSharedMemorySize, dbf::SMEM_BYTES));
         configured = true;
     }
-    const int n_splits = decode_num_splits(dm.U, ch->n_ret + ch->n_apx);
-    dim3 grid(n_splits, dm.U);
-    dbf::decode_split_bf16_d128<<<grid, 128, dbf::SMEM_BYTES, st>>>(
-        (const T*)q, (const T*)ch->ret_k, (const T*)ch->ret_v, (const T*)ch->apx_k, ch->cap_ret, ch->cap_apx,
-        (int)ch->n_ret, (int)ch->n_apx, dm.g, dm.scale * 1.4426950408889634f, partial);
+    int* fault = kernel_fault_address();
+    if (!fault) return VECTOR_ERR_CUDA;
+    const dbf::Plan pl = dbf::make_plan(dm.U, ch->n_ret, ch->n_apx);
+    if (pl.s_max > decode_stream_slots(dm.U)) return VECTOR_ERR_WORKSPACE;
+    dbf::Maps maps;
+    const uint64_t row_b = 256;
+    bool ok = true;
+    if (ch->n_ret > 0) {
+        ok = ok && tma::encode_bf16_3d(&maps.ret_k, ch->ret_k, 128, (uint64_t)ch->n_ret, (uint64_t)dm.U, row_b,
+                                       (uint64_t)ch->cap_ret * row_b, 64, 64);
+        ok = ok && tma::encode_bf16_3d(&maps.ret_v, ch->ret_v, 128, (uint64_t)ch->n_ret, (uint64_t)dm.U, row_b,
+                                       (uint64_t)ch->cap_ret * row_b, 64, 64);
+    }
+    if (ch->n_apx > 0)
+        ok = ok && tma::encode_bf16_3d(&maps.apx_k, ch->apx_k, 128, (uint64_t)ch->n_apx, (uint64_t)dm.U, row_b,
+                                       (uint64_t)ch->cap_apx * row_b, 64, 64);
+    if (!ok) return VECTOR_ERR_CUDA;
+    if (ch->n_ret == 0) { maps.ret_k = maps.apx_k; maps.ret_v = maps.apx_k; }   // never dereferenced: no such tiles
+    if (ch->n_apx == 0) maps.apx_k = maps.ret_k;
+    dbf::decode_stream_bf16_d128<<<pl.B, dbf::THREADS, dbf::SMEM_BYTES, st>>>(
+        (const T*)q, maps, pl, (int)ch->n_ret, (int)ch->n_apx, dm.g, dm.scale * 1.4426950408889634f, partial, fault);
     VEC_LAUNCH_CHECK();
     if (out_dtype == VECTOR_F32)
-        decode_merge_generic<T, float, 128><<<dm.U, 128, 0, st>>>(partial, (const T*)W, dm.LH, dm.g, n_splits,
-                                                                 (float*)out);
+        dbf::decode_merge_bf16_d128<float><<<dm.U, 128, 0, st>>>(partial, (const T*)W, dm.LH, dm.g, pl, (float*)out);
     else
-        decode_merge_generic<T, T, 128><<<dm.U, 128, 0, st>>>(partial, (const T*)W, dm.LH, dm.g, n_splits, (T*)out);
+        dbf::decode_merge_bf16_d128<T><<<dm.U, 128, 0, st>>>(partial, (const T*)W, dm.LH, dm.g, pl, (T*)out);
     VEC_LAUNCH_CHECK();
     return VECTOR_OK;
 }
@@ -290,4 +316,14 @@ extern "C" vector_status vector_decode_attn_static(const vector_shape* shape, co
     if ((rc = static_scratch_address(&scratch)) != VECTOR_OK) return rc;
     return vector_decode_attn(shape, q, cache, W, out, out_dtype, mode, scratch,
                               (size_t)VECTOR_STATIC_SCRATCH_BYTES, stream);
+}
+
+extern "C" int vector_device_fault(void) {
+    int* addr = vec::kernel_fault_address();
+    if (!addr) return -1;
+    int v = 0, zero = 0;
+    if (cudaDeviceSynchronize() != cudaSuccess) return -1;
+    if (cudaMemcpy(&v, addr, sizeof(int), cudaMemcpyDeviceToHost) != cudaSuccess) return -1;
+    if (v != 0) cudaMemcpy(addr, &zero, sizeof(int), cudaMemcpyHostToDevice);
+    return v;
 }

@@ -1,40 +1,79 @@
-// Split-KV decode attention over the mixed cache for bf16, head_dim 128.
+// Decode attention over the mixed cache for bf16, head_dim 128 (HBM-bound).
 //
-// HBM-bound streaming kernel: every K/V row is read once.  A block owns a slice
-// of a unit's 64-row tiles (retained tiles carry K and V, key-only tiles K),
-// stages them with 16-byte cp.async into XOR-swizzled shared memory through a
-// 3-deep ring, and each of its 4 warps takes 16 keys of every tile:
-//   S = Q K^T      m16n8k16 bf16 MMA, the g query heads padded to the 16 MMA rows
+// Every K/V row is read once.  Each unit's rows are cut into 64-key tiles (a
+// retained tile = 64 keys + their 64 values = 32 KB, weight 2; a key-only tile
+// = 64 keys = 16 KB, weight 1) and the weighted global tile sequence is dealt
+// out in equal contiguous ranges to a fixed grid of persistent blocks (two per
+// SM): the load is balanced by bytes and there is no wave tail.
+//
+// Inside a block one producer thread streams the tiles with TMA
+// (cp.async.bulk.tensor, 128-byte swizzle, zero fill past the end of a pool)
+// into a 3-stage ring guarded by full/empty mbarriers; four consumer warps take
+// 16 keys of every tile each and never synchronise with one another otherwise:
+//   S = Q K^T      m16n8k16 bf16 MMA, the g query heads padded to the MMA rows
 //   online softmax in fp32 registers (exp2 with the scale folded in)
-//   O += P V       (retained tile)   or   A += P K   (key-only tile: the
-//                  p-weighted key sum that the merge step multiplies by W)
-// P is fed to the second MMA as a bf16 hi + lo pair so that its rounding stays
-// near 2^-17 relative.  The MMAs only keep the FP32 pipe out of the way of the
-// memory stream; the kernel's roofline is HBM bandwidth.
+//   O += P V  (retained tile)  or  A += P K  (key-only tile: the p-weighted key
+//             sum that the merge step multiplies by W); P enters as bf16 hi in
+//             MMA rows 0-7 and bf16 lo in rows 8-15, one MMA for both parts
+// The ring keeps running across unit boundaries, where each warp writes its
+// partial record for the finished unit.  The merge kernel combines a unit's
+// records, applies W and normalises.
 #ifndef VECTOR_DECODE_BF16_CUH_
 #define VECTOR_DECODE_BF16_CUH_
 
 #include "common.cuh"
+#include "tma.cuh"
 
 namespace vec {
 namespace dbf {
 
-constexpr int TILE = 64;              // keys per tile
+constexpr int TILE = 64;                     // keys per tile
 constexpr int STAGES = 3;
-constexpr int ROW_BYTES = 256;        // 128 bf16
-constexpr int MAT_BYTES = TILE * ROW_BYTES;          // 16 KB
-constexpr int STAGE_BYTES = 2 * MAT_BYTES;           // K tile + V tile
-constexpr int STASH_BYTES = 4 * 32 * 32 * 4;         // one accumulator set per warp, parked at the pool switch
-constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + STASH_BYTES;     // 112 KB
-constexpr int REC = 2 + 2 * 128;                     // partial record floats per head
+constexpr int STAGE_BYTES = 32768;           // K tile (2 swizzled 64x128B boxes) + V tile (2 boxes)
+constexpr int BOX_BYTES = 8192;              // 64 rows x 128 bytes
+constexpr int CONSUMER_WARPS = 4;
+constexpr int THREADS = 32 * (CONSUMER_WARPS + 1);
+constexpr int REC = 4 + 2 * 128;             // m, l, value-scale, pad, acc_v[128], acc_k[128]
+constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024;   // + alignment slack; barriers live in static smem
+constexpr int MAX_BLOCKS = 2 * 148;
 
-__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
-
-__device__ __forceinline__ void cp_async16(uint32_t dst, const void* src, int src_bytes) {
-    asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;\n" ::"r"(dst), "l"(src), "r"(src_bytes));
+// How the weighted tile sequence is dealt to blocks; the same arithmetic runs on host and device.
+struct Plan {
+    int n_rt, n_at, n_tiles;   // retained / key-only / all tiles per unit
+    int Wu;                    // weight of a unit = 2 n_rt + n_at
+    long long TW;              // weight of all units
+    int B;                     // blocks
+    int s_max;                 // record slots per unit
+};
+__host__ __device__ inline Plan make_plan(int U, long long n_ret, long long n_apx) {
+    Plan p;
+    p.n_rt = (int)((n_ret + TILE - 1) / TILE);
+    p.n_at = (int)((n_apx + TILE - 1) / TILE);
+    p.n_tiles = p.n_rt + p.n_at;
+    p.Wu = 2 * p.n_rt + p.n_at;
+    p.TW = (long long)U * p.Wu;
+    long long b = p.TW / 8;                      // at least 8 weight units (4+ tiles) per block
+    if (b > MAX_BLOCKS) b = MAX_BLOCKS;
+    if (b > 11LL * U) b = 11LL * U;              // at most 12 record slots per unit (merge kernel limit)
+    p.B = (int)(b < 1 ? 1 : b);
+    p.s_max = (p.B + U - 1) / U + 1;
+    return p;
 }
-__device__ __forceinline__ void cp_commit() { asm volatile("cp.async.commit_group;\n" ::); }
-template <int N> __device__ __forceinline__ void cp_wait() { asm volatile("cp.async.wait_group %0;\n" ::"n"(N)); }
+// Block b owns the tiles whose start weight lies in [b TW / B, (b+1) TW / B).
+__host__ __device__ inline long long weight_begin(int b, const Plan& p) { return (long long)b * p.TW / p.B; }
+__host__ __device__ inline int block_of_weight(long long s, const Plan& p) { return (int)(((s + 1) * p.B - 1) / p.TW); }
+// global index of the first tile whose start weight is >= x
+__host__ __device__ inline long long tile_from_weight(long long x, const Plan& p) {
+    long long u = x / p.Wu;
+    int r = (int)(x - u * p.Wu);
+    int t = r <= 2 * p.n_rt ? (r + 1) / 2 : p.n_rt + (r - 2 * p.n_rt);
+    return u * p.n_tiles + t;
+}
+__host__ __device__ inline long long unit_first_weight(int u, const Plan& p) { return (long long)u * p.Wu; }
+__host__ __device__ inline long long unit_last_weight(int u, const Plan& p) {   // start weight of the unit's last tile
+    int t = p.n_tiles - 1;
+    return (long long)u * p.Wu + (t < p.n_rt ? 2 * t : 2 * p.n_rt + (t - p.n_rt));
+}
 
 __device__ __forceinline__ void ldsm_x4(uint32_t addr, uint32_t& r0, uint32_t& r1, uint32_t& r2, uint32_t& r3) {
     asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];\n"
@@ -44,8 +83,8 @@ __device__ __forceinline__ void ldsm_x4_t(uint32_t addr, uint32_t& r0, uint32_t&
     asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];\n"
                  : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3) : "r"(addr));
 }
-// D(16x8) += A(16x16) B(16x8); only rows 0..7 of A are non-zero, so the upper
-// accumulator half stays zero and is parked in a scratch pair.
+// D(16x8) += A(16x16) B(16x8) with A rows 8..15 zero: the upper accumulator half is fed zeros and
+// its (zero) result parked in a scratch pair.
 __device__ __forceinline__ void mma_lo8(float& c0, float& c1, float& z0, float& z1, uint32_t a0, uint32_t a2,
                                         uint32_t b0, uint32_t b1) {
     asm volatile(
@@ -53,219 +92,301 @@ __device__ __forceinline__ void mma_lo8(float& c0, float& c1, float& z0, float& 
         : "+f"(c0), "+f"(c1), "=f"(z0), "=f"(z1)
         : "r"(a0), "r"(0u), "r"(a2), "r"(0u), "r"(b0), "r"(b1), "f"(0.f));
 }
+__device__ __forceinline__ void mma_16(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0,
+                                       uint32_t b1) {
+    asm volatile(
+        "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};\n"
+        : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+        : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
     __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
     return *reinterpret_cast<uint32_t*>(&v);
 }
 
-// byte offset of 16-byte chunk `chunk` of row `row` inside a swizzled 64x256-byte tile
-__device__ __forceinline__ uint32_t swz(int row, int chunk) { return row * ROW_BYTES + ((chunk ^ (row & 7)) << 4); }
-
-struct TileDesc {
-    const __nv_bfloat16* k;   // first row of the tile's keys
-    const __nv_bfloat16* v;   // first row of its values, or nullptr for a key-only tile
-    int nrows;
+struct Maps {
+    CUtensorMap ret_k, ret_v, apx_k;     // rank 3: (128 dims, pool rows, U units), box 64 x 64 x 1, 128B swizzle
 };
 
-__device__ __forceinline__ TileDesc tile_desc(int t, int n_rt, int u, const __nv_bfloat16* ret_k,
-                                              const __nv_bfloat16* ret_v, const __nv_bfloat16* apx_k,
-                                              int64_t cap_ret, int64_t cap_apx, int n_ret, int n_apx) {
-    TileDesc d;
-    if (t < n_rt) {
-        int row0 = t * TILE;
-        d.k = ret_k + ((size_t)u * cap_ret + row0) * 128;
-        d.v = ret_v + ((size_t)u * cap_ret + row0) * 128;
-        d.nrows = min(TILE, n_ret - row0);
-    } else {
-        int row0 = (t - n_rt) * TILE;
-        d.k = apx_k + ((size_t)u * cap_apx + row0) * 128;
-        d.v = nullptr;
-        d.nrows = min(TILE, n_apx - row0);
-    }
-    return d;
-}
-
-__device__ __forceinline__ void issue_tile(const TileDesc& d, unsigned char* stage, int tid) {
-    const uint32_t ks = smem_u32(stage), vs = ks + MAT_BYTES;
-#pragma unroll
-    for (int i = 0; i < (TILE * 16) / 128; ++i) {
-        int c = tid + 128 * i, row = c >> 4, chunk = c & 15;
-        bool ok = row < d.nrows;
-        int srow = ok ? row : 0;                      // rows past the end are zero-filled, never read
-        cp_async16(ks + swz(row, chunk), (const char*)d.k + (size_t)srow * ROW_BYTES + chunk * 16, ok ? 16 : 0);
-        if (d.v) cp_async16(vs + swz(row, chunk), (const char*)d.v + (size_t)srow * ROW_BYTES + chunk * 16, ok ? 16 : 0);
-    }
-}
-
-// grid (n_splits, U), 128 threads, SMEM_BYTES dynamic shared memory.
-__global__ void __launch_bounds__(128, 2)
-decode_split_bf16_d128(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __restrict__ ret_k,
-                       const __nv_bfloat16* __restrict__ ret_v, const __nv_bfloat16* __restrict__ apx_k,
-                       int64_t cap_ret, int64_t cap_apx, int n_ret, int n_apx, int g, float scale_log2e,
-                       float* __restrict__ partial) {
-    extern __shared__ __align__(1024) unsigned char smem[];
-    const int u = blockIdx.y, split = blockIdx.x, n_splits = gridDim.x;
+// grid (plan.B), THREADS threads, SMEM_BYTES dynamic shared memory.
+// partial: [U][s_max][4 warps][g][REC]; slot of (unit u, block b) = b - block_of_weight(first weight of u).
+__global__ void __launch_bounds__(THREADS, 2)
+decode_stream_bf16_d128(const __nv_bfloat16* __restrict__ q, const __grid_constant__ Maps maps, Plan pl, int n_ret,
+                        int n_apx, int g, float scale_log2e, float* __restrict__ partial, int* __restrict__ fault) {
+    extern __shared__ unsigned char smem_raw[];
+    __shared__ __align__(8) uint64_t full_bar[STAGES];
+    __shared__ __align__(8) uint64_t empty_bar[STAGES];
+    // 128B-swizzled TMA boxes want 1024-byte aligned destinations
+    unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    const int b = blockIdx.x;
     const int tid = threadIdx.x, lane = tid & 31, wq = tid >> 5;
-    const int gid = lane >> 2, tig = lane & 3;
-    const int n_rt = (n_ret + TILE - 1) / TILE, n_at = (n_apx + TILE - 1) / TILE, n_tiles = n_rt + n_at;
-    const int t_lo = (int)((int64_t)split * n_tiles / n_splits);
-    const int t_hi = (int)((int64_t)(split + 1) * n_tiles / n_splits);
+    const long long gt_lo = tile_from_weight(weight_begin(b, pl), pl);
+    const long long gt_hi = tile_from_weight(weight_begin(b + 1, pl), pl);
+    if (gt_lo >= gt_hi) return;
+    const int n_my = (int)(gt_hi - gt_lo);
+    const int u0 = (int)(gt_lo / pl.n_tiles), t0 = (int)(gt_lo - (long long)u0 * pl.n_tiles);
 
-    // Q fragments of head row `gid` (zero for padding rows): 8 k-steps x {dims 2tig.., dims 8+2tig..}
+    if (tid == 0) {
+#pragma unroll
+        for (int s = 0; s < STAGES; ++s) { tma::mbar_init(&full_bar[s], 1); tma::mbar_init(&empty_bar[s], CONSUMER_WARPS); }
+        tma::mbar_fence_init();
+    }
+    __syncthreads();
+
+    if (wq == CONSUMER_WARPS) {
+        // ------------------------------------------------------------------ producer
+        if (lane == 0) {
+            tma::prefetch_map(&maps.ret_k); tma::prefetch_map(&maps.ret_v); tma::prefetch_map(&maps.apx_k);
+            int u = u0, t = t0;
+            bool ok = true;
+            for (int i = 0; i < n_my && ok; ++i) {
+                const int s = i % STAGES, round = i / STAGES;
+                if (round > 0) ok = tma::mbar_wait(&empty_bar[s], (round - 1) & 1, fault, 1);
+                if (!ok) break;
+                unsigned char* st = smem + s * STAGE_BYTES;
+                if (t < pl.n_rt) {
+                    const int row0 = t * TILE;
+                    tma::mbar_expect_tx(&full_bar[s], 4 * BOX_BYTES);
+                    tma::load_3d(st, &maps.ret_k, 0, row0, u, &full_bar[s]);
+                    tma::load_3d(st + BOX_BYTES, &maps.ret_k, 64, row0, u, &full_bar[s]);
+                    tma::load_3d(st + 2 * BOX_BYTES, &maps.ret_v, 0, row0, u, &full_bar[s]);
+                    tma::load_3d(st + 3 * BOX_BYTES, &maps.ret_v, 64, row0, u, &full_bar[s]);
+                } else {
+                    const int row0 = (t - pl.n_rt) * TILE;
+                    tma::mbar_expect_tx(&full_bar[s], 2 * BOX_BYTES);
+                    tma::load_3d(st, &maps.apx_k, 0, row0, u, &full_bar[s]);
+                    tma::load_3d(st + BOX_BYTES, &maps.apx_k, 64, row0, u, &full_bar[s]);
+                }
+                if (++t == pl.n_tiles) { t = 0; ++u; }
+            }
+        }
+        return;      // the consumers wait on every tile's full barrier, so no copy outlives the block
+    }
+
+    // ---------------------------------------------------------------------- consumers
+    const int gid = lane >> 2, tig = lane & 3;
+    const int kr0 = wq * 16;                       // this warp's 16 keys inside every tile
+    // per-lane ldmatrix geometry (swizzle: 16-byte chunk index XOR (row & 7), rows are 128 bytes)
+    const int mat = lane >> 3, r8 = lane & 7;
+    const uint32_t qk_row = (uint32_t)(kr0 + r8 + (mat >> 1) * 8) * 128u;      // QK: matrices = (keys 0-7|8-15) x (chunk lo|hi)
+    const uint32_t qk_x = (uint32_t)(((mat & 1) ^ r8) << 4);
+    const uint32_t pv_row = (uint32_t)(kr0 + r8 + (mat & 1) * 8) * 128u;       // PV: matrices = (chunk lo|hi) x (keys 0-7|8-15)
+    const uint32_t pv_x = (uint32_t)(((mat >> 1) ^ r8) << 4);
+
     uint32_t qa[8][2];
-    {
-        const uint32_t* qrow = reinterpret_cast<const uint32_t*>(q + ((size_t)u * g + min(gid, g - 1)) * 128);
+    float acc[16][4];                  // [dim tile][c0,c1: P_hi rows | c2,c3: P_lo rows]
+    float zz[4][2];
+    float m = -INFINITY, l = 0.f, stash_scale = 1.f;
+    bool stashed = false;
+    int u = u0, t = t0;
+
+    auto record_of = [&](int unit) -> float* {
+        const int slot = b - block_of_weight(unit_first_weight(unit, pl), pl);
+        return partial + ((((size_t)unit * pl.s_max + slot) * CONSUMER_WARPS + wq) * g + gid) * REC;
+    };
+    auto load_q = [&](int unit) {
+        const uint32_t* qrow = reinterpret_cast<const uint32_t*>(q + ((size_t)unit * g + min(gid, g - 1)) * 128);
 #pragma unroll
         for (int ks = 0; ks < 8; ++ks) {
             qa[ks][0] = gid < g ? qrow[ks * 8 + tig] : 0u;
             qa[ks][1] = gid < g ? qrow[ks * 8 + 4 + tig] : 0u;
         }
-    }
-    // One accumulator set.  A block's tiles are ordered retained first, key-only second, so the
-    // set collects sum p v until the first key-only tile, is parked in shared memory there (its
-    // later rescaling tracked by one factor), and then collects sum p k.
-    float acc[16][2];
+    };
+    auto store_acc = [&](float* dst) {       // dims n*8 + 2 tig + {0,1} of head row gid
 #pragma unroll
-    for (int n = 0; n < 16; ++n) { acc[n][0] = acc[n][1] = 0.f; }
-    float* stash = reinterpret_cast<float*>(smem + STAGES * STAGE_BYTES) + wq * 32 * 32 + lane;
-    bool stashed = false;
-    float stash_scale = 1.f;
-    float zz[4][2];                    // write-only parking for the unused accumulator halves
-    float m = -INFINITY, l = 0.f;      // running max (scaled log2 units) and this thread's share of the sum
-
-    // prologue: STAGES-1 tiles in flight
+        for (int n = 0; n < 16; ++n)
+            *reinterpret_cast<float2*>(dst + n * 8 + 2 * tig) = make_float2(acc[n][0] + acc[n][2], acc[n][1] + acc[n][3]);
+    };
+    auto zero_acc = [&]() {
 #pragma unroll
-    for (int s = 0; s < STAGES - 1; ++s) {
-        int t = t_lo + s;
-        if (t < t_hi)
-            issue_tile(tile_desc(t, n_rt, u, ret_k, ret_v, apx_k, cap_ret, cap_apx, n_ret, n_apx),
-                       smem + s * STAGE_BYTES, tid);
-        cp_commit();
-    }
-    for (int t = t_lo; t < t_hi; ++t) {
-        cp_wait<STAGES - 2>();
-        __syncthreads();
-        {   // refill the stage consumed one iteration ago
-            int tn = t + STAGES - 1;
-            if (tn < t_hi)
-                issue_tile(tile_desc(tn, n_rt, u, ret_k, ret_v, apx_k, cap_ret, cap_apx, n_ret, n_apx),
-                           smem + ((tn - t_lo) % STAGES) * STAGE_BYTES, tid);
-            cp_commit();
-        }
-        const bool retained = t < n_rt;
-        const int nrows = retained ? min(TILE, n_ret - t * TILE) : min(TILE, n_apx - (t - n_rt) * TILE);
-        const int kr0 = wq * 16;
-        if (kr0 >= nrows) continue;            // this warp's 16 keys lie past the end of the pool
-        const uint32_t ks_base = smem_u32(smem + ((t - t_lo) % STAGES) * STAGE_BYTES);
-        const uint32_t vs_base = retained ? ks_base + MAT_BYTES : ks_base;
-
-        // ---- S = Q K^T for 16 keys (two 8-key column tiles)
-        float s0[2], s1[2];
-        {
-            // four independent accumulation chains (even / odd k-steps x two key tiles)
-            float e0[2] = {0.f, 0.f}, e1[2] = {0.f, 0.f}, o0[2] = {0.f, 0.f}, o1[2] = {0.f, 0.f};
-            const int mat = lane >> 3, r = lane & 7;
-            const int key = kr0 + r + (mat >> 1) * 8;
+        for (int n = 0; n < 16; ++n) { acc[n][0] = acc[n][1] = acc[n][2] = acc[n][3] = 0.f; }
+    };
+    auto flush = [&](int unit) {
+        float lt = l;
+        lt += __shfl_xor_sync(0xffffffffu, lt, 1);
+        lt += __shfl_xor_sync(0xffffffffu, lt, 2);
+        if (gid < g) {
+            float* rec = record_of(unit);
+            if (tig == 0) *reinterpret_cast<float4*>(rec) = make_float4(m * 0.69314718055994531f, lt, stashed ? stash_scale : 1.f, 0.f);
+            if (stashed) store_acc(rec + 4 + 128);                     // value part was written at the pool switch
+            else {
+                store_acc(rec + 4);
 #pragma unroll
-            for (int ks = 0; ks < 8; ks += 2) {
-                uint32_t b0, b1, b2, b3, c0, c1, c2, c3;
-                ldsm_x4(ks_base + swz(key, ks * 2 + (mat & 1)), b0, b1, b2, b3);
-                ldsm_x4(ks_base + swz(key, ks * 2 + 2 + (mat & 1)), c0, c1, c2, c3);
-                mma_lo8(e0[0], e0[1], zz[0][0], zz[0][1], qa[ks][0], qa[ks][1], b0, b1);
-                mma_lo8(e1[0], e1[1], zz[1][0], zz[1][1], qa[ks][0], qa[ks][1], b2, b3);
-                mma_lo8(o0[0], o0[1], zz[2][0], zz[2][1], qa[ks + 1][0], qa[ks + 1][1], c0, c1);
-                mma_lo8(o1[0], o1[1], zz[3][0], zz[3][1], qa[ks + 1][0], qa[ks + 1][1], c2, c3);
+                for (int n = 0; n < 16; ++n) *reinterpret_cast<float2*>(rec + 4 + 128 + n * 8 + 2 * tig) = make_float2(0.f, 0.f);
             }
-            s0[0] = e0[0] + o0[0]; s0[1] = e0[1] + o0[1];
-            s1[0] = e1[0] + o1[0]; s1[1] = e1[1] + o1[1];
         }
-        // ---- online softmax over these 16 keys (row = head gid, shared by the 4 threads of a quad)
-        const int kc = kr0 + 2 * tig;
-        float t00 = kc < nrows ? s0[0] * scale_log2e : -INFINITY;
-        float t01 = kc + 1 < nrows ? s0[1] * scale_log2e : -INFINITY;
-        float t10 = kc + 8 < nrows ? s1[0] * scale_log2e : -INFINITY;
-        float t11 = kc + 9 < nrows ? s1[1] * scale_log2e : -INFINITY;
-        float mx = fmaxf(fmaxf(t00, t01), fmaxf(t10, t11));
-        mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
-        mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
-        if (!retained && !stashed) {               // first key-only tile this warp works on
+        zero_acc();
+        m = -INFINITY; l = 0.f; stash_scale = 1.f; stashed = false;
+    };
+
+    load_q(u);
+    zero_acc();
+    for (int i = 0; i < n_my; ++i) {
+        const int s = i % STAGES, round = i / STAGES;
+        if (!tma::mbar_wait(&full_bar[s], round & 1, fault, 2)) break;
+        const bool retained = t < pl.n_rt;
+        const int nrows = retained ? min(TILE, n_ret - t * TILE) : min(TILE, n_apx - (t - pl.n_rt) * TILE);
+        if (kr0 < nrows) {
+            const uint32_t kbase = tma::smem_u32(smem + s * STAGE_BYTES);
+            const uint32_t vbase = retained ? kbase + 2 * BOX_BYTES : kbase;
+            // ---- S = Q K^T for 16 keys: four independent chains (even / odd k-steps x two 8-key tiles)
+            float s0[2], s1[2];
+            {
+                float e0[2] = {0.f, 0.f}, e1[2] = {0.f, 0.f}, o0[2] = {0.f, 0.f}, o1[2] = {0.f, 0.f};
 #pragma unroll
-            for (int n = 0; n < 16; ++n) {
-                stash[(2 * n) * 32] = acc[n][0];
-                stash[(2 * n + 1) * 32] = acc[n][1];
-                acc[n][0] = acc[n][1] = 0.f;
+                for (int ks = 0; ks < 8; ks += 2) {
+                    uint32_t b0, b1, b2, b3, c0, c1, c2, c3;
+                    // k-step ks covers 16-byte chunks 2ks, 2ks+1 of the 256-byte row: box ks/4, chunk (2ks)%8 (+1)
+                    ldsm_x4(kbase + (ks >> 2) * BOX_BYTES + qk_row + ((((2 * ks) & 7) << 4) ^ qk_x), b0, b1, b2, b3);
+                    ldsm_x4(kbase + ((ks + 1) >> 2) * BOX_BYTES + qk_row + ((((2 * ks + 2) & 7) << 4) ^ qk_x), c0, c1, c2, c3);
+                    mma_lo8(e0[0], e0[1], zz[0][0], zz[0][1], qa[ks][0], qa[ks][1], b0, b1);
+                    mma_lo8(e1[0], e1[1], zz[1][0], zz[1][1], qa[ks][0], qa[ks][1], b2, b3);
+                    mma_lo8(o0[0], o0[1], zz[2][0], zz[2][1], qa[ks + 1][0], qa[ks + 1][1], c0, c1);
+                    mma_lo8(o1[0], o1[1], zz[3][0], zz[3][1], qa[ks + 1][0], qa[ks + 1][1], c2, c3);
+                }
+                s0[0] = e0[0] + o0[0]; s0[1] = e0[1] + o0[1];
+                s1[0] = e1[0] + o1[0]; s1[1] = e1[1] + o1[1];
             }
-            stashed = true;
-            stash_scale = 1.f;
-        }
-        const float m_new = fmaxf(m, mx);          // finite: key kr0 is valid for every row
-        const float alpha = exp2f(m - m_new);      // 0 on the first tile
-        const float p00 = exp2f(t00 - m_new), p01 = exp2f(t01 - m_new);
-        const float p10 = exp2f(t10 - m_new), p11 = exp2f(t11 - m_new);
-        l = l * alpha + (p00 + p01) + (p10 + p11);
-        m = m_new;
-        stash_scale *= alpha;
-        if (__any_sync(0xffffffffu, alpha != 1.f)) {
+            // ---- online softmax over these 16 keys (row = head gid, shared by the 4 threads of a quad)
+            const int kc = kr0 + 2 * tig;
+            const float t00 = kc < nrows ? s0[0] * scale_log2e : -INFINITY;
+            const float t01 = kc + 1 < nrows ? s0[1] * scale_log2e : -INFINITY;
+            const float t10 = kc + 8 < nrows ? s1[0] * scale_log2e : -INFINITY;
+            const float t11 = kc + 9 < nrows ? s1[1] * scale_log2e : -INFINITY;
+            float mx = fmaxf(fmaxf(t00, t01), fmaxf(t10, t11));
+            mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
+            mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
+            if (!retained && !stashed) {           // first key-only tile of this unit for this warp: park sum p v
+                if (gid < g) store_acc(record_of(u) + 4);
+                zero_acc();
+                stashed = true;
+                stash_scale = 1.f;
+            }
+            const float m_new = fmaxf(m, mx);      // finite: key kr0 is valid for every row
+            const float alpha = exp2f(m - m_new);  // 0 on the first tile
+            const float p00 = exp2f(t00 - m_new), p01 = exp2f(t01 - m_new);
+            const float p10 = exp2f(t10 - m_new), p11 = exp2f(t11 - m_new);
+            l = l * alpha + (p00 + p01) + (p10 + p11);
+            m = m_new;
+            stash_scale *= alpha;
+            if (__any_sync(0xffffffffu, alpha != 1.f)) {
 #pragma unroll
-            for (int n = 0; n < 16; ++n) { acc[n][0] *= alpha; acc[n][1] *= alpha; }
-        }
-        // P as bf16 hi + lo
-        const __nv_bfloat16 h00 = __float2bfloat16_rn(p00), h01 = __float2bfloat16_rn(p01);
-        const __nv_bfloat16 h10 = __float2bfloat16_rn(p10), h11 = __float2bfloat16_rn(p11);
-        const uint32_t pa_hi0 = pack_bf16(__bfloat162float(h00), __bfloat162float(h01));
-        const uint32_t pa_hi2 = pack_bf16(__bfloat162float(h10), __bfloat162float(h11));
-        const uint32_t pa_lo0 = pack_bf16(p00 - __bfloat162float(h00), p01 - __bfloat162float(h01));
-        const uint32_t pa_lo2 = pack_bf16(p10 - __bfloat162float(h10), p11 - __bfloat162float(h11));
-        // ---- accumulate P x (V tile | K tile) over the 16 column tiles of 8 dims
-        {
-            const int mat = lane >> 3, r = lane & 7;
-            const int key = kr0 + r + (mat & 1) * 8;
+                for (int n = 0; n < 16; ++n) { acc[n][0] *= alpha; acc[n][1] *= alpha; acc[n][2] *= alpha; acc[n][3] *= alpha; }
+            }
+            // P as bf16 hi (MMA rows 0-7) + lo (rows 8-15)
+            const __nv_bfloat16 h00 = __float2bfloat16_rn(p00), h01 = __float2bfloat16_rn(p01);
+            const __nv_bfloat16 h10 = __float2bfloat16_rn(p10), h11 = __float2bfloat16_rn(p11);
+            const uint32_t a0 = pack_bf16(__bfloat162float(h00), __bfloat162float(h01));
+            const uint32_t a2 = pack_bf16(__bfloat162float(h10), __bfloat162float(h11));
+            const uint32_t a1 = pack_bf16(p00 - __bfloat162float(h00), p01 - __bfloat162float(h01));
+            const uint32_t a3 = pack_bf16(p10 - __bfloat162float(h10), p11 - __bfloat162float(h11));
+            // ---- accumulate P x (V rows | K rows) over the 16 column tiles of 8 dims
 #pragma unroll
             for (int np = 0; np < 8; ++np) {
                 uint32_t b0, b1, b2, b3;
-                ldsm_x4_t(vs_base + swz(key, np * 2 + (mat >> 1)), b0, b1, b2, b3);
-                mma_lo8(acc[2 * np][0], acc[2 * np][1], zz[0][0], zz[0][1], pa_hi0, pa_hi2, b0, b1);
-                mma_lo8(acc[2 * np + 1][0], acc[2 * np + 1][1], zz[1][0], zz[1][1], pa_hi0, pa_hi2, b2, b3);
-                mma_lo8(acc[2 * np][0], acc[2 * np][1], zz[2][0], zz[2][1], pa_lo0, pa_lo2, b0, b1);
-                mma_lo8(acc[2 * np + 1][0], acc[2 * np + 1][1], zz[3][0], zz[3][1], pa_lo0, pa_lo2, b2, b3);
+                ldsm_x4_t(vbase + (np >> 2) * BOX_BYTES + pv_row + ((((2 * np) & 7) << 4) ^ pv_x), b0, b1, b2, b3);
+                mma_16(acc[2 * np], a0, a1, a2, a3, b0, b1);
+                mma_16(acc[2 * np + 1], a0, a1, a2, a3, b2, b3);
             }
         }
+        __syncwarp();
+        if (lane == 0) tma::mbar_arrive(&empty_bar[s]);
+        if (++t == pl.n_tiles) {
+            flush(u);
+            t = 0; ++u;
+            if (i + 1 < n_my) load_q(u);
+        }
     }
-    cp_wait<0>();
-    __syncthreads();                    // every stage is free: reuse it for the cross-warp combine
-    float* sm = reinterpret_cast<float*>(smem);          // [4 warps][8 heads][REC]
-    l += __shfl_xor_sync(0xffffffffu, l, 1);
-    l += __shfl_xor_sync(0xffffffffu, l, 2);
-    {
-        float* rec = sm + ((size_t)wq * 8 + gid) * REC;
-        if (tig == 0) { rec[0] = m; rec[1] = l; }
+    if (t != 0) flush(u);            // the range ended inside a unit
+}
+
+// Merge for head_dim 128: grid (U), 128 threads.  Combines the records of a unit, applies the
+// unit's map to the p-weighted key sum and normalises: o = (sum f s acc_v + W sum f acc_k) / sum f l.
+template <typename TO>
+__global__ void __launch_bounds__(128)
+decode_merge_bf16_d128(const float* __restrict__ partial, const __nv_bfloat16* __restrict__ W, int LH, int g,
+                       Plan pl, TO* __restrict__ out) {
+    __shared__ uint32_t Ws[128 * 65];          // W rows as bf16 pairs, row stride 65 words (conflict-free)
+    __shared__ float aks[8][128];
+    __shared__ float fv[8][48], fk[8][48];     // per head, per record: factor for the value part / the key part and l
+    __shared__ float Ls[8];
+    const int u = blockIdx.x, c = threadIdx.x;
+    const int first = block_of_weight(unit_first_weight(u, pl), pl);
+    const int n_rec = (block_of_weight(unit_last_weight(u, pl), pl) - first + 1) * CONSUMER_WARPS;   // <= 48 (checked on the host)
+    const float* base = partial + (size_t)u * pl.s_max * CONSUMER_WARPS * g * REC;
+    // W tile into shared memory while the record headers are fetched
+    const uint32_t* Wu = reinterpret_cast<const uint32_t*>(W + (size_t)(u % LH) * 128 * 128);
+#pragma unroll 16
+    for (int k = 0; k < 64; ++k) {
+        int i = c + 128 * k;
+        Ws[(i >> 6) * 65 + (i & 63)] = Wu[i];
+    }
+    if (c < 8 * 16) {
+        // thread (a = c / 16, lane16 = c % 16): headers of head a, records lane16, lane16+16, lane16+32
+        const int a = c >> 4, j0 = c & 15;
+        float mj[3], lj[3], sj[3];
+        float M = -INFINITY;
 #pragma unroll
-        for (int n = 0; n < 16; ++n) {
-            // value part: the parked set if the switch happened, else the live set; key part: the rest
-            float v0 = stashed ? stash[(2 * n) * 32] * stash_scale : acc[n][0];
-            float v1 = stashed ? stash[(2 * n + 1) * 32] * stash_scale : acc[n][1];
-            rec[2 + n * 8 + 2 * tig] = v0;
-            rec[2 + n * 8 + 2 * tig + 1] = v1;
-            rec[2 + 128 + n * 8 + 2 * tig] = stashed ? acc[n][0] : 0.f;
-            rec[2 + 128 + n * 8 + 2 * tig + 1] = stashed ? acc[n][1] : 0.f;
+        for (int k = 0; k < 3; ++k) {
+            int j = j0 + 16 * k;
+            mj[k] = -INFINITY; lj[k] = 0.f; sj[k] = 0.f;
+            if (a < g && j < n_rec) {
+                float4 h = *reinterpret_cast<const float4*>(base + ((size_t)j * g + a) * REC);
+                mj[k] = h.x; lj[k] = h.y; sj[k] = h.z;
+            }
+            M = fmaxf(M, mj[k]);
+        }
+#pragma unroll
+        for (int o = 8; o > 0; o >>= 1) M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, o));
+        float Lsum = 0.f;
+#pragma unroll
+        for (int k = 0; k < 3; ++k) {
+            int j = j0 + 16 * k;
+            float f = mj[k] > -INFINITY ? __expf(mj[k] - M) : 0.f;
+            if (j < 48) { fk[a][j] = f; fv[a][j] = f * sj[k]; }
+            Lsum += f * lj[k];
+        }
+#pragma unroll
+        for (int o = 8; o > 0; o >>= 1) Lsum += __shfl_xor_sync(0xffffffffu, Lsum, o);
+        if (j0 == 0) Ls[a] = Lsum;
+    }
+    __syncthreads();
+    float accv[8];
+#pragma unroll
+    for (int a = 0; a < 8; ++a) {
+        accv[a] = 0.f;
+        if (a < g) {
+            float av = 0.f, ak = 0.f;
+#pragma unroll 4
+            for (int j = 0; j < n_rec; ++j) {
+                const float* r = base + ((size_t)j * g + a) * REC + 4;
+                av = fmaf(fv[a][j], r[c], av);
+                ak = fmaf(fk[a][j], r[128 + c], ak);
+            }
+            accv[a] = av;
+            aks[a][c] = ak;
         }
     }
     __syncthreads();
-    float* out = partial + ((size_t)u * n_splits + split) * g * REC;
-    for (int a = 0; a < g; ++a) {
-        const float m0 = sm[(0 * 8 + a) * REC], m1 = sm[(1 * 8 + a) * REC], m2 = sm[(2 * 8 + a) * REC],
-                    m3 = sm[(3 * 8 + a) * REC];
-        const float M = fmaxf(fmaxf(m0, m1), fmaxf(m2, m3));
-        const float f0 = m0 > -INFINITY ? exp2f(m0 - M) : 0.f, f1 = m1 > -INFINITY ? exp2f(m1 - M) : 0.f;
-        const float f2 = m2 > -INFINITY ? exp2f(m2 - M) : 0.f, f3 = m3 > -INFINITY ? exp2f(m3 - M) : 0.f;
-        for (int c = tid; c < REC; c += 128) {
-            float v;
-            if (c == 0) v = M * 0.69314718055994531f;       // back to natural-log units for the merge step
-            else v = f0 * sm[(0 * 8 + a) * REC + c] + f1 * sm[(1 * 8 + a) * REC + c] +
-                     f2 * sm[(2 * 8 + a) * REC + c] + f3 * sm[(3 * 8 + a) * REC + c];
-            out[a * REC + c] = v;
+    float proj[8];
+#pragma unroll
+    for (int a = 0; a < 8; ++a) proj[a] = 0.f;
+#pragma unroll 4
+    for (int c2 = 0; c2 < 64; ++c2) {
+        const uint32_t w2 = Ws[c * 65 + c2];
+        const float w_lo = __uint_as_float(w2 << 16), w_hi = __uint_as_float(w2 & 0xffff0000u);
+#pragma unroll
+        for (int a = 0; a < 8; ++a) {
+            if (a < g) {
+                const float2 k2 = *reinterpret_cast<const float2*>(&aks[a][2 * c2]);
+                proj[a] = fmaf(w_lo, k2.x, proj[a]);
+                proj[a] = fmaf(w_hi, k2.y, proj[a]);
+            }
         }
     }
+#pragma unroll
+    for (int a = 0; a < 8; ++a)
+        if (a < g) store_out(out + ((size_t)u * g + a) * 128 + c, (accv[a] + proj[a]) / Ls[a]);
 }
 
 }  // namespace dbf

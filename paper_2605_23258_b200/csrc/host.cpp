@@ -78,7 +78,7 @@ size_t select_ws_bytes(const Dims& D, const vector_budget& b) {
 }
 
 int decode_num_splits(int U, int64_t rows) {
-    int64_t want = (8 * 148 + U - 1) / U;
+    int64_t want = (4 * 148 + U - 1) / U;
     int64_t max_by_rows = (rows + 255) / 256;   // at least 256 rows per split
     if (want > max_by_rows) want = max_by_rows;
     if (want > 64) want = 64;
@@ -86,11 +86,20 @@ int decode_num_splits(int U, int64_t rows) {
     return (int)want;
 }
 
+int decode_stream_slots(int U) {
+    int s = (2 * 148 + U - 1) / U + 1;
+    return s < 12 ? s : 12;
+}
+
 size_t decode_ws_bytes(const Dims& D) {
-    // the split count never exceeds what decode_num_splits returns for an unbounded row count
+    // the split count never exceeds what decode_num_splits returns for an unbounded row count,
+    // nor the record slots per unit of the persistent kernel
     int s = decode_num_splits(D.U, int64_t(1) << 40);
-    // per (unit, split): m[g], l[g], acc_v[g][d], acc_k[g][d]
-    return align256((size_t)D.U * s * D.g * (2 + 2 * (size_t)D.d) * sizeof(float));
+    // split kernel: per (unit, split, head) m, l, acc_v[d], acc_k[d]
+    size_t a = (size_t)D.U * s * D.g * (2 + 2 * (size_t)D.d) * sizeof(float);
+    // persistent kernel: per (unit, slot, consumer warp, head) a 4-float header, acc_v[128], acc_k[128]
+    size_t b = (size_t)D.U * decode_stream_slots(D.U) * 4 * D.g * (4 + 256) * sizeof(float);
+    return align256(a > b ? a : b);
 }
 
 }  // namespace vec

@@ -39,6 +39,8 @@ size_t score_ws_bytes(const Dims& D, int64_t N, bool need_raw);
 size_t select_ws_bytes(const Dims& D, const vector_budget& b);
 // Number of key splits of one unit in decode attention for `rows` logical keys.
 int decode_num_splits(int U, int64_t rows);
+// Record slots per unit that the persistent bf16 decode kernel may use (two blocks per SM, 148 SMs).
+int decode_stream_slots(int U);
 size_t decode_ws_bytes(const Dims& D);
 
 inline size_t align256(size_t x) { return (x + 255) & ~size_t(255); }
