@@ -182,7 +182,7 @@ static vector_status launch_decode(const Dims& dm, const void* q, const vector_c
 
 // Fault word that bounded waits inside kernels write to (0 = none).
 static __device__ int g_kernel_fault;
-static int* kernel_fault_address() {
+int* kernel_fault_address() {
     static int* addr = nullptr;           // single-device processes; looked up with the current device
     if (!addr) {
         void* p = nullptr;

@@ -63,7 +63,39 @@ int score_num_chunks(int U, int R, int64_t N) {
     return (int)want;
 }
 
+ScoreTcPlan score_tc_plan(int U, int R, int64_t N) {
+    ScoreTcPlan p;
+    p.RG = (R + 255) / 256;
+    p.nt = (int)((N + 127) / 128);
+    // chunks per unit: fill whole rounds of one block per SM, but keep chunks long enough that the
+    // per-item cost (Q load, pipeline fill) stays small
+    const int blocks = 148;
+    double best = -1.0;
+    int best_n = 1;
+    const int max_n = p.nt < 64 ? p.nt : 64;
+    for (int n = 1; n <= max_n; ++n) {
+        const int tpc = (p.nt + n - 1) / n;
+        const int n_eff = (p.nt + tpc - 1) / tpc;
+        if (n_eff != n) continue;
+        const long long items = (long long)U * p.RG * n;
+        const long long rounds = (items + blocks - 1) / blocks;
+        const double fill = (double)items / (double)(rounds * blocks);
+        const double merit = fill * tpc / (tpc + 2.0);
+        if (merit > best + 1e-9) { best = merit; best_n = n; }
+    }
+    p.n_chunks = best_n;
+    p.tpc = (p.nt + best_n - 1) / best_n;
+    p.n_items = U * p.RG * p.n_chunks;
+    return p;
+}
+
 size_t score_ws_bytes(const Dims& D, int64_t N, bool need_raw) {
+    if (score_uses_tc(D)) {
+        const ScoreTcPlan p = score_tc_plan(D.U, D.R, N);
+        return align256((size_t)D.U * p.n_chunks * D.R * 2 * sizeof(float)) +     // (max, sum) partials
+               align256((size_t)D.U * D.R * sizeof(float)) +                        // lse
+               align256((size_t)D.U * 2 * p.RG * (size_t)N * sizeof(float));        // per-row-block key sums
+    }
     size_t b = 0;
     b += align256((size_t)D.U * score_num_chunks(D.U, D.R, N) * D.R * 2 * sizeof(float));  // (max, sum) partials
     b += align256((size_t)D.U * D.R * sizeof(float));                                       // lse

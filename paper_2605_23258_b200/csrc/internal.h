@@ -36,6 +36,13 @@ void set_last_cuda_error(int e);
 // Number of key chunks the first score pass splits a unit's keys into.
 int score_num_chunks(int U, int R, int64_t N);
 size_t score_ws_bytes(const Dims& D, int64_t N, bool need_raw);
+// Work split of the tensor-core score kernels (bf16, head_dim 128): row groups of up to 256 window
+// rows, 128-key tiles, and per unit `n_chunks` chunks of `tpc` tiles; an item is (unit, chunk, row group).
+struct ScoreTcPlan { int RG, nt, tpc, n_chunks, n_items; };
+ScoreTcPlan score_tc_plan(int U, int R, int64_t N);
+inline bool score_uses_tc(const Dims& D) { return D.dtype == VECTOR_BF16 && D.d == 128; }
+// Device address of the word in which bounded waits inside kernels record that they gave up.
+int* kernel_fault_address();
 size_t select_ws_bytes(const Dims& D, const vector_budget& b);
 // Number of key splits of one unit in decode attention for `rows` logical keys.
 int decode_num_splits(int U, int64_t rows);

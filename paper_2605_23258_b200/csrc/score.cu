@@ -10,6 +10,7 @@
 //   pool    score[i] = max raw over the centred window (prefix only); +inf in the window
 #include "common.cuh"
 #include "internal.h"
+#include "score_tc.cuh"
 
 namespace vec {
 
@@ -208,6 +209,44 @@ static vector_status launch_score(const Dims& dm, const void* Q, const void* K, 
     return VECTOR_OK;
 }
 
+// bf16, head_dim 128: tcgen05 passes.  Workspace: chunk partials | lse | per-row-block key sums.
+static vector_status launch_score_tc(const Dims& dm, const void* Q, const void* K, int64_t N, float* scores,
+                                     float* raw_out, char* ws, cudaStream_t st) {
+    const ScoreTcPlan pl = score_tc_plan(dm.U, dm.R, N);
+    float2* partial = (float2*)ws;
+    ws += align256((size_t)dm.U * pl.n_chunks * dm.R * 2 * sizeof(float));
+    float* lse2 = (float*)ws;
+    ws += align256((size_t)dm.U * dm.R * sizeof(float));
+    float* raw_part = (float*)ws;
+    static bool configured = false;
+    if (!configured) {
+        VEC_CUDA_CHECK(cudaFuncSetAttribute(stc::score_pass1_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, stc::SMEM_BYTES));
+        VEC_CUDA_CHECK(cudaFuncSetAttribute(stc::score_pass2_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, stc::SMEM_BYTES));
+        configured = true;
+    }
+    int* fault = kernel_fault_address();
+    if (!fault) return VECTOR_ERR_CUDA;
+    CUtensorMap mapQ, mapK;
+    if (!tma::encode_bf16_3d(&mapQ, Q, 128, (uint64_t)dm.R, (uint64_t)dm.U, 256, (uint64_t)dm.R * 256, 64, 128) ||
+        !tma::encode_bf16_3d(&mapK, K, 128, (uint64_t)N, (uint64_t)dm.U, 256, (uint64_t)N * 256, 64, 128))
+        return VECTOR_ERR_CUDA;
+    stc::Params P;
+    P.U = dm.U; P.R = dm.R; P.RG = pl.RG; P.w = dm.w; P.N = N;
+    P.nt = pl.nt; P.tpc = pl.tpc; P.n_chunks = pl.n_chunks; P.n_items = pl.n_items;
+    P.c = dm.scale * 1.4426950408889634f;
+    const int blocks = pl.n_items < 148 ? pl.n_items : 148;
+    stc::score_pass1_tc<<<blocks, stc::THREADS, stc::SMEM_BYTES, st>>>(mapQ, mapK, P, partial, fault);
+    VEC_LAUNCH_CHECK();
+    stc::score_lse2_combine<<<dm.U, 256, 0, st>>>(partial, dm.R, pl.n_chunks, lse2);
+    VEC_LAUNCH_CHECK();
+    stc::score_pass2_tc<<<blocks, stc::THREADS, stc::SMEM_BYTES, st>>>(mapQ, mapK, P, lse2, raw_part, fault);
+    VEC_LAUNCH_CHECK();
+    dim3 gp((unsigned)((N + stc::POOL_TILE - 1) / stc::POOL_TILE), dm.U);
+    stc::score_pool_parts<<<gp, 256, 0, st>>>(raw_part, 2 * pl.RG, N, dm.w, dm.pool_kernel / 2, raw_out, scores);
+    VEC_LAUNCH_CHECK();
+    return VECTOR_OK;
+}
+
 }  // namespace vec
 
 extern "C" vector_status vector_score(const vector_shape* shape, const void* Q_obs, const void* K, int64_t N,
@@ -222,6 +261,7 @@ extern "C" vector_status vector_score(const vector_shape* shape, const void* Q_o
     const bool need_raw = raw_out == nullptr;
     if (!ws || ((uintptr_t)ws & 255) || ws_bytes < score_ws_bytes(dm, N, need_raw)) return VECTOR_ERR_WORKSPACE;
     char* p = (char*)ws;
+    if (score_uses_tc(dm)) return launch_score_tc(dm, Q_obs, K, N, scores, raw_out, p, (cudaStream_t)stream);
     float2* partial = (float2*)p;
     p += align256((size_t)dm.U * score_num_chunks(dm.U, dm.R, N) * dm.R * 2 * sizeof(float));
     float* lse = (float*)p;

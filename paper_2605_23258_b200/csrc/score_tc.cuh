@@ -1,0 +1,473 @@
+// Base importance score on the 5th-generation tensor cores (bf16, head_dim 128).
+//
+// The score of a key is the softmax mass it receives from the observation-window
+// rows (causal inside the window), so the logits Q K^T are needed twice: once
+// for the per-row normaliser, once for the per-key sum.  Both passes are
+// persistent, warp-specialised kernels around tcgen05.mma with the accumulator
+// in tensor memory; the orientation of the product is chosen per pass so that
+// the reduction a thread performs runs along its own TMEM lane:
+//
+//   pass 1   D[row][key] = Q K^T   lane = window row  -> running (max, sum exp2) per row
+//   pass 2   D[key][row] = K Q^T   lane = key         -> sum over rows of exp2(logit - lse[row])
+//
+// A work item is (unit, group of up to 256 rows, contiguous chunk of 128-key
+// tiles); items are dealt round-robin to one block per SM with the row groups of
+// a key chunk on neighbouring blocks, so that a chunk is fetched from HBM once
+// and found in L2 by the other row groups.
+//
+// Roles inside a block (320 threads):
+//   warps 0-7  softmax: two warpgroups, each thread owns one TMEM lane
+//   warp  8    producer: TMA loads of the Q row group (once per item) and of the
+//              K tiles into a 4-stage ring (128-byte swizzle, zero fill past the end)
+//   warp  9    MMA issuer (one thread) and owner of the TMEM allocation
+// All hand-offs are mbarriers; every wait is bounded and records a fault code.
+#ifndef VECTOR_SCORE_TC_CUH_
+#define VECTOR_SCORE_TC_CUH_
+
+#include "common.cuh"
+#include "tma.cuh"
+
+namespace vec {
+namespace stc {
+
+constexpr int KT = 128;                    // keys per tile
+constexpr int STAGES = 4;                  // K ring depth
+constexpr int RG_ROWS = 256;               // window rows per row group
+constexpr int BOX_BYTES = 16384;           // 128 rows x 128 bytes (64 bf16 of the head dimension)
+constexpr int Q_BYTES = 4 * BOX_BYTES;     // [k half][256 rows][128 B]
+constexpr int K_STAGE_BYTES = 2 * BOX_BYTES;   // [k half][128 keys][128 B]
+constexpr int SMEM_BYTES = Q_BYTES + STAGES * K_STAGE_BYTES + 1024;
+constexpr int SOFTMAX_WARPS = 8;
+constexpr int THREADS = 32 * (SOFTMAX_WARPS + 2);
+constexpr int TMEM_COLS = 512;
+
+struct Params {
+    int U, R, RG, w;            // units, rows per unit, row groups per unit, window
+    long long N;                // keys per unit
+    int nt, tpc, n_chunks;      // key tiles per unit, tiles per chunk, chunks per unit
+    int n_items;                // U * n_chunks * RG
+    float c;                    // logit scale * log2(e)
+};
+
+// ---- tcgen05 wrappers -------------------------------------------------------
+__device__ __forceinline__ void tmem_alloc(uint32_t* smem_dst, uint32_t ncols) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;\n"
+                 ::"r"(tma::smem_u32(smem_dst)), "r"(ncols) : "memory");
+}
+__device__ __forceinline__ void tmem_relinquish() {
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;\n" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t ncols) {
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;\n" ::"r"(taddr), "r"(ncols) : "memory");
+}
+__device__ __forceinline__ void fence_before_sync() { asm volatile("tcgen05.fence::before_thread_sync;\n" ::: "memory"); }
+__device__ __forceinline__ void fence_after_sync() { asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory"); }
+
+// D[tmem] (+)= A[smem] B[smem]^T, bf16 inputs, fp32 accumulation, one CTA.
+__device__ __forceinline__ void mma_bf16(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc,
+                                         uint32_t accumulate) {
+    asm volatile(
+        "{\n .reg .pred p;\n setp.ne.b32 p, %4, 0;\n"
+        " tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n}\n"
+        ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
+}
+// The mbarrier receives one arrival when every MMA issued so far by this thread has completed.
+__device__ __forceinline__ void mma_commit(uint64_t* bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];\n"
+                 ::"r"(tma::smem_u32(bar)) : "memory");
+}
+
+// Shared-memory operand descriptor: K-major tile of 128-byte rows under the 128-byte swizzle,
+// groups of 8 rows 1024 bytes apart.  `addr` may point 32/64/96 bytes into a row to select a
+// 16-element slice of the head dimension.
+__device__ __forceinline__ uint64_t smem_desc(uint32_t addr) {
+    uint64_t d = (uint64_t)((addr & 0x3FFFFu) >> 4);
+    d |= (uint64_t)1 << 16;                 // leading byte offset: unused for swizzled K-major operands
+    d |= (uint64_t)(1024 >> 4) << 32;       // stride between 8-row groups
+    d |= (uint64_t)1 << 46;                 // descriptor version of this architecture
+    d |= (uint64_t)2 << 61;                 // 128-byte swizzle
+    return d;
+}
+// Instruction descriptor: fp32 accumulator, bf16 A and B, both K-major, M x N.
+__host__ __device__ constexpr uint32_t instr_desc(int M, int N) {
+    return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(N >> 3) << 17) | ((uint32_t)(M >> 4) << 24);
+}
+
+// 32 consecutive fp32 columns of this thread's TMEM lane.
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,"
+        "%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];\n"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+          "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+          "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+        : "r"(taddr) : "memory");
+}
+// Completes the outstanding TMEM loads; the registers pass through so that no use of them can
+// be scheduled ahead of the wait.
+__device__ __forceinline__ void tmem_ld_wait(uint32_t (&r)[32]) {
+    asm volatile(
+        "tcgen05.wait::ld.sync.aligned;\n"
+        : "+r"(r[0]), "+r"(r[1]), "+r"(r[2]), "+r"(r[3]), "+r"(r[4]), "+r"(r[5]), "+r"(r[6]), "+r"(r[7]),
+          "+r"(r[8]), "+r"(r[9]), "+r"(r[10]), "+r"(r[11]), "+r"(r[12]), "+r"(r[13]), "+r"(r[14]), "+r"(r[15]),
+          "+r"(r[16]), "+r"(r[17]), "+r"(r[18]), "+r"(r[19]), "+r"(r[20]), "+r"(r[21]), "+r"(r[22]), "+r"(r[23]),
+          "+r"(r[24]), "+r"(r[25]), "+r"(r[26]), "+r"(r[27]), "+r"(r[28]), "+r"(r[29]), "+r"(r[30]), "+r"(r[31])
+        :: "memory");
+}
+__device__ __forceinline__ float ex2(float x) {
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;\n" : "=f"(y) : "f"(x));
+    return y;
+}
+
+struct Item { int u, chunk, rg, t0, t1; };
+__device__ __forceinline__ Item decode_item(int it, const Params& P) {
+    Item i;
+    i.rg = it % P.RG;
+    const int uc = it / P.RG;
+    i.chunk = uc % P.n_chunks;
+    i.u = uc / P.n_chunks;
+    i.t0 = i.chunk * P.tpc;
+    i.t1 = min(P.nt, i.t0 + P.tpc);
+    return i;
+}
+
+// Barriers and the TMEM base of one block.
+struct Sync {
+    uint64_t q_full, q_empty;
+    uint64_t k_full[STAGES], k_empty[STAGES];
+    uint64_t acc_full[4], acc_empty[4];
+    uint32_t tmem_base;
+};
+
+// Producer and MMA roles are the same in both passes up to which operand is A and the tile shape.
+//   PASS 1: per key tile two MMAs  D[buf = 2 (tile & 1) + rb] (128 x 128) = Q[rb] K^T
+//   PASS 2: per key tile one MMA   D[buf = tile & 1]         (128 x 256) = K Q^T
+template <int PASS>
+__device__ __forceinline__ void producer_role(const CUtensorMap* mapQ, const CUtensorMap* mapK, const Params& P,
+                                              Sync& sy, unsigned char* Qs, unsigned char* Ks, int* fault) {
+    tma::prefetch_map(mapQ);
+    tma::prefetch_map(mapK);
+    uint32_t kcount = 0, icount = 0;
+    for (int it = blockIdx.x; it < P.n_items; it += gridDim.x, ++icount) {
+        const Item im = decode_item(it, P);
+        if (icount > 0 && !tma::mbar_wait(&sy.q_empty, (icount - 1) & 1, fault, 11)) return;
+        tma::mbar_expect_tx(&sy.q_full, Q_BYTES);
+#pragma unroll
+        for (int kh = 0; kh < 2; ++kh)
+#pragma unroll
+            for (int rb = 0; rb < 2; ++rb)
+                tma::load_3d(Qs + kh * 2 * BOX_BYTES + rb * BOX_BYTES, mapQ, kh * 64, im.rg * RG_ROWS + rb * 128, im.u,
+                             &sy.q_full);
+        for (int t = im.t0; t < im.t1; ++t, ++kcount) {
+            const uint32_t s = kcount % STAGES, round = kcount / STAGES;
+            if (round > 0 && !tma::mbar_wait(&sy.k_empty[s], (round - 1) & 1, fault, 12)) return;
+            tma::mbar_expect_tx(&sy.k_full[s], K_STAGE_BYTES);
+            tma::load_3d(Ks + s * K_STAGE_BYTES, mapK, 0, t * KT, im.u, &sy.k_full[s]);
+            tma::load_3d(Ks + s * K_STAGE_BYTES + BOX_BYTES, mapK, 64, t * KT, im.u, &sy.k_full[s]);
+        }
+    }
+}
+
+template <int PASS>
+__device__ __forceinline__ void mma_role(const Params& P, Sync& sy, unsigned char* Qs, unsigned char* Ks, int* fault) {
+    const uint32_t q_addr = tma::smem_u32(Qs), k_addr = tma::smem_u32(Ks);
+    const uint32_t tmem = sy.tmem_base;
+    uint32_t kcount = 0, icount = 0;
+    for (int it = blockIdx.x; it < P.n_items; it += gridDim.x, ++icount) {
+        const Item im = decode_item(it, P);
+        if (!tma::mbar_wait(&sy.q_full, icount & 1, fault, 21)) return;
+        fence_after_sync();
+        for (int t = im.t0; t < im.t1; ++t, ++kcount) {
+            const uint32_t s = kcount % STAGES, round = kcount / STAGES;
+            if (!tma::mbar_wait(&sy.k_full[s], round & 1, fault, 22)) return;
+            fence_after_sync();
+            const uint32_t ks_addr = k_addr + s * K_STAGE_BYTES;
+            if (PASS == 1) {
+#pragma unroll
+                for (int rb = 0; rb < 2; ++rb) {
+                    const uint32_t buf = (kcount & 1) * 2 + rb, use = kcount >> 1;
+                    if (use > 0 && !tma::mbar_wait(&sy.acc_empty[buf], (use - 1) & 1, fault, 23)) return;
+                    fence_after_sync();
+#pragma unroll
+                    for (int ks = 0; ks < 8; ++ks) {
+                        const uint32_t kh = ks >> 2, ko = (ks & 3) * 32;
+                        mma_bf16(tmem + buf * 128, smem_desc(q_addr + kh * 2 * BOX_BYTES + rb * BOX_BYTES + ko),
+                                 smem_desc(ks_addr + kh * BOX_BYTES + ko), instr_desc(128, 128), ks > 0);
+                    }
+                    mma_commit(&sy.acc_full[buf]);
+                }
+            } else {
+                const uint32_t buf = kcount & 1, use = kcount >> 1;
+                if (use > 0 && !tma::mbar_wait(&sy.acc_empty[buf], (use - 1) & 1, fault, 24)) return;
+                fence_after_sync();
+#pragma unroll
+                for (int ks = 0; ks < 8; ++ks) {
+                    const uint32_t kh = ks >> 2, ko = (ks & 3) * 32;
+                    mma_bf16(tmem + buf * 256, smem_desc(ks_addr + kh * BOX_BYTES + ko),
+                             smem_desc(q_addr + kh * 2 * BOX_BYTES + ko), instr_desc(128, 256), ks > 0);
+                }
+                mma_commit(&sy.acc_full[buf]);
+            }
+            mma_commit(&sy.k_empty[s]);       // the stage is free once these MMAs have read it
+        }
+        mma_commit(&sy.q_empty);
+    }
+}
+
+__device__ __forceinline__ void block_setup(Sync& sy, int empty_count) {
+    if (threadIdx.x == 0) {
+        tma::mbar_init(&sy.q_full, 1);
+        tma::mbar_init(&sy.q_empty, 1);
+#pragma unroll
+        for (int s = 0; s < STAGES; ++s) { tma::mbar_init(&sy.k_full[s], 1); tma::mbar_init(&sy.k_empty[s], 1); }
+#pragma unroll
+        for (int b = 0; b < 4; ++b) { tma::mbar_init(&sy.acc_full[b], 1); tma::mbar_init(&sy.acc_empty[b], empty_count); }
+        tma::mbar_fence_init();
+    }
+    if ((threadIdx.x >> 5) == SOFTMAX_WARPS + 1) {
+        tmem_alloc(&sy.tmem_base, TMEM_COLS);
+        tmem_relinquish();
+    }
+    fence_before_sync();
+    __syncthreads();
+    fence_after_sync();
+}
+__device__ __forceinline__ void block_teardown(Sync& sy) {
+    fence_before_sync();
+    __syncthreads();
+    if ((threadIdx.x >> 5) == SOFTMAX_WARPS + 1) {
+        __syncwarp();
+        fence_after_sync();
+        tmem_dealloc(sy.tmem_base, TMEM_COLS);
+    }
+}
+
+// ---- pass 1 -----------------------------------------------------------------
+// partial[(u * n_chunks + chunk) * R + row] = (running max, sum of exp2) of the row over the
+// chunk's visible keys, in units of log2 (logit * scale * log2 e).  grid: one block per SM.
+__global__ void __launch_bounds__(THREADS, 1)
+score_pass1_tc(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ CUtensorMap mapK, const Params P,
+               float2* __restrict__ partial, int* __restrict__ fault) {
+    extern __shared__ unsigned char smem_raw[];
+    __shared__ Sync sy;
+    unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    unsigned char* Qs = smem;
+    unsigned char* Ks = smem + Q_BYTES;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    block_setup(sy, 4);
+
+    if (warp == SOFTMAX_WARPS) {
+        if (lane == 0) producer_role<1>(&mapQ, &mapK, P, sy, Qs, Ks, fault);
+    } else if (warp == SOFTMAX_WARPS + 1) {
+        if (lane == 0) mma_role<1>(P, sy, Qs, Ks, fault);
+    } else {
+        const int wg = warp >> 2, quarter = warp & 3;
+        const uint32_t lane_addr = sy.tmem_base + ((uint32_t)(quarter * 32) << 16);
+        const long long vis0 = P.N - P.w;               // keys below this index are visible to every row
+        uint32_t tcount = 0;
+        bool ok = true;
+        for (int it = blockIdx.x; it < P.n_items && ok; it += gridDim.x) {
+            const Item im = decode_item(it, P);
+            const int row = im.rg * RG_ROWS + wg * 128 + quarter * 32 + lane;
+            const bool wg_active = im.rg * RG_ROWS + wg * 128 < P.R;
+            const long long last_visible = vis0 + (row % P.w);
+            float m = -INFINITY, l = 0.f;
+            for (int t = im.t0; t < im.t1; ++t, ++tcount) {
+                const uint32_t buf = (tcount & 1) * 2 + wg, use = tcount >> 1;
+                if (!tma::mbar_wait(&sy.acc_full[buf], use & 1, fault, 31)) { ok = false; break; }
+                fence_after_sync();
+                if (wg_active) {
+                    const uint32_t taddr = lane_addr + buf * 128;
+                    const long long key0 = (long long)t * KT;
+                    const bool masked = key0 + KT > vis0;
+                    uint32_t ra[32], rb[32];
+                    tmem_ld32(taddr, ra);
+#pragma unroll
+                    for (int ch = 0; ch < 4; ++ch) {
+                        uint32_t (&cur)[32] = (ch & 1) ? rb : ra;
+                        uint32_t (&nxt)[32] = (ch & 1) ? ra : rb;
+                        tmem_ld_wait(cur);
+                        if (ch < 3) tmem_ld32(taddr + (ch + 1) * 32, nxt);
+                        float v[32];
+#pragma unroll
+                        for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(cur[i]);
+                        if (masked) {
+#pragma unroll
+                            for (int i = 0; i < 32; ++i)
+                                if (key0 + ch * 32 + i > last_visible) v[i] = -INFINITY;
+                        }
+                        float cm0 = fmaxf(v[0], v[1]), cm1 = fmaxf(v[2], v[3]);
+#pragma unroll
+                        for (int i = 4; i < 32; i += 2) { cm0 = fmaxf(cm0, v[i]); cm1 = fmaxf(cm1, v[i + 1]); }
+                        const float m_new = fmaxf(m, fmaxf(cm0, cm1) * P.c);
+                        if (m_new > -INFINITY) {         // false only while every key so far is masked
+                            l *= ex2(m - m_new);         // exp2(-inf) = 0 on the first visible chunk
+                            const float neg = -m_new;
+                            float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
+#pragma unroll
+                            for (int i = 0; i < 32; i += 4) {
+                                s0 += ex2(fmaf(v[i], P.c, neg));
+                                s1 += ex2(fmaf(v[i + 1], P.c, neg));
+                                s2 += ex2(fmaf(v[i + 2], P.c, neg));
+                                s3 += ex2(fmaf(v[i + 3], P.c, neg));
+                            }
+                            l += (s0 + s1) + (s2 + s3);
+                            m = m_new;
+                        }
+                    }
+                }
+                fence_before_sync();
+                __syncwarp();
+                if (lane == 0) tma::mbar_arrive(&sy.acc_empty[buf]);
+            }
+            if (ok && row < P.R) partial[((size_t)im.u * P.n_chunks + im.chunk) * P.R + row] = make_float2(m, l);
+        }
+    }
+    block_teardown(sy);
+}
+
+// lse2[u][row] = log2 sum over all visible keys of exp2(logit2), from the chunk partials.  grid (U).
+__global__ void score_lse2_combine(const float2* __restrict__ partial, int R, int n_chunks, float* __restrict__ lse2) {
+    const int u = blockIdx.x;
+    for (int row = threadIdx.x; row < R; row += blockDim.x) {
+        float M = -INFINITY;
+        for (int c = 0; c < n_chunks; ++c) M = fmaxf(M, partial[((size_t)u * n_chunks + c) * R + row].x);
+        float L = 0.f;
+        for (int c = 0; c < n_chunks; ++c) {
+            const float2 p = partial[((size_t)u * n_chunks + c) * R + row];
+            if (p.x > -INFINITY) L += p.y * exp2f(p.x - M);
+        }
+        lse2[(size_t)u * R + row] = M + log2f(L);
+    }
+}
+
+// ---- pass 2 -----------------------------------------------------------------
+// raw_part[(u * 2 RG + 2 rg + h) * N + key] = sum over rows [rg*256 + h*128, +128) of the softmax
+// probability of `key`; the parts are added up by the pooling kernel.  grid: one block per SM.
+__global__ void __launch_bounds__(THREADS, 1)
+score_pass2_tc(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ CUtensorMap mapK, const Params P,
+               const float* __restrict__ lse2, float* __restrict__ raw_part, int* __restrict__ fault) {
+    extern __shared__ unsigned char smem_raw[];
+    __shared__ Sync sy;
+    __shared__ __align__(16) float neg_lse[RG_ROWS];       // -lse2 of the item's rows; -inf for padding rows
+    unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    unsigned char* Qs = smem;
+    unsigned char* Ks = smem + Q_BYTES;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    block_setup(sy, 8);
+
+    if (warp == SOFTMAX_WARPS) {
+        if (lane == 0) producer_role<2>(&mapQ, &mapK, P, sy, Qs, Ks, fault);
+    } else if (warp == SOFTMAX_WARPS + 1) {
+        if (lane == 0) mma_role<2>(P, sy, Qs, Ks, fault);
+    } else {
+        const int wg = warp >> 2, quarter = warp & 3;
+        const uint32_t lane_addr = sy.tmem_base + ((uint32_t)(quarter * 32) << 16);
+        const int key_in_tile = quarter * 32 + lane;
+        const long long vis0 = P.N - P.w;
+        uint32_t tcount = 0;
+        bool ok = true;
+        for (int it = blockIdx.x; it < P.n_items; it += gridDim.x) {
+            const Item im = decode_item(it, P);
+            // the item's normalisers: all softmax threads leave the old table, refill it, publish it
+            asm volatile("bar.sync 1, 256;\n" ::: "memory");
+            {
+                const int row = im.rg * RG_ROWS + threadIdx.x;
+                neg_lse[threadIdx.x] = row < P.R ? -lse2[(size_t)im.u * P.R + row] : -INFINITY;
+            }
+            asm volatile("bar.sync 1, 256;\n" ::: "memory");
+            if (!ok) continue;                       // keep meeting the others at the barriers above
+            const bool wg_active = im.rg * RG_ROWS + wg * 128 < P.R;
+            const int row_base = im.rg * RG_ROWS + wg * 128;
+            float* out = raw_part + ((size_t)im.u * 2 * P.RG + 2 * im.rg + wg) * P.N;
+            for (int t = im.t0; t < im.t1; ++t, ++tcount) {
+                const uint32_t buf = tcount & 1, use = tcount >> 1;
+                if (!tma::mbar_wait(&sy.acc_full[buf], use & 1, fault, 32)) { ok = false; break; }
+                fence_after_sync();
+                const long long key = (long long)t * KT + key_in_tile;
+                float colsum = 0.f;
+                if (wg_active) {
+                    const uint32_t taddr = lane_addr + buf * 256 + wg * 128;
+                    const bool masked = (long long)t * KT + KT > vis0;
+                    uint32_t ra[32], rb[32];
+                    tmem_ld32(taddr, ra);
+                    float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
+#pragma unroll
+                    for (int ch = 0; ch < 4; ++ch) {
+                        uint32_t (&cur)[32] = (ch & 1) ? rb : ra;
+                        uint32_t (&nxt)[32] = (ch & 1) ? ra : rb;
+                        tmem_ld_wait(cur);
+                        if (ch < 3) tmem_ld32(taddr + (ch + 1) * 32, nxt);
+                        const float4* nl = reinterpret_cast<const float4*>(neg_lse + wg * 128 + ch * 32);
+                        if (!masked) {
+#pragma unroll
+                            for (int i = 0; i < 8; ++i) {
+                                const float4 n4 = nl[i];
+                                s0 += ex2(fmaf(__uint_as_float(cur[4 * i]), P.c, n4.x));
+                                s1 += ex2(fmaf(__uint_as_float(cur[4 * i + 1]), P.c, n4.y));
+                                s2 += ex2(fmaf(__uint_as_float(cur[4 * i + 2]), P.c, n4.z));
+                                s3 += ex2(fmaf(__uint_as_float(cur[4 * i + 3]), P.c, n4.w));
+                            }
+                        } else {
+                            // row r = a * w + j sees the keys up to N - w + j
+#pragma unroll
+                            for (int i = 0; i < 32; ++i) {
+                                const int j = (row_base + ch * 32 + i) % P.w;
+                                const float p = ex2(fmaf(__uint_as_float(cur[i]), P.c, neg_lse[wg * 128 + ch * 32 + i]));
+                                if (key <= vis0 + j) s0 += p;
+                            }
+                        }
+                    }
+                    colsum = (s0 + s1) + (s2 + s3);
+                }
+                fence_before_sync();
+                __syncwarp();
+                if (lane == 0) tma::mbar_arrive(&sy.acc_empty[buf]);
+                if (key < P.N) out[key] = colsum;
+            }
+        }
+    }
+    block_teardown(sy);
+}
+
+// raw[i] = sum of the parts; score[i] = max of raw over the centred window restricted to the
+// prefix i < N - w; +inf for the window tokens.  grid (ceil(N / 1024), U), 256 threads.
+constexpr int POOL_TILE = 1024;
+__global__ void __launch_bounds__(256)
+score_pool_parts(const float* __restrict__ raw_part, int parts, long long N, int w, int r, float* __restrict__ raw_out,
+                 float* __restrict__ score) {
+    __shared__ float rs[POOL_TILE + 16];
+    const int u = blockIdx.y;
+    const long long i0 = (long long)blockIdx.x * POOL_TILE;
+    const float* base = raw_part + (size_t)u * parts * N;
+    const long long P = N - w;
+    for (int e = threadIdx.x; e < POOL_TILE + 2 * r; e += 256) {
+        const long long i = i0 - r + e;
+        float v = -INFINITY;
+        if (i >= 0 && i < N) {
+            v = 0.f;
+            for (int p = 0; p < parts; ++p) v += base[(size_t)p * N + i];
+            if (raw_out && e >= r && e < POOL_TILE + r) raw_out[(size_t)u * N + i] = v;
+            if (i >= P) v = -INFINITY;           // pooling looks at the prefix only
+        }
+        rs[e] = v;
+    }
+    __syncthreads();
+    for (int e = threadIdx.x; e < POOL_TILE; e += 256) {
+        const long long i = i0 + e;
+        if (i >= N) break;
+        float best = INFINITY;
+        if (i < P) {
+            best = rs[e];
+            for (int k = 1; k <= 2 * r; ++k) best = fmaxf(best, rs[e + k]);
+        }
+        score[(size_t)u * N + i] = best;
+    }
+}
+
+}  // namespace stc
+}  // namespace vec
+#endif

@@ -39,6 +39,9 @@ SCORE_CASES = [
     (1, {"N": 70, "n_kv_heads": 1, "n_q_heads": 1, "window": 3, "pool_kernel": 1}),        # g=1, tiny window
     (0, {"N": 640, "head_dim": 128, "dtype": "bf16"}),
     (1, {"N": 900, "head_dim": 64, "n_kv_heads": 1, "n_q_heads": 2}),                      # bf16 d=64
+    (2, {"N": 1500, "n_layers": 20}),                           # 160 units: several items per block, ring wraps
+    (4, {"N": 3000, "n_layers": 3, "n_kv_heads": 2, "n_q_heads": 16}),    # 6 units x 4 row groups of 256 rows
+    (1, {"N": 777, "n_kv_heads": 1, "n_q_heads": 6, "window": 50}),       # 300 rows: second row group of 44 rows
 ]
 
 
