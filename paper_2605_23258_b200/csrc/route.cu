@@ -8,6 +8,7 @@
 // sums place the chosen indices in ascending order.  One thread block per unit.
 #include "common.cuh"
 #include "internal.h"
+#include "residual_tc.cuh"
 
 namespace vec {
 
@@ -213,9 +214,34 @@ static vector_status launch_residual(const Dims& dm, const void* K, const void* 
     return VECTOR_OK;
 }
 
+// bf16, head_dim 128: gather + tcgen05 residual kernel.
+static vector_status launch_residual_tc(const Dims& dm, const void* K, const void* V, const void* W, int64_t N,
+                                        const int32_t* idx, int64_t n_idx, float* eps, cudaStream_t st) {
+    if (n_idx == 0) return VECTOR_OK;
+    static bool configured = false;
+    if (!configured) {
+        VEC_CUDA_CHECK(cudaFuncSetAttribute(rtc::residual_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, rtc::SMEM_BYTES));
+        configured = true;
+    }
+    int* fault = kernel_fault_address();
+    if (!fault) return VECTOR_ERR_CUDA;
+    CUtensorMap mapW;
+    if (!tma::encode_bf16_3d(&mapW, W, 128, 128, (uint64_t)dm.LH, 256, 128 * 256, 64, 128)) return VECTOR_ERR_CUDA;
+    rtc::Params P;
+    P.U = dm.U; P.LH = dm.LH; P.n_idx = (int)n_idx; P.N = N;
+    P.tpu = (int)((n_idx + rtc::TILE - 1) / rtc::TILE);
+    P.n_tiles = (long long)dm.U * P.tpu;
+    const int blocks = (int)(P.n_tiles < 148 ? P.n_tiles : 148);
+    rtc::residual_tc<<<blocks, rtc::THREADS, rtc::SMEM_BYTES, st>>>((const __nv_bfloat16*)K, (const __nv_bfloat16*)V, mapW,
+                                                                    idx, P, eps, fault);
+    VEC_LAUNCH_CHECK();
+    return VECTOR_OK;
+}
+
 static vector_status residual_dispatch(const Dims& dm, const void* K, const void* V, const void* W, int64_t N,
                                        const int32_t* idx, int64_t n_idx, float* eps, cudaStream_t st) {
     if (dm.rope) return VECTOR_ERR_UNSUPPORTED;
+    if (dm.dtype == VECTOR_BF16 && dm.d == 128) return launch_residual_tc(dm, K, V, W, N, idx, n_idx, eps, st);
     if (dm.dtype == VECTOR_F32)
         return dm.d == 64 ? launch_residual<float, 64>(dm, K, V, W, N, idx, n_idx, eps, st)
                           : launch_residual<float, 128>(dm, K, V, W, N, idx, n_idx, eps, st);

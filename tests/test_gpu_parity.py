@@ -97,7 +97,9 @@ def test_pool_select_bit_exact(oracle, N, n_pool, ties):
 
 @pytest.mark.parametrize("base,over,n_idx", [(0, {}, 384), (1, {"N": 3000, "n_kv_heads": 2, "n_q_heads": 8}, 1001),
                                              (1, {"N": 500, "head_dim": 64, "n_kv_heads": 1, "n_q_heads": 2}, 77),
-                                             (0, {"N": 300, "head_dim": 128}, 300)])
+                                             (0, {"N": 300, "head_dim": 128}, 300),
+                                             # 160 units x 10 tiles: blocks own ranges that cross unit boundaries
+                                             (2, {"N": 1500, "n_layers": 20}, 1200)])
 def test_residual_parity(oracle, base, over, n_idx):
     wl = synth.shrink(synth.WORKLOADS[base], n_calib=1024, **over)
     K, V, _ = synth.context(wl, DEV)
