@@ -92,7 +92,7 @@ ScoreTcPlan score_tc_plan(int U, int R, int64_t N) {
 size_t score_ws_bytes(const Dims& D, int64_t N, bool need_raw) {
     if (score_uses_tc(D)) {
         const ScoreTcPlan p = score_tc_plan(D.U, D.R, N);
-        return align256((size_t)D.U * p.n_chunks * D.R * 2 * sizeof(float)) +     // (max, sum) partials
+        return align256((size_t)D.U * 2 * p.n_chunks * D.R * 2 * sizeof(float)) + // (reference, sum) partials, two per chunk
                align256((size_t)D.U * D.R * sizeof(float)) +                        // lse
                align256((size_t)D.U * 2 * p.RG * (size_t)N * sizeof(float));        // per-row-block key sums
     }

@@ -214,7 +214,7 @@ static vector_status launch_score_tc(const Dims& dm, const void* Q, const void* 
                                      float* raw_out, char* ws, cudaStream_t st) {
     const ScoreTcPlan pl = score_tc_plan(dm.U, dm.R, N);
     float2* partial = (float2*)ws;
-    ws += align256((size_t)dm.U * pl.n_chunks * dm.R * 2 * sizeof(float));
+    ws += align256((size_t)dm.U * 2 * pl.n_chunks * dm.R * 2 * sizeof(float));
     float* lse2 = (float*)ws;
     ws += align256((size_t)dm.U * dm.R * sizeof(float));
     float* raw_part = (float*)ws;
@@ -237,7 +237,7 @@ static vector_status launch_score_tc(const Dims& dm, const void* Q, const void* 
     const int blocks = pl.n_items < 148 ? pl.n_items : 148;
     stc::score_pass1_tc<<<blocks, stc::THREADS, stc::SMEM_BYTES, st>>>(mapQ, mapK, P, partial, fault);
     VEC_LAUNCH_CHECK();
-    stc::score_lse2_combine<<<dm.U, 256, 0, st>>>(partial, dm.R, pl.n_chunks, lse2);
+    stc::score_lse2_combine<<<dm.U, 256, 0, st>>>(partial, dm.R, 2 * pl.n_chunks, lse2);
     VEC_LAUNCH_CHECK();
     stc::score_pass2_tc<<<blocks, stc::THREADS, stc::SMEM_BYTES, st>>>(mapQ, mapK, P, lse2, raw_part, fault);
     VEC_LAUNCH_CHECK();

@@ -15,11 +15,13 @@
 // a key chunk on neighbouring blocks, so that a chunk is fetched from HBM once
 // and found in L2 by the other row groups.
 //
-// Roles inside a block (320 threads):
-//   warps 0-7  softmax: two warpgroups, each thread owns one TMEM lane
-//   warp  8    producer: TMA loads of the Q row group (once per item) and of the
+// Roles inside a block (576 threads):
+//   warps 0-15 softmax: two groups of two warpgroups; group 0 takes the block's even tiles,
+//              group 1 the odd ones, so that while one group waits for its accumulator to be
+//              refilled the other keeps the exponential unit busy; each thread owns one TMEM lane
+//   warp  16   producer: TMA loads of the Q row group (once per item) and of the
 //              K tiles into a 4-stage ring (128-byte swizzle, zero fill past the end)
-//   warp  9    MMA issuer (one thread) and owner of the TMEM allocation
+//   warp  17   MMA issuer (one thread) and owner of the TMEM allocation
 // All hand-offs are mbarriers; every wait is bounded and records a fault code.
 #ifndef VECTOR_SCORE_TC_CUH_
 #define VECTOR_SCORE_TC_CUH_
@@ -40,7 +42,7 @@ constexpr int BOX_BYTES = 16384;           // 128 rows x 128 bytes (64 bf16 of t
 constexpr int Q_BYTES = 4 * BOX_BYTES;     // [k half][256 rows][128 B]
 constexpr int K_STAGE_BYTES = 2 * BOX_BYTES;   // [k half][128 keys][128 B]
 constexpr int SMEM_BYTES = Q_BYTES + STAGES * K_STAGE_BYTES + 1024;
-constexpr int SOFTMAX_WARPS = 8;
+constexpr int SOFTMAX_WARPS = 16;
 constexpr int THREADS = 32 * (SOFTMAX_WARPS + 2);
 constexpr int TMEM_COLS = 512;
 
@@ -175,9 +177,152 @@ __device__ __forceinline__ void block_teardown(Sync& sy) {
     }
 }
 
+// sum_i exp2(v[i] * c + n[i]) over 32 accumulator columns; n is either one value for all columns
+// (pass 1: minus the row's reference) or a table in shared memory (pass 2: minus the rows' lse).
+// Written in three stages (all FMAs, all exponentials, a tree of adds) so that the 32 MUFU
+// operations issue back to back and nothing waits on the result of the one just before it.
+__device__ __forceinline__ void sum_tree32(const float (&e)[32], uint64_t& acc) {
+    uint64_t p[16];
+#pragma unroll
+    for (int i = 0; i < 16; ++i) p[i] = pack2(e[2 * i], e[2 * i + 1]);
+#pragma unroll
+    for (int w = 8; w >= 1; w >>= 1)
+#pragma unroll
+        for (int i = 0; i < w; ++i) p[i] = add2(p[i], p[i + w]);
+    acc = add2(acc, p[0]);
+}
+__device__ __forceinline__ float exp2_sum32(const uint32_t (&v)[32], float c, float n) {
+    const uint64_t c2 = pack2(c, c), n2 = pack2(n, n);
+    float x[32], e[32];
+#pragma unroll
+    for (int i = 0; i < 32; i += 2) unpack2(fma2(pack2(v[i], v[i + 1]), c2, n2), x[i], x[i + 1]);
+#pragma unroll
+    for (int i = 0; i < 32; ++i) e[i] = ex2(x[i]);
+    uint64_t acc = pack2(0.f, 0.f);
+    sum_tree32(e, acc);
+    float s0, s1;
+    unpack2(acc, s0, s1);
+    return s0 + s1;
+}
+__device__ __forceinline__ void exp2_acc32(const uint32_t (&v)[32], float c, const float4* __restrict__ n, uint64_t& acc) {
+    const uint64_t c2 = pack2(c, c);
+    float x[32], e[32];
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+        const float4 n4 = n[i];
+        unpack2(fma2(pack2(v[4 * i], v[4 * i + 1]), c2, pack2(n4.x, n4.y)), x[4 * i], x[4 * i + 1]);
+        unpack2(fma2(pack2(v[4 * i + 2], v[4 * i + 3]), c2, pack2(n4.z, n4.w)), x[4 * i + 2], x[4 * i + 3]);
+    }
+#pragma unroll
+    for (int i = 0; i < 32; ++i) e[i] = ex2(x[i]);
+    sum_tree32(e, acc);
+}
+__device__ __forceinline__ float max32(const uint32_t (&v)[32]) {
+    float a = max3(__uint_as_float(v[0]), __uint_as_float(v[1]), __uint_as_float(v[2]));
+    float b = max3(__uint_as_float(v[3]), __uint_as_float(v[4]), __uint_as_float(v[5]));
+#pragma unroll
+    for (int i = 6; i < 30; i += 4) {
+        a = max3(a, __uint_as_float(v[i]), __uint_as_float(v[i + 1]));
+        b = max3(b, __uint_as_float(v[i + 2]), __uint_as_float(v[i + 3]));
+    }
+    return max3(a, b, fmaxf(__uint_as_float(v[30]), __uint_as_float(v[31])));
+}
+
+// One accumulator tile of pass 1 for this thread's row: 128 columns in four TMEM loads.  The
+// buffer is handed back to the MMA warp as soon as the last load has completed.  The running sum l
+// is kept against a reference m that lags behind the true maximum: the exponentials of a chunk do
+// not wait for the chunk's maximum, and only when a logit exceeds the reference by more than 2^64
+// (always on an item's first chunk, where m = -inf) is the reference moved and the chunk summed again.
+template <bool MASKED>
+__device__ __forceinline__ void softmax_tile_pass1(uint32_t taddr, float c, long long key0, long long last_visible,
+                                                   float& m, float& l, uint64_t& empty_bar, int lane) {
+    uint32_t ra[32], rb[32];
+    tmem_ld32(taddr, ra);
+#pragma unroll
+    for (int ch = 0; ch < 4; ++ch) {
+        uint32_t (&cur)[32] = (ch & 1) ? rb : ra;
+        uint32_t (&nxt)[32] = (ch & 1) ? ra : rb;
+        tmem_ld_wait(cur);
+        if (ch < 3) {
+            tmem_ld32(taddr + (ch + 1) * 32, nxt);
+        } else {
+            fence_before_sync();
+            __syncwarp();
+            if (lane == 0) tma::mbar_arrive(&empty_bar);
+        }
+        if (!MASKED) {
+            const float cm = max32(cur) * c;
+            float s;
+            bool again;
+#pragma unroll 1
+            do {
+                s = exp2_sum32(cur, c, -m);
+                again = cm > m + 64.f;
+                if (again) { l *= ex2(m - cm); m = cm; }
+            } while (again);
+            l += s;
+        } else {
+            float v[32];
+#pragma unroll
+            for (int i = 0; i < 32; ++i) v[i] = key0 + ch * 32 + i > last_visible ? -INFINITY : __uint_as_float(cur[i]);
+            float cm = v[0];
+#pragma unroll
+            for (int i = 1; i < 32; ++i) cm = fmaxf(cm, v[i]);
+            const float m_new = fmaxf(m, cm * c);
+            if (m_new > -INFINITY) {     // false only while every key so far is masked
+                l *= ex2(m - m_new);     // exp2(-inf) = 0 on the first visible chunk
+                float s0 = 0.f;
+#pragma unroll
+                for (int i = 0; i < 32; ++i) s0 += ex2(fmaf(v[i], c, -m_new));
+                l += s0;
+                m = m_new;
+            }
+        }
+    }
+}
+
+// One accumulator tile of pass 2 for this thread's key: sum over 128 rows of exp2(logit2 - lse2[row]).
+// Masked tiles: row j of the window (j0 = window index of the tile's first row, advancing cyclically
+// with period w) sees this key only if key - (N - w) <= j.
+template <bool MASKED>
+__device__ __forceinline__ float softmax_tile_pass2(uint32_t taddr, float c, const float* nl_w, long long key_rel,
+                                                    int j0, int w, uint64_t& empty_bar, int lane) {
+    uint32_t ra[32], rb[32];
+    tmem_ld32(taddr, ra);
+    uint64_t acc = pack2(0.f, 0.f);
+    float sm = 0.f;
+    int j = j0;
+#pragma unroll
+    for (int ch = 0; ch < 4; ++ch) {
+        uint32_t (&cur)[32] = (ch & 1) ? rb : ra;
+        uint32_t (&nxt)[32] = (ch & 1) ? ra : rb;
+        tmem_ld_wait(cur);
+        if (ch < 3) {
+            tmem_ld32(taddr + (ch + 1) * 32, nxt);
+        } else {
+            fence_before_sync();
+            __syncwarp();
+            if (lane == 0) tma::mbar_arrive(&empty_bar);
+        }
+        if (!MASKED) {
+            exp2_acc32(cur, c, reinterpret_cast<const float4*>(nl_w + ch * 32), acc);
+        } else {
+#pragma unroll
+            for (int i = 0; i < 32; ++i) {
+                const float p = ex2(fmaf(__uint_as_float(cur[i]), c, nl_w[ch * 32 + i]));
+                if (key_rel <= j) sm += p;
+                if (++j == w) j = 0;
+            }
+        }
+    }
+    float s0, s1;
+    unpack2(acc, s0, s1);
+    return (s0 + s1) + sm;
+}
+
 // ---- pass 1 -----------------------------------------------------------------
-// partial[(u * n_chunks + chunk) * R + row] = (running max, sum of exp2) of the row over the
-// chunk's visible keys, in units of log2 (logit * scale * log2 e).  grid: one block per SM.
+// partial[((u * n_chunks + chunk) * 2 + group) * R + row] = (reference, sum of exp2 against it) of the
+// row over the visible keys of the chunk's even (group 0) or odd (group 1) tiles, in units of log2 (logit * scale * log2 e).  grid: one block per SM.
 __global__ void __launch_bounds__(THREADS, 1)
 score_pass1_tc(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ CUtensorMap mapK, const Params P,
                float2* __restrict__ partial, int* __restrict__ fault) {
@@ -194,7 +339,7 @@ score_pass1_tc(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
     } else if (warp == SOFTMAX_WARPS + 1) {
         if (lane == 0) mma_role<1>(P, sy, Qs, Ks, fault);
     } else {
-        const int wg = warp >> 2, quarter = warp & 3;
+        const int grp = warp >> 3, wg = (warp >> 2) & 1, quarter = warp & 3;
         const uint32_t lane_addr = sy.tmem_base + ((uint32_t)(quarter * 32) << 16);
         const long long vis0 = P.N - P.w;               // keys below this index are visible to every row
         uint32_t tcount = 0;
@@ -206,54 +351,22 @@ score_pass1_tc(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
             const long long last_visible = vis0 + (row % P.w);
             float m = -INFINITY, l = 0.f;
             for (int t = im.t0; t < im.t1; ++t, ++tcount) {
+                if ((int)(tcount & 1) != grp) continue;
                 const uint32_t buf = (tcount & 1) * 2 + wg, use = tcount >> 1;
                 if (!tma::mbar_wait(&sy.acc_full[buf], use & 1, fault, 31)) { ok = false; break; }
                 fence_after_sync();
                 if (wg_active) {
                     const uint32_t taddr = lane_addr + buf * 128;
                     const long long key0 = (long long)t * KT;
-                    const bool masked = key0 + KT > vis0;
-                    uint32_t ra[32], rb[32];
-                    tmem_ld32(taddr, ra);
-#pragma unroll
-                    for (int ch = 0; ch < 4; ++ch) {
-                        uint32_t (&cur)[32] = (ch & 1) ? rb : ra;
-                        uint32_t (&nxt)[32] = (ch & 1) ? ra : rb;
-                        tmem_ld_wait(cur);
-                        if (ch < 3) tmem_ld32(taddr + (ch + 1) * 32, nxt);
-                        float v[32];
-#pragma unroll
-                        for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(cur[i]);
-                        if (masked) {
-#pragma unroll
-                            for (int i = 0; i < 32; ++i)
-                                if (key0 + ch * 32 + i > last_visible) v[i] = -INFINITY;
-                        }
-                        float cm0 = fmaxf(v[0], v[1]), cm1 = fmaxf(v[2], v[3]);
-#pragma unroll
-                        for (int i = 4; i < 32; i += 2) { cm0 = fmaxf(cm0, v[i]); cm1 = fmaxf(cm1, v[i + 1]); }
-                        const float m_new = fmaxf(m, fmaxf(cm0, cm1) * P.c);
-                        if (m_new > -INFINITY) {         // false only while every key so far is masked
-                            l *= ex2(m - m_new);         // exp2(-inf) = 0 on the first visible chunk
-                            const float neg = -m_new;
-                            float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
-#pragma unroll
-                            for (int i = 0; i < 32; i += 4) {
-                                s0 += ex2(fmaf(v[i], P.c, neg));
-                                s1 += ex2(fmaf(v[i + 1], P.c, neg));
-                                s2 += ex2(fmaf(v[i + 2], P.c, neg));
-                                s3 += ex2(fmaf(v[i + 3], P.c, neg));
-                            }
-                            l += (s0 + s1) + (s2 + s3);
-                            m = m_new;
-                        }
-                    }
+                    if (key0 + KT <= vis0) softmax_tile_pass1<false>(taddr, P.c, 0, 0, m, l, sy.acc_empty[buf], lane);
+                    else softmax_tile_pass1<true>(taddr, P.c, key0, last_visible, m, l, sy.acc_empty[buf], lane);
+                } else {
+                    __syncwarp();
+                    if (lane == 0) tma::mbar_arrive(&sy.acc_empty[buf]);
                 }
-                fence_before_sync();
-                __syncwarp();
-                if (lane == 0) tma::mbar_arrive(&sy.acc_empty[buf]);
             }
-            if (ok && row < P.R) partial[((size_t)im.u * P.n_chunks + im.chunk) * P.R + row] = make_float2(m, l);
+            if (ok && row < P.R)
+                partial[(((size_t)im.u * P.n_chunks + im.chunk) * 2 + grp) * P.R + row] = make_float2(m, l);
         }
     }
     block_teardown(sy);
@@ -282,7 +395,7 @@ score_pass2_tc(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
                const float* __restrict__ lse2, float* __restrict__ raw_part, int* __restrict__ fault) {
     extern __shared__ unsigned char smem_raw[];
     __shared__ Sync sy;
-    __shared__ __align__(16) float neg_lse[RG_ROWS];       // -lse2 of the item's rows; -inf for padding rows
+    __shared__ __align__(16) float neg_lse[SOFTMAX_WARPS][128];
     unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     unsigned char* Qs = smem;
     unsigned char* Ks = smem + Q_BYTES;
@@ -294,26 +407,27 @@ score_pass2_tc(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
     } else if (warp == SOFTMAX_WARPS + 1) {
         if (lane == 0) mma_role<2>(P, sy, Qs, Ks, fault);
     } else {
-        const int wg = warp >> 2, quarter = warp & 3;
+        const int grp = warp >> 3, wg = (warp >> 2) & 1, quarter = warp & 3;
         const uint32_t lane_addr = sy.tmem_base + ((uint32_t)(quarter * 32) << 16);
         const int key_in_tile = quarter * 32 + lane;
         const long long vis0 = P.N - P.w;
+        float* nl_w = neg_lse[warp];                   // this warp's copy of -lse2 of its 128 rows
         uint32_t tcount = 0;
         bool ok = true;
-        for (int it = blockIdx.x; it < P.n_items; it += gridDim.x) {
+        for (int it = blockIdx.x; it < P.n_items && ok; it += gridDim.x) {
             const Item im = decode_item(it, P);
-            // the item's normalisers: all softmax threads leave the old table, refill it, publish it
-            asm volatile("bar.sync 1, 256;\n" ::: "memory");
-            {
-                const int row = im.rg * RG_ROWS + threadIdx.x;
-                neg_lse[threadIdx.x] = row < P.R ? -lse2[(size_t)im.u * P.R + row] : -INFINITY;
-            }
-            asm volatile("bar.sync 1, 256;\n" ::: "memory");
-            if (!ok) continue;                       // keep meeting the others at the barriers above
             const bool wg_active = im.rg * RG_ROWS + wg * 128 < P.R;
             const int row_base = im.rg * RG_ROWS + wg * 128;
+            __syncwarp();
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+                const int row = row_base + k * 32 + lane;
+                nl_w[k * 32 + lane] = row < P.R ? -lse2[(size_t)im.u * P.R + row] : -INFINITY;   // -inf: padding rows add 0
+            }
+            __syncwarp();
             float* out = raw_part + ((size_t)im.u * 2 * P.RG + 2 * im.rg + wg) * P.N;
             for (int t = im.t0; t < im.t1; ++t, ++tcount) {
+                if ((int)(tcount & 1) != grp) continue;
                 const uint32_t buf = tcount & 1, use = tcount >> 1;
                 if (!tma::mbar_wait(&sy.acc_full[buf], use & 1, fault, 32)) { ok = false; break; }
                 fence_after_sync();
@@ -321,42 +435,15 @@ score_pass2_tc(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
                 float colsum = 0.f;
                 if (wg_active) {
                     const uint32_t taddr = lane_addr + buf * 256 + wg * 128;
-                    const bool masked = (long long)t * KT + KT > vis0;
-                    uint32_t ra[32], rb[32];
-                    tmem_ld32(taddr, ra);
-                    float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
-#pragma unroll
-                    for (int ch = 0; ch < 4; ++ch) {
-                        uint32_t (&cur)[32] = (ch & 1) ? rb : ra;
-                        uint32_t (&nxt)[32] = (ch & 1) ? ra : rb;
-                        tmem_ld_wait(cur);
-                        if (ch < 3) tmem_ld32(taddr + (ch + 1) * 32, nxt);
-                        const float4* nl = reinterpret_cast<const float4*>(neg_lse + wg * 128 + ch * 32);
-                        if (!masked) {
-#pragma unroll
-                            for (int i = 0; i < 8; ++i) {
-                                const float4 n4 = nl[i];
-                                s0 += ex2(fmaf(__uint_as_float(cur[4 * i]), P.c, n4.x));
-                                s1 += ex2(fmaf(__uint_as_float(cur[4 * i + 1]), P.c, n4.y));
-                                s2 += ex2(fmaf(__uint_as_float(cur[4 * i + 2]), P.c, n4.z));
-                                s3 += ex2(fmaf(__uint_as_float(cur[4 * i + 3]), P.c, n4.w));
-                            }
-                        } else {
-                            // row r = a * w + j sees the keys up to N - w + j
-#pragma unroll
-                            for (int i = 0; i < 32; ++i) {
-                                const int j = (row_base + ch * 32 + i) % P.w;
-                                const float p = ex2(fmaf(__uint_as_float(cur[i]), P.c, neg_lse[wg * 128 + ch * 32 + i]));
-                                if (key <= vis0 + j) s0 += p;
-                            }
-                        }
-                    }
-                    colsum = (s0 + s1) + (s2 + s3);
+                    if ((long long)t * KT + KT <= vis0)
+                        colsum = softmax_tile_pass2<false>(taddr, P.c, nl_w, 0, 0, 0, sy.acc_empty[buf], lane);
+                    else
+                        colsum = softmax_tile_pass2<true>(taddr, P.c, nl_w, key - vis0, row_base % P.w, P.w, sy.acc_empty[buf], lane);
+                } else {
+                    __syncwarp();
+                    if (lane == 0) tma::mbar_arrive(&sy.acc_empty[buf]);
                 }
-                fence_before_sync();
-                __syncwarp();
-                if (lane == 0) tma::mbar_arrive(&sy.acc_empty[buf]);
-                if (key < P.N) out[key] = colsum;
+                if (key < P.N) out[key] = colsum;           // zero for a row block past the last row
             }
         }
     }
