@@ -191,13 +191,48 @@ __device__ __forceinline__ void sum_tree32(const float (&e)[32], uint64_t& acc) 
         for (int i = 0; i < w; ++i) p[i] = add2(p[i], p[i + w]);
     acc = add2(acc, p[0]);
 }
+// The exponential unit (16 results per clock per SM) is what bounds both passes, so POLY16 of every
+// 16 exponentials are evaluated on the FMA pipe instead: 2^x = 2^n p(f) with n = round(x),
+// f = x - n in [-1/2, 1/2] and p the degree-4 minimax polynomial of 2^f (relative error 2.7e-6);
+// n is added to the exponent field.  x is clamped at -126 (results below 2^-126 do not matter
+// to a sum whose largest term is of order one).
+#ifndef VECTOR_SCORE_POLY16
+#define VECTOR_SCORE_POLY16 4
+#endif
+constexpr int POLY16 = VECTOR_SCORE_POLY16;
+__device__ __forceinline__ void exp2_poly_pair(float x0, float x1, float& e0, float& e1) {
+    const float magic = 12582912.f;                    // 1.5 * 2^23: adding it leaves round(x) in the low mantissa bits
+    x0 = fmaxf(x0, -126.f);
+    x1 = fmaxf(x1, -126.f);
+    const uint64_t x2 = pack2(x0, x1);
+    const uint64_t t2 = add2(x2, pack2(magic, magic));
+    const uint64_t n2 = add2(t2, pack2(-magic, -magic));
+    const uint64_t f2 = fma2(n2, pack2(-1.f, -1.f), x2);
+    uint64_t p2 = pack2(0.009570101276040077f, 0.009570101276040077f);
+    p2 = fma2(p2, f2, pack2(0.05591785907745361f, 0.05591785907745361f));
+    p2 = fma2(p2, f2, pack2(0.240247443318367f, 0.240247443318367f));
+    p2 = fma2(p2, f2, pack2(0.6931217908859253f, 0.6931217908859253f));
+    p2 = fma2(p2, f2, pack2(0.9999992847442627f, 0.9999992847442627f));
+    float p0, p1, t0, t1;
+    unpack2(p2, p0, p1);
+    unpack2(t2, t0, t1);
+    e0 = __uint_as_float(__float_as_uint(p0) + (__float_as_uint(t0) << 23));
+    e1 = __uint_as_float(__float_as_uint(p1) + (__float_as_uint(t1) << 23));
+}
+// e[i] = 2^x[i] for 32 exponents: the first POLY16 of every 16 by polynomial, the rest by MUFU.
+__device__ __forceinline__ void exp2_32(const float (&x)[32], float (&e)[32]) {
+#pragma unroll
+    for (int i = 0; i < 32; i += 2) {
+        if ((i & 15) < POLY16) exp2_poly_pair(x[i], x[i + 1], e[i], e[i + 1]);
+        else { e[i] = ex2(x[i]); e[i + 1] = ex2(x[i + 1]); }
+    }
+}
 __device__ __forceinline__ float exp2_sum32(const uint32_t (&v)[32], float c, float n) {
     const uint64_t c2 = pack2(c, c), n2 = pack2(n, n);
     float x[32], e[32];
 #pragma unroll
     for (int i = 0; i < 32; i += 2) unpack2(fma2(pack2(v[i], v[i + 1]), c2, n2), x[i], x[i + 1]);
-#pragma unroll
-    for (int i = 0; i < 32; ++i) e[i] = ex2(x[i]);
+    exp2_32(x, e);
     uint64_t acc = pack2(0.f, 0.f);
     sum_tree32(e, acc);
     float s0, s1;
@@ -213,8 +248,7 @@ __device__ __forceinline__ void exp2_acc32(const uint32_t (&v)[32], float c, con
         unpack2(fma2(pack2(v[4 * i], v[4 * i + 1]), c2, pack2(n4.x, n4.y)), x[4 * i], x[4 * i + 1]);
         unpack2(fma2(pack2(v[4 * i + 2], v[4 * i + 3]), c2, pack2(n4.z, n4.w)), x[4 * i + 2], x[4 * i + 3]);
     }
-#pragma unroll
-    for (int i = 0; i < 32; ++i) e[i] = ex2(x[i]);
+    exp2_32(x, e);
     sum_tree32(e, acc);
 }
 __device__ __forceinline__ float max32(const uint32_t (&v)[32]) {
