@@ -1,22 +1,27 @@
 // Decode attention over the mixed cache for bf16, head_dim 128 (HBM-bound).
 //
-// Every K/V row is read once.  Each unit's rows are cut into 64-key tiles (a
-// retained tile = 64 keys + their 64 values = 32 KB, weight 2; a key-only tile
-// = 64 keys = 16 KB, weight 1) and the weighted global tile sequence is dealt
-// out in equal contiguous ranges to a fixed grid of persistent blocks (two per
-// SM): the load is balanced by bytes and there is no wave tail.
+// Every K/V row is read once.  Each unit's rows are cut into 32 KB tiles -- a
+// retained tile = 64 keys + their 64 values, a key-only tile = 128 keys -- and
+// the global tile sequence is dealt out in equal contiguous ranges to one
+// persistent block per SM: the load is balanced by bytes and there is no wave tail.
 //
 // Inside a block one producer thread streams the tiles with TMA
 // (cp.async.bulk.tensor, 128-byte swizzle, zero fill past the end of a pool)
-// into a 3-stage ring guarded by full/empty mbarriers; four consumer warps take
-// 16 keys of every tile each and never synchronise with one another otherwise:
-//   S = Q K^T      m16n8k16 bf16 MMA, the g query heads padded to the MMA rows
-//   online softmax in fp32 registers (exp2 with the scale folded in)
+// into six 32 KB slots guarded by full/empty mbarriers.  Tiles go round-robin
+// to three consumer warps, each with two slots of its own (tile i: warp i % 3,
+// slot i % 6), so a warp sees every phase of the barriers it waits on -- with a
+// parity wait, a waiter that skipped a phase could take an old completion for
+// the one it wants, since TMA copies land out of order.  A warp works through a
+// whole tile on its own, 64 keys at a time, and never synchronises with the others:
+//   S = Q K^T      64 m16n8k16 bf16 MMAs (eight independent accumulators), the g
+//                  query heads padded to the MMA rows
+//   online softmax in fp32 registers, one rescale per 64 keys (exp2, scale folded in)
 //   O += P V  (retained tile)  or  A += P K  (key-only tile: the p-weighted key
 //             sum that the merge step multiplies by W); P enters as bf16 hi in
 //             MMA rows 0-7 and bf16 lo in rows 8-15, one MMA for both parts
-// The ring keeps running across unit boundaries, where each warp writes its
-// partial record for the finished unit.  The merge kernel combines a unit's
+// A warp keeps one running state (m, l, O or A) per unit and writes it as its
+// partial record when it leaves the unit; a warp that met no tile of a unit the
+// block touches writes an empty record.  The merge kernel combines a unit's
 // records, applies W and normalises.
 #ifndef VECTOR_DECODE_BF16_CUH_
 #define VECTOR_DECODE_BF16_CUH_
@@ -27,53 +32,40 @@
 namespace vec {
 namespace dbf {
 
-constexpr int TILE = 64;                     // keys per tile
-constexpr int STAGES = 3;
-constexpr int STAGE_BYTES = 32768;           // K tile (2 swizzled 64x128B boxes) + V tile (2 boxes)
+constexpr int KEYS = 64;                     // keys per softmax step (and per TMA box)
+constexpr int SLOTS = 6;                     // a multiple of CONSUMER_WARPS: a slot always serves the same warp
+constexpr int SLOT_BYTES = 32768;            // retained: K 16 KB | V 16 KB; key-only: keys 0-63 | keys 64-127
+constexpr int HALF_BYTES = 16384;            // 64 rows of 256 B as two swizzled 64 x 128 B boxes
 constexpr int BOX_BYTES = 8192;              // 64 rows x 128 bytes
-constexpr int CONSUMER_WARPS = 4;
+constexpr int CONSUMER_WARPS = 3;
 constexpr int THREADS = 32 * (CONSUMER_WARPS + 1);
 constexpr int REC = 4 + 2 * 128;             // m, l, value-scale, pad, acc_v[128], acc_k[128]
-constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024;   // + alignment slack; barriers live in static smem
-constexpr int MAX_BLOCKS = 2 * 148;
+constexpr int SMEM_BYTES = SLOTS * SLOT_BYTES + 1024;   // + alignment slack; barriers live in static smem
+constexpr int MAX_BLOCKS = 148;
 
-// How the weighted tile sequence is dealt to blocks; the same arithmetic runs on host and device.
+// How the tile sequence is dealt to blocks; the same arithmetic runs on host and device.
 struct Plan {
     int n_rt, n_at, n_tiles;   // retained / key-only / all tiles per unit
-    int Wu;                    // weight of a unit = 2 n_rt + n_at
-    long long TW;              // weight of all units
+    long long T;               // tiles of all units
     int B;                     // blocks
     int s_max;                 // record slots per unit
 };
 __host__ __device__ inline Plan make_plan(int U, long long n_ret, long long n_apx) {
     Plan p;
-    p.n_rt = (int)((n_ret + TILE - 1) / TILE);
-    p.n_at = (int)((n_apx + TILE - 1) / TILE);
+    p.n_rt = (int)((n_ret + KEYS - 1) / KEYS);
+    p.n_at = (int)((n_apx + 2 * KEYS - 1) / (2 * KEYS));
     p.n_tiles = p.n_rt + p.n_at;
-    p.Wu = 2 * p.n_rt + p.n_at;
-    p.TW = (long long)U * p.Wu;
-    long long b = p.TW / 8;                      // at least 8 weight units (4+ tiles) per block
+    p.T = (long long)U * p.n_tiles;
+    long long b = p.T / 2;                       // at least two tiles per block
     if (b > MAX_BLOCKS) b = MAX_BLOCKS;
     if (b > 11LL * U) b = 11LL * U;              // at most 12 record slots per unit (merge kernel limit)
     p.B = (int)(b < 1 ? 1 : b);
     p.s_max = (p.B + U - 1) / U + 1;
     return p;
 }
-// Block b owns the tiles whose start weight lies in [b TW / B, (b+1) TW / B).
-__host__ __device__ inline long long weight_begin(int b, const Plan& p) { return (long long)b * p.TW / p.B; }
-__host__ __device__ inline int block_of_weight(long long s, const Plan& p) { return (int)(((s + 1) * p.B - 1) / p.TW); }
-// global index of the first tile whose start weight is >= x
-__host__ __device__ inline long long tile_from_weight(long long x, const Plan& p) {
-    long long u = x / p.Wu;
-    int r = (int)(x - u * p.Wu);
-    int t = r <= 2 * p.n_rt ? (r + 1) / 2 : p.n_rt + (r - 2 * p.n_rt);
-    return u * p.n_tiles + t;
-}
-__host__ __device__ inline long long unit_first_weight(int u, const Plan& p) { return (long long)u * p.Wu; }
-__host__ __device__ inline long long unit_last_weight(int u, const Plan& p) {   // start weight of the unit's last tile
-    int t = p.n_tiles - 1;
-    return (long long)u * p.Wu + (t < p.n_rt ? 2 * t : 2 * p.n_rt + (t - p.n_rt));
-}
+// Block b owns the tiles [b T / B, (b+1) T / B).
+__host__ __device__ inline long long tile_begin(int b, const Plan& p) { return (long long)b * p.T / p.B; }
+__host__ __device__ inline int block_of_tile(long long x, const Plan& p) { return (int)(((x + 1) * p.B - 1) / p.T); }
 
 __device__ __forceinline__ void ldsm_x4(uint32_t addr, uint32_t& r0, uint32_t& r1, uint32_t& r2, uint32_t& r3) {
     asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];\n"
@@ -104,31 +96,33 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
     return *reinterpret_cast<uint32_t*>(&v);
 }
 
+static_assert(SLOTS % CONSUMER_WARPS == 0, "a slot must always be consumed by the same warp");
+
 struct Maps {
     CUtensorMap ret_k, ret_v, apx_k;     // rank 3: (128 dims, pool rows, U units), box 64 x 64 x 1, 128B swizzle
 };
 
 // grid (plan.B), THREADS threads, SMEM_BYTES dynamic shared memory.
-// partial: [U][s_max][4 warps][g][REC]; slot of (unit u, block b) = b - block_of_weight(first weight of u).
-__global__ void __launch_bounds__(THREADS, 2)
+// partial: [U][s_max][CONSUMER_WARPS][g][REC]; slot of (unit u, block b) = b - block_of_tile(first tile of u).
+__global__ void __launch_bounds__(THREADS, 1)
 decode_stream_bf16_d128(const __nv_bfloat16* __restrict__ q, const __grid_constant__ Maps maps, Plan pl, int n_ret,
                         int n_apx, int g, float scale_log2e, float* __restrict__ partial, int* __restrict__ fault) {
     extern __shared__ unsigned char smem_raw[];
-    __shared__ __align__(8) uint64_t full_bar[STAGES];
-    __shared__ __align__(8) uint64_t empty_bar[STAGES];
+    __shared__ __align__(8) uint64_t full_bar[SLOTS];
+    __shared__ __align__(8) uint64_t empty_bar[SLOTS];
     // 128B-swizzled TMA boxes want 1024-byte aligned destinations
     unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     const int b = blockIdx.x;
     const int tid = threadIdx.x, lane = tid & 31, wq = tid >> 5;
-    const long long gt_lo = tile_from_weight(weight_begin(b, pl), pl);
-    const long long gt_hi = tile_from_weight(weight_begin(b + 1, pl), pl);
+    const long long gt_lo = tile_begin(b, pl), gt_hi = tile_begin(b + 1, pl);
     if (gt_lo >= gt_hi) return;
     const int n_my = (int)(gt_hi - gt_lo);
     const int u0 = (int)(gt_lo / pl.n_tiles), t0 = (int)(gt_lo - (long long)u0 * pl.n_tiles);
+    const int u_last = (int)((gt_hi - 1) / pl.n_tiles);
 
     if (tid == 0) {
 #pragma unroll
-        for (int s = 0; s < STAGES; ++s) { tma::mbar_init(&full_bar[s], 1); tma::mbar_init(&empty_bar[s], CONSUMER_WARPS); }
+        for (int s = 0; s < SLOTS; ++s) { tma::mbar_init(&full_bar[s], 1); tma::mbar_init(&empty_bar[s], 1); }
         tma::mbar_fence_init();
     }
     __syncthreads();
@@ -138,24 +132,23 @@ decode_stream_bf16_d128(const __nv_bfloat16* __restrict__ q, const __grid_consta
         if (lane == 0) {
             tma::prefetch_map(&maps.ret_k); tma::prefetch_map(&maps.ret_v); tma::prefetch_map(&maps.apx_k);
             int u = u0, t = t0;
-            bool ok = true;
-            for (int i = 0; i < n_my && ok; ++i) {
-                const int s = i % STAGES, round = i / STAGES;
-                if (round > 0) ok = tma::mbar_wait(&empty_bar[s], (round - 1) & 1, fault, 1);
-                if (!ok) break;
-                unsigned char* st = smem + s * STAGE_BYTES;
+            for (int i = 0; i < n_my; ++i) {
+                const int s = i % SLOTS, round = i / SLOTS;
+                if (round > 0 && !tma::mbar_wait(&empty_bar[s], (round - 1) & 1, fault, 1)) break;
+                unsigned char* st = smem + s * SLOT_BYTES;
+                tma::mbar_expect_tx(&full_bar[s], SLOT_BYTES);
                 if (t < pl.n_rt) {
-                    const int row0 = t * TILE;
-                    tma::mbar_expect_tx(&full_bar[s], 4 * BOX_BYTES);
+                    const int row0 = t * KEYS;
                     tma::load_3d(st, &maps.ret_k, 0, row0, u, &full_bar[s]);
                     tma::load_3d(st + BOX_BYTES, &maps.ret_k, 64, row0, u, &full_bar[s]);
-                    tma::load_3d(st + 2 * BOX_BYTES, &maps.ret_v, 0, row0, u, &full_bar[s]);
-                    tma::load_3d(st + 3 * BOX_BYTES, &maps.ret_v, 64, row0, u, &full_bar[s]);
+                    tma::load_3d(st + HALF_BYTES, &maps.ret_v, 0, row0, u, &full_bar[s]);
+                    tma::load_3d(st + HALF_BYTES + BOX_BYTES, &maps.ret_v, 64, row0, u, &full_bar[s]);
                 } else {
-                    const int row0 = (t - pl.n_rt) * TILE;
-                    tma::mbar_expect_tx(&full_bar[s], 2 * BOX_BYTES);
+                    const int row0 = (t - pl.n_rt) * 2 * KEYS;
                     tma::load_3d(st, &maps.apx_k, 0, row0, u, &full_bar[s]);
                     tma::load_3d(st + BOX_BYTES, &maps.apx_k, 64, row0, u, &full_bar[s]);
+                    tma::load_3d(st + HALF_BYTES, &maps.apx_k, 0, row0 + KEYS, u, &full_bar[s]);
+                    tma::load_3d(st + HALF_BYTES + BOX_BYTES, &maps.apx_k, 64, row0 + KEYS, u, &full_bar[s]);
                 }
                 if (++t == pl.n_tiles) { t = 0; ++u; }
             }
@@ -165,23 +158,21 @@ decode_stream_bf16_d128(const __nv_bfloat16* __restrict__ q, const __grid_consta
 
     // ---------------------------------------------------------------------- consumers
     const int gid = lane >> 2, tig = lane & 3;
-    const int kr0 = wq * 16;                       // this warp's 16 keys inside every tile
     // per-lane ldmatrix geometry (swizzle: 16-byte chunk index XOR (row & 7), rows are 128 bytes)
     const int mat = lane >> 3, r8 = lane & 7;
-    const uint32_t qk_row = (uint32_t)(kr0 + r8 + (mat >> 1) * 8) * 128u;      // QK: matrices = (keys 0-7|8-15) x (chunk lo|hi)
+    const uint32_t qk_row = (uint32_t)(r8 + (mat >> 1) * 8) * 128u;      // QK: matrices = (keys 0-7|8-15) x (chunk lo|hi)
     const uint32_t qk_x = (uint32_t)(((mat & 1) ^ r8) << 4);
-    const uint32_t pv_row = (uint32_t)(kr0 + r8 + (mat & 1) * 8) * 128u;       // PV: matrices = (chunk lo|hi) x (keys 0-7|8-15)
+    const uint32_t pv_row = (uint32_t)(r8 + (mat & 1) * 8) * 128u;       // PV: matrices = (chunk lo|hi) x (keys 0-7|8-15)
     const uint32_t pv_x = (uint32_t)(((mat >> 1) ^ r8) << 4);
 
     uint32_t qa[8][2];
     float acc[16][4];                  // [dim tile][c0,c1: P_hi rows | c2,c3: P_lo rows]
-    float zz[4][2];
     float m = -INFINITY, l = 0.f, stash_scale = 1.f;
     bool stashed = false;
-    int u = u0, t = t0;
 
     auto record_of = [&](int unit) -> float* {
-        const int slot = b - block_of_weight(unit_first_weight(unit, pl), pl);
+        int slot = b - block_of_tile((long long)unit * pl.n_tiles, pl);
+        if (slot < 0 || slot >= pl.s_max) { atomicCAS(fault, 0, 5); slot = 0; }     // cannot happen; never write out of bounds
         return partial + ((((size_t)unit * pl.s_max + slot) * CONSUMER_WARPS + wq) * g + gid) * REC;
     };
     auto load_q = [&](int unit) {
@@ -201,6 +192,7 @@ decode_stream_bf16_d128(const __nv_bfloat16* __restrict__ q, const __grid_consta
 #pragma unroll
         for (int n = 0; n < 16; ++n) { acc[n][0] = acc[n][1] = acc[n][2] = acc[n][3] = 0.f; }
     };
+    // Writes this warp's record of `unit` (an all-zero one with m = -inf if it met none of its tiles).
     auto flush = [&](int unit) {
         float lt = l;
         lt += __shfl_xor_sync(0xffffffffu, lt, 1);
@@ -218,86 +210,101 @@ decode_stream_bf16_d128(const __nv_bfloat16* __restrict__ q, const __grid_consta
         zero_acc();
         m = -INFINITY; l = 0.f; stash_scale = 1.f; stashed = false;
     };
-
-    load_q(u);
-    zero_acc();
-    for (int i = 0; i < n_my; ++i) {
-        const int s = i % STAGES, round = i / STAGES;
-        if (!tma::mbar_wait(&full_bar[s], round & 1, fault, 2)) break;
-        const bool retained = t < pl.n_rt;
-        const int nrows = retained ? min(TILE, n_ret - t * TILE) : min(TILE, n_apx - (t - pl.n_rt) * TILE);
-        if (kr0 < nrows) {
-            const uint32_t kbase = tma::smem_u32(smem + s * STAGE_BYTES);
-            const uint32_t vbase = retained ? kbase + 2 * BOX_BYTES : kbase;
-            // ---- S = Q K^T for 16 keys: four independent chains (even / odd k-steps x two 8-key tiles)
-            float s0[2], s1[2];
-            {
-                float e0[2] = {0.f, 0.f}, e1[2] = {0.f, 0.f}, o0[2] = {0.f, 0.f}, o1[2] = {0.f, 0.f};
+    // 64 keys at kbase (two swizzled boxes), "values" at vbase (the keys themselves for a key-only tile).
+    auto step64 = [&](uint32_t kbase, uint32_t vbase, int nrows, bool retained, int unit) {
+        // ---- S = Q K^T: eight 8-key column tiles, each its own accumulator chain over the 8 k-steps
+        float sc[8][2], zz[2];
 #pragma unroll
-                for (int ks = 0; ks < 8; ks += 2) {
-                    uint32_t b0, b1, b2, b3, c0, c1, c2, c3;
-                    // k-step ks covers 16-byte chunks 2ks, 2ks+1 of the 256-byte row: box ks/4, chunk (2ks)%8 (+1)
-                    ldsm_x4(kbase + (ks >> 2) * BOX_BYTES + qk_row + ((((2 * ks) & 7) << 4) ^ qk_x), b0, b1, b2, b3);
-                    ldsm_x4(kbase + ((ks + 1) >> 2) * BOX_BYTES + qk_row + ((((2 * ks + 2) & 7) << 4) ^ qk_x), c0, c1, c2, c3);
-                    mma_lo8(e0[0], e0[1], zz[0][0], zz[0][1], qa[ks][0], qa[ks][1], b0, b1);
-                    mma_lo8(e1[0], e1[1], zz[1][0], zz[1][1], qa[ks][0], qa[ks][1], b2, b3);
-                    mma_lo8(o0[0], o0[1], zz[2][0], zz[2][1], qa[ks + 1][0], qa[ks + 1][1], c0, c1);
-                    mma_lo8(o1[0], o1[1], zz[3][0], zz[3][1], qa[ks + 1][0], qa[ks + 1][1], c2, c3);
-                }
-                s0[0] = e0[0] + o0[0]; s0[1] = e0[1] + o0[1];
-                s1[0] = e1[0] + o1[0]; s1[1] = e1[1] + o1[1];
-            }
-            // ---- online softmax over these 16 keys (row = head gid, shared by the 4 threads of a quad)
-            const int kc = kr0 + 2 * tig;
-            const float t00 = kc < nrows ? s0[0] * scale_log2e : -INFINITY;
-            const float t01 = kc + 1 < nrows ? s0[1] * scale_log2e : -INFINITY;
-            const float t10 = kc + 8 < nrows ? s1[0] * scale_log2e : -INFINITY;
-            const float t11 = kc + 9 < nrows ? s1[1] * scale_log2e : -INFINITY;
-            float mx = fmaxf(fmaxf(t00, t01), fmaxf(t10, t11));
-            mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
-            mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
-            if (!retained && !stashed) {           // first key-only tile of this unit for this warp: park sum p v
-                if (gid < g) store_acc(record_of(u) + 4);
-                zero_acc();
-                stashed = true;
-                stash_scale = 1.f;
-            }
-            const float m_new = fmaxf(m, mx);      // finite: key kr0 is valid for every row
-            const float alpha = exp2f(m - m_new);  // 0 on the first tile
-            const float p00 = exp2f(t00 - m_new), p01 = exp2f(t01 - m_new);
-            const float p10 = exp2f(t10 - m_new), p11 = exp2f(t11 - m_new);
-            l = l * alpha + (p00 + p01) + (p10 + p11);
-            m = m_new;
-            stash_scale *= alpha;
-            if (__any_sync(0xffffffffu, alpha != 1.f)) {
+        for (int n = 0; n < 8; ++n) { sc[n][0] = 0.f; sc[n][1] = 0.f; }
 #pragma unroll
-                for (int n = 0; n < 16; ++n) { acc[n][0] *= alpha; acc[n][1] *= alpha; acc[n][2] *= alpha; acc[n][3] *= alpha; }
+        for (int ks = 0; ks < 8; ++ks) {
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {          // 16 keys per ldmatrix
+                uint32_t b0, b1, b2, b3;
+                // k-step ks covers 16-byte chunks 2ks, 2ks+1 of the 256-byte row: box ks/4, chunk (2ks)%8 (+1)
+                ldsm_x4(kbase + (ks >> 2) * BOX_BYTES + j * 16 * 128 + qk_row + ((((2 * ks) & 7) << 4) ^ qk_x), b0, b1, b2, b3);
+                mma_lo8(sc[2 * j][0], sc[2 * j][1], zz[0], zz[1], qa[ks][0], qa[ks][1], b0, b1);
+                mma_lo8(sc[2 * j + 1][0], sc[2 * j + 1][1], zz[0], zz[1], qa[ks][0], qa[ks][1], b2, b3);
             }
+        }
+        // ---- online softmax over these 64 keys (row = head gid, shared by the 4 threads of a quad)
+        float mx = -INFINITY;
+#pragma unroll
+        for (int n = 0; n < 8; ++n) {
+            const int kc = n * 8 + 2 * tig;
+            sc[n][0] = kc < nrows ? sc[n][0] * scale_log2e : -INFINITY;
+            sc[n][1] = kc + 1 < nrows ? sc[n][1] * scale_log2e : -INFINITY;
+            mx = fmaxf(mx, fmaxf(sc[n][0], sc[n][1]));
+        }
+        mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
+        mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
+        if (!retained && !stashed) {           // first key-only keys of this unit for this warp: park sum p v
+            if (gid < g) store_acc(record_of(unit) + 4);
+            zero_acc();
+            stashed = true;
+            stash_scale = 1.f;
+        }
+        const float m_new = fmaxf(m, mx);      // finite: key 0 of the step is valid for every row
+        const float alpha = exp2f(m - m_new);  // 0 on the first step
+        float ls = 0.f;
+#pragma unroll
+        for (int n = 0; n < 8; ++n) {
+            sc[n][0] = exp2f(sc[n][0] - m_new);
+            sc[n][1] = exp2f(sc[n][1] - m_new);
+            ls += sc[n][0] + sc[n][1];
+        }
+        l = l * alpha + ls;
+        m = m_new;
+        stash_scale *= alpha;
+        if (__any_sync(0xffffffffu, alpha != 1.f)) {
+#pragma unroll
+            for (int n = 0; n < 16; ++n) { acc[n][0] *= alpha; acc[n][1] *= alpha; acc[n][2] *= alpha; acc[n][3] *= alpha; }
+        }
+        // ---- accumulate P x (V rows | K rows): four k-steps of 16 keys x 16 column tiles of 8 dims
+#pragma unroll
+        for (int kk = 0; kk < 4; ++kk) {
             // P as bf16 hi (MMA rows 0-7) + lo (rows 8-15)
+            const float p00 = sc[2 * kk][0], p01 = sc[2 * kk][1], p10 = sc[2 * kk + 1][0], p11 = sc[2 * kk + 1][1];
             const __nv_bfloat16 h00 = __float2bfloat16_rn(p00), h01 = __float2bfloat16_rn(p01);
             const __nv_bfloat16 h10 = __float2bfloat16_rn(p10), h11 = __float2bfloat16_rn(p11);
             const uint32_t a0 = pack_bf16(__bfloat162float(h00), __bfloat162float(h01));
             const uint32_t a2 = pack_bf16(__bfloat162float(h10), __bfloat162float(h11));
             const uint32_t a1 = pack_bf16(p00 - __bfloat162float(h00), p01 - __bfloat162float(h01));
             const uint32_t a3 = pack_bf16(p10 - __bfloat162float(h10), p11 - __bfloat162float(h11));
-            // ---- accumulate P x (V rows | K rows) over the 16 column tiles of 8 dims
 #pragma unroll
             for (int np = 0; np < 8; ++np) {
                 uint32_t b0, b1, b2, b3;
-                ldsm_x4_t(vbase + (np >> 2) * BOX_BYTES + pv_row + ((((2 * np) & 7) << 4) ^ pv_x), b0, b1, b2, b3);
+                ldsm_x4_t(vbase + (np >> 2) * BOX_BYTES + kk * 16 * 128 + pv_row + ((((2 * np) & 7) << 4) ^ pv_x), b0, b1, b2, b3);
                 mma_16(acc[2 * np], a0, a1, a2, a3, b0, b1);
                 mma_16(acc[2 * np + 1], a0, a1, a2, a3, b2, b3);
             }
         }
-        __syncwarp();
-        if (lane == 0) tma::mbar_arrive(&empty_bar[s]);
-        if (++t == pl.n_tiles) {
-            flush(u);
-            t = 0; ++u;
-            if (i + 1 < n_my) load_q(u);
+    };
+
+    zero_acc();
+    // Walk the units the block touches; this warp owns the block's tiles i with i % CONSUMER_WARPS == wq.
+    int i = wq;                                        // index into the block's tile sequence
+    for (int u = u0; u <= u_last; ++u) {
+        const long long unit_end = (long long)(u + 1) * pl.n_tiles - gt_lo;     // first sequence index past the unit
+        bool loaded = false;
+        for (; i < n_my && i < unit_end; i += CONSUMER_WARPS) {
+            if (!loaded) { load_q(u); loaded = true; }
+            const int s = i % SLOTS, round = i / SLOTS;
+            const int t = (int)(gt_lo + i - (long long)u * pl.n_tiles);
+            if (!tma::mbar_wait_warp(&full_bar[s], round & 1, fault, 2)) return;
+            const uint32_t base = tma::smem_u32(smem + s * SLOT_BYTES);
+            if (t < pl.n_rt) {
+                step64(base, base + HALF_BYTES, min(KEYS, n_ret - t * KEYS), true, u);
+            } else {
+                const int r0 = (t - pl.n_rt) * 2 * KEYS;
+                step64(base, base, min(KEYS, n_apx - r0), false, u);
+                if (n_apx - r0 > KEYS) step64(base + HALF_BYTES, base + HALF_BYTES, min(KEYS, n_apx - r0 - KEYS), false, u);
+            }
+            __syncwarp();
+            if (lane == 0) tma::mbar_arrive(&empty_bar[s]);
         }
+        flush(u);
     }
-    if (t != 0) flush(u);            // the range ended inside a unit
 }
 
 // Merge for head_dim 128: grid (U), 128 threads.  Combines the records of a unit, applies the
@@ -311,8 +318,8 @@ decode_merge_bf16_d128(const float* __restrict__ partial, const __nv_bfloat16* _
     __shared__ float fv[8][48], fk[8][48];     // per head, per record: factor for the value part / the key part and l
     __shared__ float Ls[8];
     const int u = blockIdx.x, c = threadIdx.x;
-    const int first = block_of_weight(unit_first_weight(u, pl), pl);
-    const int n_rec = (block_of_weight(unit_last_weight(u, pl), pl) - first + 1) * CONSUMER_WARPS;   // <= 48 (checked on the host)
+    const int first = block_of_tile((long long)u * pl.n_tiles, pl);
+    const int n_rec = (block_of_tile((long long)(u + 1) * pl.n_tiles - 1, pl) - first + 1) * CONSUMER_WARPS;   // <= 48 (checked on the host)
     const float* base = partial + (size_t)u * pl.s_max * CONSUMER_WARPS * g * REC;
     // W tile into shared memory while the record headers are fetched
     const uint32_t* Wu = reinterpret_cast<const uint32_t*>(W + (size_t)(u % LH) * 128 * 128);

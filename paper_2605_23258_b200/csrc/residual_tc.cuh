@@ -188,7 +188,7 @@ residual_tc(const __nv_bfloat16* __restrict__ K, const __nv_bfloat16* __restrict
         const uint32_t lane_addr = sy.tmem_base + ((uint32_t)(quarter * 32) << 16);
         for (int i = 0; i < n_my; ++i) {
             const int s = i % STAGES, round = i / STAGES;
-            if (!tma::mbar_wait(&sy.done[s], round & 1, fault, 45)) break;
+            if (!tma::mbar_wait_warp(&sy.done[s], round & 1, fault, 45)) break;
             tc::fence_after_sync();
             const long long gt = gt_lo + i;
             const int u = (int)(gt / P.tpu), t = (int)(gt - (long long)u * P.tpu);

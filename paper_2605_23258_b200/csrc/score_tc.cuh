@@ -387,7 +387,7 @@ score_pass1_tc(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
             for (int t = im.t0; t < im.t1; ++t, ++tcount) {
                 if ((int)(tcount & 1) != grp) continue;
                 const uint32_t buf = (tcount & 1) * 2 + wg, use = tcount >> 1;
-                if (!tma::mbar_wait(&sy.acc_full[buf], use & 1, fault, 31)) { ok = false; break; }
+                if (!tma::mbar_wait_warp(&sy.acc_full[buf], use & 1, fault, 31)) { ok = false; break; }
                 fence_after_sync();
                 if (wg_active) {
                     const uint32_t taddr = lane_addr + buf * 128;
@@ -463,7 +463,7 @@ score_pass2_tc(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
             for (int t = im.t0; t < im.t1; ++t, ++tcount) {
                 if ((int)(tcount & 1) != grp) continue;
                 const uint32_t buf = tcount & 1, use = tcount >> 1;
-                if (!tma::mbar_wait(&sy.acc_full[buf], use & 1, fault, 32)) { ok = false; break; }
+                if (!tma::mbar_wait_warp(&sy.acc_full[buf], use & 1, fault, 32)) { ok = false; break; }
                 fence_after_sync();
                 const long long key = (long long)t * KT + key_in_tile;
                 float colsum = 0.f;

@@ -44,6 +44,15 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, int* f
     return false;
 }
 
+// The same wait for a whole warp: every lane polls, and the warp leaves the wait converged (the
+// warp-wide .aligned instructions that follow such a wait -- ldmatrix, mma, tcgen05.ld -- require
+// it).  All lanes get the same answer.
+__device__ __forceinline__ bool mbar_wait_warp(uint64_t* bar, uint32_t parity, int* fault, int code) {
+    const bool ok = mbar_wait(bar, parity, fault, code);
+    __syncwarp();
+    return __all_sync(0xffffffffu, ok);
+}
+
 // One box of a rank-3 tensor into shared memory; completion is signalled on `bar` by byte count.
 __device__ __forceinline__ void load_3d(void* dst, const CUtensorMap* map, int x, int y, int z, uint64_t* bar) {
     asm volatile(
