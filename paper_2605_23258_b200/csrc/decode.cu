@@ -223,11 +223,23 @@ static vector_status launch_decode_bf16_d128(const Dims& dm, const void* q, cons
     dbf::decode_stream_bf16_d128<<<pl.B, dbf::THREADS, dbf::SMEM_BYTES, st>>>(
         (const T*)q, maps, pl, (int)ch->n_ret, (int)ch->n_apx, dm.g, dm.scale * 1.4426950408889634f, partial, fault);
     VEC_LAUNCH_CHECK();
+    // programmatic dependent launch: the merge blocks start while the streaming kernel drains
+    cudaLaunchAttribute attr;
+    attr.id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr.val.programmaticStreamSerializationAllowed = 1;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(dm.U);
+    cfg.blockDim = dim3(128);
+    cfg.dynamicSmemBytes = 0;
+    cfg.stream = st;
+    cfg.attrs = &attr;
+    cfg.numAttrs = 1;
+    const float* rec = partial;
+    const T* Wp = (const T*)W;
     if (out_dtype == VECTOR_F32)
-        dbf::decode_merge_bf16_d128<float><<<dm.U, 128, 0, st>>>(partial, (const T*)W, dm.LH, dm.g, pl, (float*)out);
+        VEC_CUDA_CHECK(cudaLaunchKernelEx(&cfg, dbf::decode_merge_bf16_d128<float>, rec, Wp, dm.LH, dm.g, pl, (float*)out));
     else
-        dbf::decode_merge_bf16_d128<T><<<dm.U, 128, 0, st>>>(partial, (const T*)W, dm.LH, dm.g, pl, (T*)out);
-    VEC_LAUNCH_CHECK();
+        VEC_CUDA_CHECK(cudaLaunchKernelEx(&cfg, dbf::decode_merge_bf16_d128<T>, rec, Wp, dm.LH, dm.g, pl, (T*)out));
     return VECTOR_OK;
 }
 

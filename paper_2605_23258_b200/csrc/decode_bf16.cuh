@@ -120,6 +120,10 @@ decode_stream_bf16_d128(const __nv_bfloat16* __restrict__ q, const __grid_consta
     const int u0 = (int)(gt_lo / pl.n_tiles), t0 = (int)(gt_lo - (long long)u0 * pl.n_tiles);
     const int u_last = (int)((gt_hi - 1) / pl.n_tiles);
 
+    // The merge kernel is launched as a programmatic dependent of this one: its blocks may be
+    // scheduled (and fetch W) as soon as SMs free up; it reads the records only after its own
+    // griddepcontrol.wait, which returns once this whole grid has finished and flushed.
+    asm volatile("griddepcontrol.launch_dependents;\n" ::: "memory");
     if (tid == 0) {
 #pragma unroll
         for (int s = 0; s < SLOTS; ++s) { tma::mbar_init(&full_bar[s], 1); tma::mbar_init(&empty_bar[s], 1); }
@@ -321,13 +325,15 @@ decode_merge_bf16_d128(const float* __restrict__ partial, const __nv_bfloat16* _
     const int first = block_of_tile((long long)u * pl.n_tiles, pl);
     const int n_rec = (block_of_tile((long long)(u + 1) * pl.n_tiles - 1, pl) - first + 1) * CONSUMER_WARPS;   // <= 48 (checked on the host)
     const float* base = partial + (size_t)u * pl.s_max * CONSUMER_WARPS * g * REC;
-    // W tile into shared memory while the record headers are fetched
+    // W tile into shared memory (overlaps the tail of the streaming kernel)
     const uint32_t* Wu = reinterpret_cast<const uint32_t*>(W + (size_t)(u % LH) * 128 * 128);
 #pragma unroll 16
     for (int k = 0; k < 64; ++k) {
         int i = c + 128 * k;
         Ws[(i >> 6) * 65 + (i & 63)] = Wu[i];
     }
+    // everything above reads only W, which the streaming kernel does not write; its records from here on
+    asm volatile("griddepcontrol.wait;\n" ::: "memory");
     if (c < 8 * 16) {
         // thread (a = c / 16, lane16 = c % 16): headers of head a, records lane16, lane16+16, lane16+32
         const int a = c >> 4, j0 = c & 15;
