@@ -229,7 +229,7 @@ static vector_status launch_decode_bf16_d128(const Dims& dm, const void* q, cons
     attr.val.programmaticStreamSerializationAllowed = 1;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(dm.U);
-    cfg.blockDim = dim3(128);
+    cfg.blockDim = dim3(128 * dm.g);
     cfg.dynamicSmemBytes = 0;
     cfg.stream = st;
     cfg.attrs = &attr;

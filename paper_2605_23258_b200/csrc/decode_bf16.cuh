@@ -311,95 +311,86 @@ decode_stream_bf16_d128(const __nv_bfloat16* __restrict__ q, const __grid_consta
     }
 }
 
-// Merge for head_dim 128: grid (U), 128 threads.  Combines the records of a unit, applies the
-// unit's map to the p-weighted key sum and normalises: o = (sum f s acc_v + W sum f acc_k) / sum f l.
+// Merge for head_dim 128: grid (U), 128 g threads -- thread (a, c) owns output dim c of head a.
+// Combines the records of a unit, applies the unit's map to the p-weighted key sum and normalises:
+//   o = (sum_j f_j s_j acc_v_j + W sum_j f_j acc_k_j) / sum_j f_j l_j,   f_j = exp(m_j - max m).
+// Every load of a phase is independent of the others, so a phase costs one memory latency.
 template <typename TO>
-__global__ void __launch_bounds__(128)
+__global__ void __launch_bounds__(1024)
 decode_merge_bf16_d128(const float* __restrict__ partial, const __nv_bfloat16* __restrict__ W, int LH, int g,
                        Plan pl, TO* __restrict__ out) {
     __shared__ uint32_t Ws[128 * 65];          // W rows as bf16 pairs, row stride 65 words (conflict-free)
-    __shared__ float aks[8][128];
-    __shared__ float fv[8][48], fk[8][48];     // per head, per record: factor for the value part / the key part and l
+    __shared__ __align__(8) float aks[8][128];
+    __shared__ float fv[8][48], fk[8][48];     // per head, per record: factor for the value part / the key part
     __shared__ float Ls[8];
-    const int u = blockIdx.x, c = threadIdx.x;
-    const int first = block_of_tile((long long)u * pl.n_tiles, pl);
-    const int n_rec = (block_of_tile((long long)(u + 1) * pl.n_tiles - 1, pl) - first + 1) * CONSUMER_WARPS;   // <= 48 (checked on the host)
-    const float* base = partial + (size_t)u * pl.s_max * CONSUMER_WARPS * g * REC;
-    // W tile into shared memory (overlaps the tail of the streaming kernel)
-    const uint32_t* Wu = reinterpret_cast<const uint32_t*>(W + (size_t)(u % LH) * 128 * 128);
-#pragma unroll 16
-    for (int k = 0; k < 64; ++k) {
-        int i = c + 128 * k;
-        Ws[(i >> 6) * 65 + (i & 63)] = Wu[i];
+    const int u = blockIdx.x, tid = threadIdx.x, a = tid >> 7, c = tid & 127, lane = tid & 31;
+    const int nthr = blockDim.x;
+    // W tile into shared memory (overlaps the tail of the streaming kernel): 2048 16-byte pieces
+    const uint4* Wu = reinterpret_cast<const uint4*>(W + (size_t)(u % LH) * 128 * 128);
+    for (int i = tid; i < 2048; i += nthr) {
+        const uint4 v = Wu[i];
+        uint32_t* dst = Ws + (i >> 4) * 65 + (i & 15) * 4;      // 16 pieces per 256-byte row
+        dst[0] = v.x; dst[1] = v.y; dst[2] = v.z; dst[3] = v.w;
     }
     // everything above reads only W, which the streaming kernel does not write; its records from here on
     asm volatile("griddepcontrol.wait;\n" ::: "memory");
-    if (c < 8 * 16) {
-        // thread (a = c / 16, lane16 = c % 16): headers of head a, records lane16, lane16+16, lane16+32
-        const int a = c >> 4, j0 = c & 15;
-        float mj[3], lj[3], sj[3];
-        float M = -INFINITY;
+    const int first = block_of_tile((long long)u * pl.n_tiles, pl);
+    const int n_rec = (block_of_tile((long long)(u + 1) * pl.n_tiles - 1, pl) - first + 1) * CONSUMER_WARPS;   // <= 36
+    const float* base = partial + (size_t)u * pl.s_max * CONSUMER_WARPS * g * REC;
+    if (c < 32) {
+        // first warp of head a: headers of records lane and lane + 32
+        float mj[2], lj[2], sj[2];
 #pragma unroll
-        for (int k = 0; k < 3; ++k) {
-            int j = j0 + 16 * k;
+        for (int k = 0; k < 2; ++k) {
+            const int j = lane + 32 * k;
             mj[k] = -INFINITY; lj[k] = 0.f; sj[k] = 0.f;
-            if (a < g && j < n_rec) {
-                float4 h = *reinterpret_cast<const float4*>(base + ((size_t)j * g + a) * REC);
+            if (j < n_rec) {
+                const float4 h = *reinterpret_cast<const float4*>(base + ((size_t)j * g + a) * REC);
                 mj[k] = h.x; lj[k] = h.y; sj[k] = h.z;
             }
-            M = fmaxf(M, mj[k]);
         }
-#pragma unroll
-        for (int o = 8; o > 0; o >>= 1) M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, o));
+        const float M = warp_max(fmaxf(mj[0], mj[1]));
         float Lsum = 0.f;
 #pragma unroll
-        for (int k = 0; k < 3; ++k) {
-            int j = j0 + 16 * k;
-            float f = mj[k] > -INFINITY ? __expf(mj[k] - M) : 0.f;
+        for (int k = 0; k < 2; ++k) {
+            const int j = lane + 32 * k;
+            const float f = mj[k] > -INFINITY ? __expf(mj[k] - M) : 0.f;
             if (j < 48) { fk[a][j] = f; fv[a][j] = f * sj[k]; }
             Lsum += f * lj[k];
         }
-#pragma unroll
-        for (int o = 8; o > 0; o >>= 1) Lsum += __shfl_xor_sync(0xffffffffu, Lsum, o);
-        if (j0 == 0) Ls[a] = Lsum;
+        Lsum = warp_sum(Lsum);
+        if (lane == 0) Ls[a] = Lsum;
     }
     __syncthreads();
-    float accv[8];
+    float av = 0.f, ak = 0.f;
+    for (int j0 = 0; j0 < n_rec; j0 += 6) {
+        float rv[6], rk[6];
 #pragma unroll
-    for (int a = 0; a < 8; ++a) {
-        accv[a] = 0.f;
-        if (a < g) {
-            float av = 0.f, ak = 0.f;
-#pragma unroll 4
-            for (int j = 0; j < n_rec; ++j) {
-                const float* r = base + ((size_t)j * g + a) * REC + 4;
-                av = fmaf(fv[a][j], r[c], av);
-                ak = fmaf(fk[a][j], r[128 + c], ak);
+        for (int k = 0; k < 6; ++k) {
+            const int j = min(j0 + k, n_rec - 1);
+            const float* r = base + ((size_t)j * g + a) * REC + 4;
+            rv[k] = r[c];
+            rk[k] = r[128 + c];
+        }
+#pragma unroll
+        for (int k = 0; k < 6; ++k) {
+            if (j0 + k < n_rec) {
+                av = fmaf(fv[a][j0 + k], rv[k], av);
+                ak = fmaf(fk[a][j0 + k], rk[k], ak);
             }
-            accv[a] = av;
-            aks[a][c] = ak;
         }
     }
+    aks[a][c] = ak;
     __syncthreads();
-    float proj[8];
-#pragma unroll
-    for (int a = 0; a < 8; ++a) proj[a] = 0.f;
-#pragma unroll 4
+    float p0 = 0.f, p1 = 0.f;
+#pragma unroll 8
     for (int c2 = 0; c2 < 64; ++c2) {
         const uint32_t w2 = Ws[c * 65 + c2];
-        const float w_lo = __uint_as_float(w2 << 16), w_hi = __uint_as_float(w2 & 0xffff0000u);
-#pragma unroll
-        for (int a = 0; a < 8; ++a) {
-            if (a < g) {
-                const float2 k2 = *reinterpret_cast<const float2*>(&aks[a][2 * c2]);
-                proj[a] = fmaf(w_lo, k2.x, proj[a]);
-                proj[a] = fmaf(w_hi, k2.y, proj[a]);
-            }
-        }
+        const float2 k2 = *reinterpret_cast<const float2*>(&aks[a][2 * c2]);
+        p0 = fmaf(__uint_as_float(w2 << 16), k2.x, p0);
+        p1 = fmaf(__uint_as_float(w2 & 0xffff0000u), k2.y, p1);
     }
-#pragma unroll
-    for (int a = 0; a < 8; ++a)
-        if (a < g) store_out(out + ((size_t)u * g + a) * 128 + c, (accv[a] + proj[a]) / Ls[a]);
+    store_out(out + ((size_t)u * g + a) * 128 + c, (av + p0 + p1) / Ls[a]);
 }
 
 }  // namespace dbf

@@ -276,6 +276,30 @@ def test_decode_degenerate_pools(oracle):
             assert np.max(np.abs(out[u].cpu().double().numpy() - o)) <= 2e-2, (n_ret, n_apx, u)
 
 
+def test_decode_long_block_ranges(oracle):
+    """Few units with long pools: every block's tile range wraps its shared-memory ring several times and
+    crosses a unit boundary; g = 4 and g = 8; a pool end that leaves a key-only tile half empty."""
+    for base, over, n_ret, n_apx in [(1, {"N": 8192, "n_kv_heads": 2, "n_q_heads": 8}, 3000, 6000 + 37),
+                                     (4, {"N": 8192, "n_layers": 1, "n_kv_heads": 1, "n_q_heads": 8}, 4100, 4090)]:
+        wl = synth.shrink(synth.WORKLOADS[base], n_calib=1024, **over)
+        K, V, _ = synth.context(wl, DEV)
+        W = calibrated_maps(wl).to(DEV)
+        sh = shape_of(wl)
+        _, sq, _ = synth.all_head_params(wl, DEV)
+        q = synth.decode_q(wl, 0, DEV, sq)
+        ws = vec.alloc_workspace(sh, budget_of(wl, 50))
+        out = torch.empty(wl.units, wl.group, wl.head_dim, dtype=torch.float32, device=DEV)
+        ipos = torch.arange(wl.N, dtype=torch.int32, device=DEV).repeat(wl.units, 1).contiguous()
+        cache = vec.Cache(K.clone(), V.clone(), K.flip(1).contiguous(), ipos, ipos.clone(), n_ret, n_apx)
+        vec.vector_decode_attn(sh, q, cache, W, out, 0, ws)
+        torch.cuda.synchronize()
+        assert vec.vector_device_fault() == 0
+        for u in range(wl.units):
+            _, o = oracle.attend(q[u].cpu(), cache.ret_k[u, :n_ret].cpu(), cache.ret_v[u, :n_ret].cpu(),
+                                 cache.apx_k[u, :n_apx].cpu(), W[u].cpu(), 1.0 / np.sqrt(wl.head_dim))
+            assert np.max(np.abs(out[u].cpu().double().numpy() - o)) <= 2e-2, (base, u)
+
+
 def test_full_size_bench_configuration_sampled_units(oracle):
     """Config 2 at full size in the launch shape the benchmark times; the oracle checks sampled units."""
     wl = synth.WORKLOADS[2]
