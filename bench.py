@@ -288,6 +288,7 @@ def main():
     t_end.record()
     barrier()
     clocks = sampler.stop()
+    clocks_hint_mhz = clocks["sm_mhz"] or 1965.0
     total_ms = t_begin.elapsed_time(t_end)
     phase = {"score": [], "route": [], "compact": [], "decode": []}
     for m in all_marks:
@@ -323,9 +324,22 @@ def main():
         {"kernel": "vector_decode_attn (split + merge)", "bound": "hbm",
          "achieved": decode_bytes / (ms["decode"] * 1e-3) / 1e9, "peak": hbm, "unit": "GB/s", "ms": ms["decode"]},
     ]
+    # DRAM bytes per call from the ncu capture summarised under profiles/ (64 units of this workload,
+    # scaled by the unit count: traffic of these kernels grows in proportion to it); None for other
+    # workloads and for kernels changed since the capture.
+    ncu_traffic_per_unit = {"vector_score (logit passes)": (541.4e6 + 5.3e6 + 541.5e6 + 17.1e6) / 64,
+                            "vector_compact": (217.3e6 + 172.7e6) / 64,
+                            "vector_decode_attn (split + merge)": (214.9e6 + 4.6e6 + 4.7e6) / 64}
+    exps = 2.0 * g * w * N * U                                  # one exp2 per logit and pass
+    xu_peak = 16.0 * 148 * (clocks_hint_mhz * 1e6)              # MUFU results per second at the sampled SM clock
     for k in kernels:
         k["frac"] = k["achieved"] / k["peak"]
         k["traffic"] = None
+        if args.config == 2 and args.budget is None and k["kernel"] in ncu_traffic_per_unit:
+            per_call = ncu_traffic_per_unit[k["kernel"]] * U
+            k["traffic"] = per_call * (D if k["kernel"].startswith("vector_decode") else 1)
+    kernels[0]["xu_exp_per_s"] = exps / (ms["score"] * 1e-3)
+    kernels[0]["xu_frac_of_16_per_clk_per_sm"] = kernels[0]["xu_exp_per_s"] / xu_peak
     dominant = max(kernels, key=lambda k: k["ms"])
     roofline = {k: dominant[k] for k in ("bound", "achieved", "peak", "unit", "frac", "traffic")}
     roofline["kernel"] = dominant["kernel"]
