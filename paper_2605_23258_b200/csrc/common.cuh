@@ -32,5 +32,20 @@ __device__ __forceinline__ float warp_max(float v) {
     return v;
 }
 
+
+// Rotary angle of channel pair c at position pos: pos * theta^(-2c/d).  The product is formed and
+// reduced to [-pi, pi] in fp64 (positions reach 1e5 rad, where fp32 would be off by 1e-2), the sine
+// and cosine of the remainder are taken in fp32.
+__device__ __forceinline__ void rope_cos_sin(double pos, double inv_freq, float& cs, float& sn) {
+    const double ang = pos * inv_freq;
+    const double n = rint(ang * 0.15915494309189535);
+    const double r = fma(-n, 6.283185307179586, ang);
+    sincosf((float)r, &sn, &cs);
+}
+// Inverse frequencies theta^(-2c/d), c < d/2, into shared memory (fp64); callers synchronise.
+__device__ __forceinline__ void rope_fill_inv_freq(double* inv_freq, int d, float theta) {
+    for (int c = threadIdx.x; c < d / 2; c += blockDim.x) inv_freq[c] = pow((double)theta, -2.0 * (double)c / (double)d);
+}
+
 }  // namespace vec
 #endif

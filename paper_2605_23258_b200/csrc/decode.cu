@@ -46,14 +46,20 @@ template <> struct RowLoad<__nv_bfloat16, 2> {
 // Partial record per (unit, split, head): [m, l, acc_v[D], acc_k[D]]
 template <int D> struct Rec { static constexpr int floats = 2 + 2 * D; };
 
-template <typename T, int D, int G>
+// With ROPE the approximated value is W applied to the key turned back by its original position
+// (apx_pos): the logit still uses the stored key, only the p-weighted key sum takes the turned one.
+// A lane holds EPL consecutive channels; the partner channel c +- D/2 sits in lane ^ 16.
+template <typename T, int D, int G, bool ROPE>
 __global__ void __launch_bounds__(128)
 decode_split_generic(const T* __restrict__ q, const T* __restrict__ ret_k, const T* __restrict__ ret_v,
-                     const T* __restrict__ apx_k, int64_t cap_ret, int64_t cap_apx, int n_ret, int n_apx,
-                     int g, float scale, float* __restrict__ partial) {
+                     const T* __restrict__ apx_k, const int32_t* __restrict__ apx_pos, int64_t cap_ret,
+                     int64_t cap_apx, int n_ret, int n_apx, int g, float scale, float theta,
+                     float* __restrict__ partial) {
     constexpr int EPL = D / 32;
     constexpr int REC = Rec<D>::floats;
     __shared__ float sm[4][G][REC];
+    __shared__ double inv_freq[D / 2];
+    if (ROPE) { rope_fill_inv_freq(inv_freq, D, theta); __syncthreads(); }
     const int u = blockIdx.y, split = blockIdx.x, n_splits = gridDim.x;
     const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
     const int total = n_ret + n_apx;
@@ -80,6 +86,19 @@ decode_split_generic(const T* __restrict__ q, const T* __restrict__ ret_k, const
         float kx[EPL], vx[EPL];
         RowLoad<T, EPL>::load(kp, lane, kx);
         if (retained) RowLoad<T, EPL>::load(ret_v + ((size_t)u * cap_ret + i) * D, lane, vx);
+        float kt[EPL];                       // what an approximated token contributes: the key, or the key turned back
+#pragma unroll
+        for (int e = 0; e < EPL; ++e) kt[e] = kx[e];
+        if (ROPE && !retained) {
+            const double pos = (double)apx_pos[(size_t)u * cap_apx + (i - n_ret)];
+#pragma unroll
+            for (int e = 0; e < EPL; ++e) {
+                float cs, sn;
+                rope_cos_sin(pos, inv_freq[(lane * EPL + e) % (D / 2)], cs, sn);
+                const float other = __shfl_xor_sync(0xffffffffu, kx[e], 16);
+                kt[e] = lane < 16 ? fmaf(kx[e], cs, other * sn) : fmaf(kx[e], cs, -other * sn);
+            }
+        }
 #pragma unroll
         for (int a = 0; a < G; ++a) {
             if (a < g) {
@@ -97,7 +116,7 @@ decode_split_generic(const T* __restrict__ q, const T* __restrict__ ret_k, const
                     av[a][e] *= corr;
                     ak[a][e] *= corr;
                     if (retained) av[a][e] = fmaf(p, vx[e], av[a][e]);
-                    else          ak[a][e] = fmaf(p, kx[e], ak[a][e]);
+                    else          ak[a][e] = fmaf(p, kt[e], ak[a][e]);
                 }
             }
         }
@@ -166,9 +185,10 @@ static vector_status launch_decode(const Dims& dm, const void* q, const vector_c
                                    int out_dtype, float* partial, cudaStream_t st) {
     const int n_splits = decode_num_splits(dm.U, ch->n_ret + ch->n_apx);
     dim3 grid(n_splits, dm.U);
-    decode_split_generic<T, D, G><<<grid, 128, 0, st>>>((const T*)q, (const T*)ch->ret_k, (const T*)ch->ret_v,
-                                                        (const T*)ch->apx_k, ch->cap_ret, ch->cap_apx,
-                                                        (int)ch->n_ret, (int)ch->n_apx, dm.g, dm.scale, partial);
+    auto kern = dm.rope ? decode_split_generic<T, D, G, true> : decode_split_generic<T, D, G, false>;
+    kern<<<grid, 128, 0, st>>>((const T*)q, (const T*)ch->ret_k, (const T*)ch->ret_v, (const T*)ch->apx_k,
+                               ch->apx_pos, ch->cap_ret, ch->cap_apx, (int)ch->n_ret, (int)ch->n_apx, dm.g,
+                               dm.scale, dm.theta, partial);
     VEC_LAUNCH_CHECK();
     if (out_dtype == VECTOR_F32)
         decode_merge_generic<T, float, D><<<dm.U, D, 0, st>>>(partial, (const T*)W, dm.LH, dm.g, n_splits,
@@ -271,14 +291,17 @@ extern "C" vector_status vector_decode_attn(const vector_shape* shape, const voi
     if (cache->n_ret > 0 && (!cache->ret_k || !cache->ret_v)) return VECTOR_ERR_NULL;
     if (cache->n_apx > 0 && !cache->apx_k) return VECTOR_ERR_NULL;
     if (!ws || ((uintptr_t)ws & 255) || ws_bytes < decode_ws_bytes(dm)) return VECTOR_ERR_WORKSPACE;
-    if (mode == 1 || dm.rope) return VECTOR_ERR_UNSUPPORTED;
+    if (mode == 1) return VECTOR_ERR_UNSUPPORTED;
+    if (dm.rope && cache->n_apx > 0 && !cache->apx_pos) return VECTOR_ERR_NULL;
     cudaStream_t st = (cudaStream_t)stream;
     float* partial = (float*)ws;
     if (dm.dtype == VECTOR_F32)
         return dm.d == 64 ? launch_decode_g<float, 64>(dm, q, cache, W, out, out_dtype, partial, st)
                           : launch_decode_g<float, 128>(dm, q, cache, W, out, out_dtype, partial, st);
-    return dm.d == 64 ? launch_decode_g<__nv_bfloat16, 64>(dm, q, cache, W, out, out_dtype, partial, st)
-                      : launch_decode_bf16_d128(dm, q, cache, W, out, out_dtype, partial, st);
+    if (dm.d == 64) return launch_decode_g<__nv_bfloat16, 64>(dm, q, cache, W, out, out_dtype, partial, st);
+    // the de-rotating variant exists on the CUDA-core path only
+    return dm.rope ? launch_decode_g<__nv_bfloat16, 128>(dm, q, cache, W, out, out_dtype, partial, st)
+                   : launch_decode_bf16_d128(dm, q, cache, W, out, out_dtype, partial, st);
 }
 
 // ---------------------------------------------------------------------------

@@ -161,13 +161,17 @@ truncate_kernel(const float* __restrict__ eps, const int32_t* __restrict__ pool_
 
 // Step 2 on CUDA cores.  grid (ceil(n_idx / 64), U), 256 threads; W^T staged in
 // dynamic shared memory as fp32 (D * (D+1) floats) plus one key row per warp.
-template <typename T, int D>
+// With ROPE the regressor sees the key turned back by its position (the token index): channel c
+// pairs with c + D/2, angle -pos * theta^(-2c/D).
+template <typename T, int D, bool ROPE>
 __global__ void __launch_bounds__(256)
 residual_generic(const T* __restrict__ K, const T* __restrict__ V, const T* __restrict__ W, int64_t N,
-                 int LH, const int32_t* __restrict__ idx, int n_idx, float* __restrict__ eps) {
+                 int LH, const int32_t* __restrict__ idx, int n_idx, float theta, float* __restrict__ eps) {
     extern __shared__ float smem[];
+    __shared__ double inv_freq[D / 2];
     float* Wt = smem;                       // Wt[c_in * (D+1) + c_out]
     float* ks = smem + D * (D + 1);         // [8][D]
+    if (ROPE) rope_fill_inv_freq(inv_freq, D, theta);
     const int u = blockIdx.y, lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
     const T* Wu = W + (size_t)(u % LH) * D * D;
     for (int e = threadIdx.x; e < D * D; e += 256) {
@@ -186,6 +190,17 @@ residual_generic(const T* __restrict__ K, const T* __restrict__ V, const T* __re
 #pragma unroll
         for (int c = lane; c < D; c += 32) kw[c] = to_f32(kr[c]);
         __syncwarp();
+        if (ROPE) {
+#pragma unroll
+            for (int c = lane; c < D / 2; c += 32) {
+                float cs, sn;
+                rope_cos_sin((double)tok, inv_freq[c], cs, sn);
+                const float x = kw[c], y = kw[c + D / 2];
+                kw[c] = fmaf(x, cs, y * sn);
+                kw[c + D / 2] = fmaf(y, cs, -x * sn);
+            }
+            __syncwarp();
+        }
         float e = 0.f;
 #pragma unroll
         for (int m = 0; m < D / 32; ++m) {
@@ -206,10 +221,10 @@ static vector_status launch_residual(const Dims& dm, const void* K, const void* 
                                      const int32_t* idx, int64_t n_idx, float* eps, cudaStream_t st) {
     if (n_idx == 0) return VECTOR_OK;
     size_t smem = (size_t)(D * (D + 1) + 8 * D) * sizeof(float);
-    auto kern = residual_generic<T, D>;
+    auto kern = dm.rope ? residual_generic<T, D, true> : residual_generic<T, D, false>;
     VEC_CUDA_CHECK(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     dim3 grid((unsigned)((n_idx + 63) / 64), dm.U);
-    kern<<<grid, 256, smem, st>>>((const T*)K, (const T*)V, (const T*)W, N, dm.LH, idx, (int)n_idx, eps);
+    kern<<<grid, 256, smem, st>>>((const T*)K, (const T*)V, (const T*)W, N, dm.LH, idx, (int)n_idx, dm.theta, eps);
     VEC_LAUNCH_CHECK();
     return VECTOR_OK;
 }
@@ -240,8 +255,8 @@ static vector_status launch_residual_tc(const Dims& dm, const void* K, const voi
 
 static vector_status residual_dispatch(const Dims& dm, const void* K, const void* V, const void* W, int64_t N,
                                        const int32_t* idx, int64_t n_idx, float* eps, cudaStream_t st) {
-    if (dm.rope) return VECTOR_ERR_UNSUPPORTED;
-    if (dm.dtype == VECTOR_BF16 && dm.d == 128) return launch_residual_tc(dm, K, V, W, N, idx, n_idx, eps, st);
+    // the de-rotating variant exists on the CUDA-core path only
+    if (!dm.rope && dm.dtype == VECTOR_BF16 && dm.d == 128) return launch_residual_tc(dm, K, V, W, N, idx, n_idx, eps, st);
     if (dm.dtype == VECTOR_F32)
         return dm.d == 64 ? launch_residual<float, 64>(dm, K, V, W, N, idx, n_idx, eps, st)
                           : launch_residual<float, 128>(dm, K, V, W, N, idx, n_idx, eps, st);

@@ -218,3 +218,18 @@ def decode_kv(wl: Workload, step: int, device, sigma_k_all, w_true_all, units=No
         fac = lo + (hi - lo) * layer / max(wl.n_layers - 1, 1)
     v = torch.einsum("uce,ue->uc", w_true_all[lh], k) + 0.5 * fac[:, None] * zv
     return k.to(wl.torch_dtype), v.to(wl.torch_dtype)
+
+
+def rope_keys(K: torch.Tensor, theta: float = 10000.0, first_pos: int = 0) -> torch.Tensor:
+    """Stored (post-RoPE) keys from pre-rotation keys K [..., n, d]: row i is turned by its position
+    first_pos + i, half-split pairing (channel c with c + d/2, angle pos * theta^(-2c/d)).  Input
+    shaping only: this is the model's positional encoding, applied in fp64 and rounded once."""
+    d = K.shape[-1]
+    h = d // 2
+    pos = torch.arange(first_pos, first_pos + K.shape[-2], device=K.device, dtype=torch.float64)
+    inv = torch.pow(torch.tensor(theta, dtype=torch.float64, device=K.device),
+                    -2.0 * torch.arange(h, device=K.device, dtype=torch.float64) / d)
+    ang = pos[:, None] * inv[None, :]
+    cs, sn = torch.cos(ang), torch.sin(ang)
+    x, y = K[..., :h].double(), K[..., h:].double()
+    return torch.cat([x * cs - y * sn, x * sn + y * cs], dim=-1).to(K.dtype)
