@@ -345,6 +345,22 @@ def main():
     roofline["kernel"] = dominant["kernel"]
     roofline["peak_source"] = f"{peaks['source']} ({'copy GB/s' if dominant['bound'] == 'hbm' else 'sustained bf16 TFLOP/s'})"
 
+    # ---- the alternative form of the reconstruction (mode 1: W k formed per tile), outside the timed step
+    per_tile = None
+    if wl.dtype == "bf16" and d == 128:
+        comp.cache.n_ret = budget.n_ret
+        for _ in range(3):
+            comp.decode(qs[0], Wm, out, mode=1)
+        a, b_ = ev(), ev()
+        torch.cuda.synchronize(); a.record()
+        for i in range(10):
+            comp.decode(qs[i % n_q], Wm, out, mode=1)
+        b_.record(); torch.cuda.synchronize()
+        us = a.elapsed_time(b_) * 1e3 / 10
+        step_bytes = U * (2 * n_ret + n_apx) * d * es
+        per_tile = {"us_per_step": us, "gbs": step_bytes / us / 1e3,
+                    "extra_flop_per_step": 2.0 * U * n_apx * d * d}
+
     # ---- end to end through host buffers (rank 0 semantics on every rank; reported from rank 0)
     e2e = None
     if not args.no_e2e:
@@ -426,7 +442,7 @@ def main():
         "decode": {"gbs": decode_bytes / (dec_ms_max * 1e-3) / 1e9, "frac_of_measured_copy": decode_bytes / (dec_ms_max * 1e-3) / 1e9 / hbm,
                    "frac_of_8tbs": decode_bytes / (dec_ms_max * 1e-3) / 1e9 / 8000.0, "us_per_step": dec_ms_max * 1e3 / D,
                    "tokens_per_s": world * wl.batch * D / (dec_ms_max * 1e-3), "bytes_per_step": decode_bytes / D},
-        "roofline": roofline, "roofline_kernels": kernels, "cpu_baseline": cpu, "e2e": e2e,
+        "decode_per_tile": per_tile, "roofline": roofline, "roofline_kernels": kernels, "cpu_baseline": cpu, "e2e": e2e,
         "gpu_launches": kernels_per_step * K_steps, "clocks": clocks,
     }
     print(json.dumps(line))

@@ -213,12 +213,14 @@ int* kernel_fault_address() {
 
 // bf16, head_dim 128: persistent TMA + tensor-core streaming kernel and the record merge.
 static vector_status launch_decode_bf16_d128(const Dims& dm, const void* q, const vector_cache* ch, const void* W,
-                                             void* out, int out_dtype, float* partial, cudaStream_t st) {
+                                             void* out, int out_dtype, int mode, float* partial, cudaStream_t st) {
     using T = __nv_bfloat16;
     static bool configured = false;
     if (!configured) {
-        VEC_CUDA_CHECK(cudaFuncSetAttribute(dbf::decode_stream_bf16_d128,
+        VEC_CUDA_CHECK(cudaFuncSetAttribute(dbf::decode_stream_bf16_d128<false>,
                                             cudaFuncAttributeMaxDynamicSharedMemorySize, dbf::SMEM_BYTES));
+        VEC_CUDA_CHECK(cudaFuncSetAttribute(dbf::decode_stream_bf16_d128<true>,
+                                            cudaFuncAttributeMaxDynamicSharedMemorySize, dbf::SMEM_BYTES_PER_TILE));
         configured = true;
     }
     int* fault = kernel_fault_address();
@@ -237,11 +239,17 @@ static vector_status launch_decode_bf16_d128(const Dims& dm, const void* q, cons
     if (ch->n_apx > 0)
         ok = ok && tma::encode_bf16_3d(&maps.apx_k, ch->apx_k, 128, (uint64_t)ch->n_apx, (uint64_t)dm.U, row_b,
                                        (uint64_t)ch->cap_apx * row_b, 64, 64);
+    ok = ok && tma::encode_bf16_3d(&maps.w, W, 128, 128, (uint64_t)dm.LH, row_b, 128 * row_b, 64, 128);
     if (!ok) return VECTOR_ERR_CUDA;
     if (ch->n_ret == 0) { maps.ret_k = maps.apx_k; maps.ret_v = maps.apx_k; }   // never dereferenced: no such tiles
     if (ch->n_apx == 0) maps.apx_k = maps.ret_k;
-    dbf::decode_stream_bf16_d128<<<pl.B, dbf::THREADS, dbf::SMEM_BYTES, st>>>(
-        (const T*)q, maps, pl, (int)ch->n_ret, (int)ch->n_apx, dm.g, dm.scale * 1.4426950408889634f, partial, fault);
+    const float c2 = dm.scale * 1.4426950408889634f;
+    if (mode == 1)
+        dbf::decode_stream_bf16_d128<true><<<pl.B, dbf::THREADS, dbf::SMEM_BYTES_PER_TILE, st>>>(
+            (const T*)q, maps, pl, (int)ch->n_ret, (int)ch->n_apx, dm.g, dm.LH, c2, partial, fault);
+    else
+        dbf::decode_stream_bf16_d128<false><<<pl.B, dbf::THREADS, dbf::SMEM_BYTES, st>>>(
+            (const T*)q, maps, pl, (int)ch->n_ret, (int)ch->n_apx, dm.g, dm.LH, c2, partial, fault);
     VEC_LAUNCH_CHECK();
     // programmatic dependent launch: the merge blocks start while the streaming kernel drains
     cudaLaunchAttribute attr;
@@ -255,11 +263,12 @@ static vector_status launch_decode_bf16_d128(const Dims& dm, const void* q, cons
     cfg.attrs = &attr;
     cfg.numAttrs = 1;
     const float* rec = partial;
+    const int apply_w = mode == 1 ? 0 : 1;
     const T* Wp = (const T*)W;
     if (out_dtype == VECTOR_F32)
-        VEC_CUDA_CHECK(cudaLaunchKernelEx(&cfg, dbf::decode_merge_bf16_d128<float>, rec, Wp, dm.LH, dm.g, pl, (float*)out));
+        VEC_CUDA_CHECK(cudaLaunchKernelEx(&cfg, dbf::decode_merge_bf16_d128<float>, rec, Wp, dm.LH, dm.g, pl, apply_w, (float*)out));
     else
-        VEC_CUDA_CHECK(cudaLaunchKernelEx(&cfg, dbf::decode_merge_bf16_d128<T>, rec, Wp, dm.LH, dm.g, pl, (T*)out));
+        VEC_CUDA_CHECK(cudaLaunchKernelEx(&cfg, dbf::decode_merge_bf16_d128<T>, rec, Wp, dm.LH, dm.g, pl, apply_w, (T*)out));
     return VECTOR_OK;
 }
 
@@ -291,7 +300,8 @@ extern "C" vector_status vector_decode_attn(const vector_shape* shape, const voi
     if (cache->n_ret > 0 && (!cache->ret_k || !cache->ret_v)) return VECTOR_ERR_NULL;
     if (cache->n_apx > 0 && !cache->apx_k) return VECTOR_ERR_NULL;
     if (!ws || ((uintptr_t)ws & 255) || ws_bytes < decode_ws_bytes(dm)) return VECTOR_ERR_WORKSPACE;
-    if (mode == 1) return VECTOR_ERR_UNSUPPORTED;
+    // per-tile reconstruction exists for bf16 with head_dim 128 and stored (not rotated-back) keys
+    if (mode == 1 && (dm.rope || dm.dtype != VECTOR_BF16 || dm.d != 128)) return VECTOR_ERR_UNSUPPORTED;
     if (dm.rope && cache->n_apx > 0 && !cache->apx_pos) return VECTOR_ERR_NULL;
     cudaStream_t st = (cudaStream_t)stream;
     float* partial = (float*)ws;
@@ -301,7 +311,7 @@ extern "C" vector_status vector_decode_attn(const vector_shape* shape, const voi
     if (dm.d == 64) return launch_decode_g<__nv_bfloat16, 64>(dm, q, cache, W, out, out_dtype, partial, st);
     // the de-rotating variant exists on the CUDA-core path only
     return dm.rope ? launch_decode_g<__nv_bfloat16, 128>(dm, q, cache, W, out, out_dtype, partial, st)
-                   : launch_decode_bf16_d128(dm, q, cache, W, out, out_dtype, partial, st);
+                   : launch_decode_bf16_d128(dm, q, cache, W, out, out_dtype, mode, partial, st);
 }
 
 // ---------------------------------------------------------------------------

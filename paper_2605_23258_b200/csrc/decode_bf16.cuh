@@ -19,6 +19,10 @@
 //   O += P V  (retained tile)  or  A += P K  (key-only tile: the p-weighted key
 //             sum that the merge step multiplies by W); P enters as bf16 hi in
 //             MMA rows 0-7 and bf16 lo in rows 8-15, one MMA for both parts
+// Per-tile reconstruction (PER_TILE, the alternative form o = sum_R p v + sum_A p (W k)): for a
+// key-only step the warp first forms V^T = W K^T for its 64 keys on the tensor cores (W of the unit in
+// shared memory, 512 MMAs), then accumulates O^T += V^T P^T with V^T and P split into bf16 hi + lo; the
+// merge step then adds that part without applying W.
 // A warp keeps one running state (m, l, O or A) per unit and writes it as its
 // partial record when it leaves the unit; a warp that met no tile of a unit the
 // block touches writes an empty record.  The merge kernel combines a unit's
@@ -41,6 +45,8 @@ constexpr int CONSUMER_WARPS = 3;
 constexpr int THREADS = 32 * (CONSUMER_WARPS + 1);
 constexpr int REC = 4 + 2 * 128;             // m, l, value-scale, pad, acc_v[128], acc_k[128]
 constexpr int SMEM_BYTES = SLOTS * SLOT_BYTES + 1024;   // + alignment slack; barriers live in static smem
+constexpr int W_BYTES = 32768;               // the unit's map as two swizzled 128 x 128 B boxes (per-tile form only)
+constexpr int SMEM_BYTES_PER_TILE = SMEM_BYTES + W_BYTES;
 constexpr int MAX_BLOCKS = 148;
 
 // How the tile sequence is dealt to blocks; the same arithmetic runs on host and device.
@@ -100,16 +106,20 @@ static_assert(SLOTS % CONSUMER_WARPS == 0, "a slot must always be consumed by th
 
 struct Maps {
     CUtensorMap ret_k, ret_v, apx_k;     // rank 3: (128 dims, pool rows, U units), box 64 x 64 x 1, 128B swizzle
+    CUtensorMap w;                       // rank 3: (128 in, 128 out, L*Hkv maps), box 64 x 128 x 1 (per-tile form only)
 };
 
 // grid (plan.B), THREADS threads, SMEM_BYTES dynamic shared memory.
 // partial: [U][s_max][CONSUMER_WARPS][g][REC]; slot of (unit u, block b) = b - block_of_tile(first tile of u).
+template <bool PER_TILE>
 __global__ void __launch_bounds__(THREADS, 1)
 decode_stream_bf16_d128(const __nv_bfloat16* __restrict__ q, const __grid_constant__ Maps maps, Plan pl, int n_ret,
-                        int n_apx, int g, float scale_log2e, float* __restrict__ partial, int* __restrict__ fault) {
+                        int n_apx, int g, int LH, float scale_log2e, float* __restrict__ partial,
+                        int* __restrict__ fault) {
     extern __shared__ unsigned char smem_raw[];
     __shared__ __align__(8) uint64_t full_bar[SLOTS];
     __shared__ __align__(8) uint64_t empty_bar[SLOTS];
+    __shared__ __align__(8) uint64_t w_bar;
     // 128B-swizzled TMA boxes want 1024-byte aligned destinations
     unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     const int b = blockIdx.x;
@@ -127,6 +137,7 @@ decode_stream_bf16_d128(const __nv_bfloat16* __restrict__ q, const __grid_consta
     if (tid == 0) {
 #pragma unroll
         for (int s = 0; s < SLOTS; ++s) { tma::mbar_init(&full_bar[s], 1); tma::mbar_init(&empty_bar[s], 1); }
+        tma::mbar_init(&w_bar, 1);
         tma::mbar_fence_init();
     }
     __syncthreads();
@@ -169,8 +180,9 @@ decode_stream_bf16_d128(const __nv_bfloat16* __restrict__ q, const __grid_consta
     const uint32_t pv_row = (uint32_t)(r8 + (mat & 1) * 8) * 128u;       // PV: matrices = (chunk lo|hi) x (keys 0-7|8-15)
     const uint32_t pv_x = (uint32_t)(((mat >> 1) ^ r8) << 4);
 
+    const uint32_t wbase = tma::smem_u32(smem + SLOTS * SLOT_BYTES);     // the unit's W (per-tile form only)
     uint32_t qa[8][2];
-    float acc[16][4];                  // [dim tile][c0,c1: P_hi rows | c2,c3: P_lo rows]
+    float acc[16][4];                  // [dim tile][c0,c1: P_hi rows | c2,c3: P_lo rows]; per-tile form: acc[0..7] = O^T
     float m = -INFINITY, l = 0.f, stash_scale = 1.f;
     bool stashed = false;
 
@@ -204,11 +216,21 @@ decode_stream_bf16_d128(const __nv_bfloat16* __restrict__ q, const __grid_consta
         if (gid < g) {
             float* rec = record_of(unit);
             if (tig == 0) *reinterpret_cast<float4*>(rec) = make_float4(m * 0.69314718055994531f, lt, stashed ? stash_scale : 1.f, 0.f);
-            if (stashed) store_acc(rec + 4 + 128);                     // value part was written at the pool switch
+            if (stashed) { if (!PER_TILE) store_acc(rec + 4 + 128); }  // value part was written at the pool switch
             else {
                 store_acc(rec + 4);
 #pragma unroll
                 for (int n = 0; n < 16; ++n) *reinterpret_cast<float2*>(rec + 4 + 128 + n * 8 + 2 * tig) = make_float2(0.f, 0.f);
+            }
+        }
+        if (PER_TILE && stashed) {
+            // acc[mt] holds O^T: dims mt*16 + gid (+8) x heads 2 tig, 2 tig + 1; it goes where the key sum would
+            float* rec0 = record_of(unit) - (size_t)gid * REC + 4 + 128;       // head 0 of this warp's record group
+#pragma unroll
+            for (int mt = 0; mt < 8; ++mt) {
+                const int dim = mt * 16 + gid;
+                if (2 * tig < g) { rec0[(size_t)(2 * tig) * REC + dim] = acc[mt][0]; rec0[(size_t)(2 * tig) * REC + dim + 8] = acc[mt][2]; }
+                if (2 * tig + 1 < g) { rec0[(size_t)(2 * tig + 1) * REC + dim] = acc[mt][1]; rec0[(size_t)(2 * tig + 1) * REC + dim + 8] = acc[mt][3]; }
             }
         }
         zero_acc();
@@ -261,8 +283,89 @@ decode_stream_bf16_d128(const __nv_bfloat16* __restrict__ q, const __grid_consta
         m = m_new;
         stash_scale *= alpha;
         if (__any_sync(0xffffffffu, alpha != 1.f)) {
+            if (PER_TILE && stashed) {
+                // O^T: this thread's columns are heads 2 tig and 2 tig + 1, whose factors live in the quads of those rows
+                const float al0 = __shfl_sync(0xffffffffu, alpha, 8 * tig), al1 = __shfl_sync(0xffffffffu, alpha, 8 * tig + 4);
 #pragma unroll
-            for (int n = 0; n < 16; ++n) { acc[n][0] *= alpha; acc[n][1] *= alpha; acc[n][2] *= alpha; acc[n][3] *= alpha; }
+                for (int n = 0; n < 8; ++n) { acc[n][0] *= al0; acc[n][1] *= al1; acc[n][2] *= al0; acc[n][3] *= al1; }
+            } else {
+#pragma unroll
+                for (int n = 0; n < 16; ++n) { acc[n][0] *= alpha; acc[n][1] *= alpha; acc[n][2] *= alpha; acc[n][3] *= alpha; }
+            }
+        }
+        if (PER_TILE && !retained) {
+            // ---- P^T as B operands (k = keys, n = heads), bf16 hi and lo, per 16-key k-step
+            uint32_t pb_hi[4][2], pb_lo[4][2];
+#pragma unroll
+            for (int kk = 0; kk < 4; ++kk) {
+#pragma unroll
+                for (int h = 0; h < 2; ++h) {
+                    const float p0 = sc[2 * kk + h][0], p1 = sc[2 * kk + h][1];
+                    const float h0 = __bfloat162float(__float2bfloat16_rn(p0)), h1 = __bfloat162float(__float2bfloat16_rn(p1));
+                    pb_hi[kk][h] = pack_bf16(h0, h1);
+                    pb_lo[kk][h] = pack_bf16(p0 - h0, p1 - h1);
+                }
+            }
+            const uint32_t w_row = (uint32_t)((lane & 7) + ((lane >> 3) & 1) * 8);      // A operand rows inside a 16-row tile
+            const uint32_t w_hi = (uint32_t)(lane >> 4);                              // second 16-byte chunk of the k-step
+#pragma unroll 1
+            for (int mg = 0; mg < 4; ++mg) {           // 32 output dims at a time
+                float vt[2][8][4];                     // V^T[dim][key] for two 16-dim row tiles x eight 8-key column tiles
+#pragma unroll
+                for (int i = 0; i < 2; ++i)
+#pragma unroll
+                    for (int n = 0; n < 8; ++n) { vt[i][n][0] = vt[i][n][1] = vt[i][n][2] = vt[i][n][3] = 0.f; }
+#pragma unroll
+                for (int ks = 0; ks < 8; ++ks) {
+                    uint32_t wa[2][4];
+#pragma unroll
+                    for (int i = 0; i < 2; ++i) {
+                        const uint32_t row = (uint32_t)((2 * mg + i) * 16) + w_row, chunk = 2 * ks + w_hi;
+                        ldsm_x4(wbase + (chunk >> 3) * 16384 + row * 128 + (((chunk & 7) ^ (row & 7)) << 4), wa[i][0], wa[i][1],
+                                wa[i][2], wa[i][3]);
+                    }
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) {
+                        uint32_t b0, b1, b2, b3;
+                        ldsm_x4(kbase + (ks >> 2) * BOX_BYTES + j * 16 * 128 + qk_row + ((((2 * ks) & 7) << 4) ^ qk_x), b0, b1, b2, b3);
+#pragma unroll
+                        for (int i = 0; i < 2; ++i) {
+                            mma_16(vt[i][2 * j], wa[i][0], wa[i][1], wa[i][2], wa[i][3], b0, b1);
+                            mma_16(vt[i][2 * j + 1], wa[i][0], wa[i][1], wa[i][2], wa[i][3], b2, b3);
+                        }
+                    }
+                }
+                // ---- O^T[dims][heads] += V^T P^T, V^T as A operand (accumulator layout = A layout), hi + lo
+                float ot[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
+#pragma unroll
+                for (int i = 0; i < 2; ++i) {
+#pragma unroll
+                    for (int kk = 0; kk < 4; ++kk) {
+                        uint32_t ah[4], al[4];
+#pragma unroll
+                        for (int r = 0; r < 4; ++r) {       // a0, a1: key tile 2kk rows gid, gid+8; a2, a3: key tile 2kk+1
+                            const float x0 = vt[i][2 * kk + (r >> 1)][(r & 1) * 2], x1 = vt[i][2 * kk + (r >> 1)][(r & 1) * 2 + 1];
+                            const float h0 = __bfloat162float(__float2bfloat16_rn(x0)), h1 = __bfloat162float(__float2bfloat16_rn(x1));
+                            ah[r] = pack_bf16(h0, h1);
+                            al[r] = pack_bf16(x0 - h0, x1 - h1);
+                        }
+                        mma_16(ot[i], ah[0], ah[1], ah[2], ah[3], pb_hi[kk][0], pb_hi[kk][1]);
+                        mma_16(ot[i], al[0], al[1], al[2], al[3], pb_hi[kk][0], pb_hi[kk][1]);
+                        mma_16(ot[i], ah[0], ah[1], ah[2], ah[3], pb_lo[kk][0], pb_lo[kk][1]);
+                    }
+                }
+                // add into the running O^T; the loop over mg stays rolled, so the register index is made static
+#pragma unroll
+                for (int ms = 0; ms < 4; ++ms) {
+                    if (ms == mg) {
+#pragma unroll
+                        for (int i = 0; i < 2; ++i)
+#pragma unroll
+                            for (int r = 0; r < 4; ++r) acc[2 * ms + i][r] += ot[i][r];
+                    }
+                }
+            }
+            return;
         }
         // ---- accumulate P x (V rows | K rows): four k-steps of 16 keys x 16 column tiles of 8 dims
 #pragma unroll
@@ -288,14 +391,28 @@ decode_stream_bf16_d128(const __nv_bfloat16* __restrict__ q, const __grid_consta
     zero_acc();
     // Walk the units the block touches; this warp owns the block's tiles i with i % CONSUMER_WARPS == wq.
     int i = wq;                                        // index into the block's tile sequence
-    for (int u = u0; u <= u_last; ++u) {
+    bool ok = true;                                    // false once a wait gave up: keep walking, touch nothing
+    uint32_t units_done = 0;
+    for (int u = u0; u <= u_last; ++u, ++units_done) {
+        if (PER_TILE) {
+            // all three warps have left the previous unit: its W may be replaced
+            asm volatile("bar.sync 1, %0;\n" ::"n"(32 * CONSUMER_WARPS) : "memory");
+            if (wq == 0 && lane == 0) {
+                tma::mbar_expect_tx(&w_bar, W_BYTES);
+                tma::load_3d(smem + SLOTS * SLOT_BYTES, &maps.w, 0, 0, u % LH, &w_bar);
+                tma::load_3d(smem + SLOTS * SLOT_BYTES + W_BYTES / 2, &maps.w, 64, 0, u % LH, &w_bar);
+            }
+            if (ok) ok = tma::mbar_wait_warp(&w_bar, units_done & 1, fault, 4);
+        }
         const long long unit_end = (long long)(u + 1) * pl.n_tiles - gt_lo;     // first sequence index past the unit
         bool loaded = false;
         for (; i < n_my && i < unit_end; i += CONSUMER_WARPS) {
+            if (!ok) continue;
             if (!loaded) { load_q(u); loaded = true; }
             const int s = i % SLOTS, round = i / SLOTS;
             const int t = (int)(gt_lo + i - (long long)u * pl.n_tiles);
-            if (!tma::mbar_wait_warp(&full_bar[s], round & 1, fault, 2)) return;
+            ok = tma::mbar_wait_warp(&full_bar[s], round & 1, fault, 2);
+            if (!ok) continue;
             const uint32_t base = tma::smem_u32(smem + s * SLOT_BYTES);
             if (t < pl.n_rt) {
                 step64(base, base + HALF_BYTES, min(KEYS, n_ret - t * KEYS), true, u);
@@ -318,7 +435,7 @@ decode_stream_bf16_d128(const __nv_bfloat16* __restrict__ q, const __grid_consta
 template <typename TO>
 __global__ void __launch_bounds__(1024)
 decode_merge_bf16_d128(const float* __restrict__ partial, const __nv_bfloat16* __restrict__ W, int LH, int g,
-                       Plan pl, TO* __restrict__ out) {
+                       Plan pl, int apply_w, TO* __restrict__ out) {
     __shared__ uint32_t Ws[128 * 65];          // W rows as bf16 pairs, row stride 65 words (conflict-free)
     __shared__ __align__(8) float aks[8][128];
     __shared__ float fv[8][48], fk[8][48];     // per head, per record: factor for the value part / the key part
@@ -327,7 +444,7 @@ decode_merge_bf16_d128(const float* __restrict__ partial, const __nv_bfloat16* _
     const int nthr = blockDim.x;
     // W tile into shared memory (overlaps the tail of the streaming kernel): 2048 16-byte pieces
     const uint4* Wu = reinterpret_cast<const uint4*>(W + (size_t)(u % LH) * 128 * 128);
-    for (int i = tid; i < 2048; i += nthr) {
+    for (int i = tid; i < (apply_w ? 2048 : 0); i += nthr) {
         const uint4 v = Wu[i];
         uint32_t* dst = Ws + (i >> 4) * 65 + (i & 15) * 4;      // 16 pieces per 256-byte row
         dst[0] = v.x; dst[1] = v.y; dst[2] = v.z; dst[3] = v.w;
@@ -379,6 +496,10 @@ decode_merge_bf16_d128(const float* __restrict__ partial, const __nv_bfloat16* _
                 ak = fmaf(fk[a][j0 + k], rk[k], ak);
             }
         }
+    }
+    if (!apply_w) {           // per-tile form: the second part of a record is already sum p (W k)
+        store_out(out + ((size_t)u * g + a) * 128 + c, (av + ak) / Ls[a]);
+        return;
     }
     aks[a][c] = ak;
     __syncthreads();

@@ -247,6 +247,14 @@ def _run_pipeline_case(oracle, wl, percent, units=None, decode_steps=2, n_a=-1, 
             assert err <= 2e-2, f"decode step {step} unit {units[j]}: abs err {err}"
             errb = np.abs(out_bf[j].cpu().double().numpy() - o_fac)
             assert np.all(errb <= 2e-2 + 2.0 ** -8 * np.abs(o_fac))
+        if wl.dtype == "bf16" and wl.head_dim == 128 and theta is None:
+            comp.decode(q, W, out, mode=1)              # per-tile reconstruction: sum_A p (W k) formed tile by tile
+            torch.cuda.synchronize()
+            for j in range(len(units)):
+                o_tok, _ = oracle.attend(q[j].cpu(), c.ret_k[j, : c.n_ret].cpu(), c.ret_v[j, : c.n_ret].cpu(),
+                                         c.apx_k[j, : c.n_apx].cpu(), W[j].cpu(), scale)
+                err = np.max(np.abs(out[j].cpu().double().numpy() - o_tok))
+                assert err <= 2e-2, f"per-tile decode step {step} unit {units[j]}: abs err {err}"
         kn, vn = synth.decode_kv(wl, step, DEV, sk, wt, units)
         comp.append(kn, vn, wl.N + step)
 
@@ -344,12 +352,13 @@ def test_decode_degenerate_pools(oracle):
     ipos = torch.arange(512, dtype=torch.int32, device=DEV).repeat(wl.units, 1).contiguous()
     for n_ret, n_apx in [(512, 0), (0, 512), (1, 0), (0, 1), (300, 1), (1, 300), (257, 255)]:
         cache = vec.Cache(K.clone(), V.clone(), K.flip(1).contiguous(), ipos, ipos.clone(), n_ret, n_apx)
-        vec.vector_decode_attn(sh, q, cache, W, out, 0, ws)
-        torch.cuda.synchronize()
-        for u in range(wl.units):
-            _, o = oracle.attend(q[u].cpu(), cache.ret_k[u, :n_ret].cpu(), cache.ret_v[u, :n_ret].cpu(),
-                                 cache.apx_k[u, :n_apx].cpu(), W[u].cpu(), scale)
-            assert np.max(np.abs(out[u].cpu().double().numpy() - o)) <= 2e-2, (n_ret, n_apx, u)
+        for mode in (0, 1):
+            vec.vector_decode_attn(sh, q, cache, W, out, mode, ws)
+            torch.cuda.synchronize()
+            for u in range(wl.units):
+                _, o = oracle.attend(q[u].cpu(), cache.ret_k[u, :n_ret].cpu(), cache.ret_v[u, :n_ret].cpu(),
+                                     cache.apx_k[u, :n_apx].cpu(), W[u].cpu(), scale)
+                assert np.max(np.abs(out[u].cpu().double().numpy() - o)) <= 2e-2, (n_ret, n_apx, u, mode)
 
 
 def test_decode_long_block_ranges(oracle):
@@ -367,13 +376,16 @@ def test_decode_long_block_ranges(oracle):
         out = torch.empty(wl.units, wl.group, wl.head_dim, dtype=torch.float32, device=DEV)
         ipos = torch.arange(wl.N, dtype=torch.int32, device=DEV).repeat(wl.units, 1).contiguous()
         cache = vec.Cache(K.clone(), V.clone(), K.flip(1).contiguous(), ipos, ipos.clone(), n_ret, n_apx)
+        out1 = torch.empty_like(out)
         vec.vector_decode_attn(sh, q, cache, W, out, 0, ws)
+        vec.vector_decode_attn(sh, q, cache, W, out1, 1, ws)
         torch.cuda.synchronize()
         assert vec.vector_device_fault() == 0
         for u in range(wl.units):
-            _, o = oracle.attend(q[u].cpu(), cache.ret_k[u, :n_ret].cpu(), cache.ret_v[u, :n_ret].cpu(),
-                                 cache.apx_k[u, :n_apx].cpu(), W[u].cpu(), 1.0 / np.sqrt(wl.head_dim))
+            o_tok, o = oracle.attend(q[u].cpu(), cache.ret_k[u, :n_ret].cpu(), cache.ret_v[u, :n_ret].cpu(),
+                                     cache.apx_k[u, :n_apx].cpu(), W[u].cpu(), 1.0 / np.sqrt(wl.head_dim))
             assert np.max(np.abs(out[u].cpu().double().numpy() - o)) <= 2e-2, (base, u)
+            assert np.max(np.abs(out1[u].cpu().double().numpy() - o_tok)) <= 2e-2, (base, u, "per tile")
 
 
 def test_full_size_bench_configuration_sampled_units(oracle):
