@@ -296,13 +296,9 @@ def main():
             phase[name].append(m[i].elapsed_time(m[i + 1]))
     ms = {k: statistics.mean(v) for k, v in phase.items()}
     compress_ms = ms["score"] + ms["route"] + ms["compact"]
-    if world > 1:
-        import torch.distributed as dist
-        t = torch.tensor([total_ms, compress_ms, ms["decode"]], device=dev, dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        total_ms, compress_ms, dec_ms_max = t.tolist()
-    else:
-        dec_ms_max = ms["decode"]
+    # every rank is an independent replica: the job's time is the slowest replica's
+    from paper_2605_23258_b200 import replicas
+    total_ms, compress_ms, dec_ms_max = replicas.slowest([total_ms, compress_ms, ms["decode"]], dev)
 
     # ---- algorithmic work (per step, one replica)
     n_ret, n_apx, n_pool = budget.n_ret, budget.n_apx, budget.n_pool
@@ -400,11 +396,7 @@ def main():
             e2e_decode()
         b_.record(); torch.cuda.synchronize()
         ed_ms = a.elapsed_time(b_) / 20
-        if world > 1:
-            import torch.distributed as dist
-            t = torch.tensor([e_ms, ed_ms], device=dev, dtype=torch.float64)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            e_ms, ed_ms = t.tolist()
+        e_ms, ed_ms = replicas.slowest([e_ms, ed_ms], dev)
         h2d = (hK.numel() + hV.numel() + hQ.numel()) * es
         d2h = h_tier.numel() + (h_ret.numel() + h_apx.numel()) * 4
         e2e = {"value": world * wl.batch * N / (e_ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
