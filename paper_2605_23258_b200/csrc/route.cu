@@ -26,6 +26,20 @@ __device__ __forceinline__ uint32_t select_image(float v) {
     return SMALLEST ? ~k : k;
 }
 
+// hist[bin] += 1 for every lane with `valid`.  When the whole warp hits one bin (common in the later
+// passes, where the surviving keys share their leading bits) a single lane adds the count.
+// Every lane of the warp must call it.
+__device__ __forceinline__ void hist_add(int* hist, int bin, bool valid) {
+    const unsigned active = __ballot_sync(0xffffffffu, valid);
+    if (active == 0) return;
+    const int first = __shfl_sync(0xffffffffu, bin, __ffs(active) - 1);
+    if (__ballot_sync(0xffffffffu, valid && bin != first) == 0) {
+        if ((int)(threadIdx.x & 31) == __ffs(active) - 1) atomicAdd(&hist[first], __popc(active));
+    } else if (valid) {
+        atomicAdd(&hist[bin], 1);
+    }
+}
+
 // Finds the k-th largest image among vals[0..n) (1 <= k <= n).  All threads of the
 // block call it and all get the result.  hist: 256 ints of shared memory; bc: 2 ints.
 template <bool SMALLEST>
@@ -35,24 +49,46 @@ __device__ SelectResult radix_select(const float* __restrict__ vals, int n, int 
     for (int shift = 24; shift >= 0; shift -= 8) {
         for (int b = threadIdx.x; b < 256; b += blockDim.x) hist[b] = 0;
         __syncthreads();
-        for (int i = threadIdx.x; i < n; i += blockDim.x) {
-            uint32_t key = select_image<SMALLEST>(vals[i]);
-            if ((key & mask) == prefix) atomicAdd(&hist[(key >> shift) & 255], 1);
+        // eight independent loads in flight per thread: the pass is bound by memory latency otherwise
+        for (int base = 0; base < n; base += 8 * blockDim.x) {
+            float v[8];
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+                const int i = base + j * blockDim.x + threadIdx.x;
+                v[j] = i < n ? vals[i] : 0.f;
+            }
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+                const int i = base + j * blockDim.x + threadIdx.x;
+                const uint32_t key = select_image<SMALLEST>(v[j]);
+                hist_add(hist, (key >> shift) & 255, i < n && (key & mask) == prefix);
+            }
         }
         __syncthreads();
-        if (threadIdx.x == 0) {
-            int cum = 0, b = 255;
-            for (; b > 0; --b) {
-                if (cum + hist[b] >= remaining) break;
-                cum += hist[b];
+        if (threadIdx.x < 32) {
+            // warp 0: the bin, counted from the top, in which the cumulative count reaches `remaining`
+            int c[8], tot = 0;
+#pragma unroll
+            for (int j = 0; j < 8; ++j) { c[j] = hist[255 - (threadIdx.x * 8 + j)]; tot += c[j]; }
+            int inc = tot;
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                const int t = __shfl_up_sync(0xffffffffu, inc, o);
+                if ((int)threadIdx.x >= o) inc += t;
             }
-            bc[0] = b;
-            bc[1] = remaining - cum;    // rank wanted inside bin b (1-based)
+            int cum = inc - tot;                            // count in the bins above this lane's eight
+            if (cum < remaining && inc >= remaining) {      // exactly one lane
+#pragma unroll
+                for (int j = 0; j < 8; ++j) {
+                    if (cum + c[j] >= remaining) { bc[0] = 255 - (threadIdx.x * 8 + j); bc[1] = remaining - cum; break; }
+                    cum += c[j];
+                }
+            }
         }
         __syncthreads();
         prefix |= (uint32_t)bc[0] << shift;
         mask |= 255u << shift;
-        remaining = bc[1];
+        remaining = bc[1];              // rank wanted inside the chosen bin (1-based)
         __syncthreads();
     }
     SelectResult r;
@@ -61,69 +97,94 @@ __device__ SelectResult radix_select(const float* __restrict__ vals, int n, int 
     return r;
 }
 
-// Block-wide exclusive prefix sum of one int per thread; returns the exclusive
-// prefix and writes the block total to *total.  warp_tot: 32 ints of shared memory.
-__device__ __forceinline__ int block_exclusive_scan(int v, int* warp_tot, int* total) {
+// The ordered pass both selections end with.  Every warp owns a contiguous piece of the input and
+// walks it 32 elements at a time (coalesced); positions inside a warp come from ballots, the
+// offsets of the warps from one small scan by warp 0.  `emit(i, chosen, pos)` is called for every
+// element i: pos is its rank among the chosen ones if chosen, else among the others.
+struct OrderedScratch { int gt[32], tie[32], out[32], quota[32]; };
+
+template <bool SMALLEST, typename Emit>
+__device__ __forceinline__ void ordered_pass(const float* __restrict__ vals, int n, const SelectResult& sel, bool any,
+                                             OrderedScratch& sc, Emit emit) {
     const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5, nw = blockDim.x >> 5;
-    int inc = v;
+    const unsigned lt = (1u << lane) - 1u;
+    const int per_w = (((n + nw - 1) / nw) + 31) & ~31;
+    const int w0 = min(n, wid * per_w), w1 = min(n, w0 + per_w);
+    int n_gt = 0, n_tie = 0;
+    if (any) {
+        for (int base = w0; base < w1; base += 128) {
+            float v[4];
 #pragma unroll
-    for (int o = 1; o < 32; o <<= 1) {
-        int t = __shfl_up_sync(0xffffffffu, inc, o);
-        if (lane >= o) inc += t;
+            for (int j = 0; j < 4; ++j) v[j] = base + 32 * j + lane < w1 ? vals[base + 32 * j + lane] : 0.f;
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                const bool in = base + 32 * j + lane < w1;
+                const uint32_t key = select_image<SMALLEST>(v[j]);
+                n_gt += __popc(__ballot_sync(0xffffffffu, in && key > sel.kth_key));
+                n_tie += __popc(__ballot_sync(0xffffffffu, in && key == sel.kth_key));
+            }
+        }
     }
-    __syncthreads();            // protects warp_tot against the previous call's readers
-    if (lane == 31) warp_tot[wid] = inc;
+    if (lane == 0) { sc.gt[wid] = n_gt; sc.tie[wid] = n_tie; }
     __syncthreads();
     if (wid == 0) {
-        int t = lane < nw ? warp_tot[lane] : 0;
-        int ti = t;
+        const int t = lane < nw ? sc.tie[lane] : 0;
+        int inc = t;
 #pragma unroll
-        for (int o = 1; o < 32; o <<= 1) {
-            int s = __shfl_up_sync(0xffffffffu, ti, o);
-            if (lane >= o) ti += s;
-        }
-        warp_tot[lane] = ti - t;   // exclusive warp offsets; lane 31 holds total - last
-        if (lane == 31) *total = ti;
+        for (int o = 1; o < 32; o <<= 1) { const int x = __shfl_up_sync(0xffffffffu, inc, o); if (lane >= o) inc += x; }
+        const int quota = max(0, min(t, sel.take_ties - (inc - t)));       // ties go to the lowest indices
+        const int c = (lane < nw ? sc.gt[lane] : 0) + quota;
+        int ci = c;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) { const int x = __shfl_up_sync(0xffffffffu, ci, o); if (lane >= o) ci += x; }
+        sc.out[lane] = ci - c;
+        sc.quota[lane] = quota;
     }
     __syncthreads();
-    return warp_tot[wid] + inc - v;
+    int pos = sc.out[wid], ties_left = sc.quota[wid];
+    for (int base = w0; base < w1; base += 128) {
+        float v[4];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) v[j] = base + 32 * j + lane < w1 ? vals[base + 32 * j + lane] : 0.f;
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const int i = base + 32 * j + lane;
+            const bool in = i < w1;
+            const uint32_t key = select_image<SMALLEST>(v[j]);
+            const bool tie = any && in && key == sel.kth_key;
+            const unsigned tb = __ballot_sync(0xffffffffu, tie);
+            const bool chosen = any && in && (key > sel.kth_key || (tie && __popc(tb & lt) < ties_left));
+            const unsigned cb = __ballot_sync(0xffffffffu, chosen);
+            const int before = pos + __popc(cb & lt);               // chosen elements before this one in the unit
+            if (in) emit(i, chosen, chosen ? before : i - before);
+            pos += __popc(cb);
+            ties_left -= min(ties_left, __popc(tb));
+        }
+    }
 }
 
 // Step 1.  grid (U), SEL_THREADS threads.
-__global__ void __launch_bounds__(SEL_THREADS)
+__global__ void __launch_bounds__(SEL_THREADS, 2)
 pool_select_kernel(const float* __restrict__ scores, int64_t N, int n_pool, int32_t* __restrict__ pool_idx) {
     __shared__ int hist[256];
     __shared__ int bc[2];
-    __shared__ int warp_tot[32];
-    __shared__ int tot;
+    __shared__ OrderedScratch sc;
     const int u = blockIdx.x, n = (int)N;
     const float* s = scores + (size_t)u * N;
     int32_t* out = pool_idx + (size_t)u * n_pool;
     if (n_pool <= 0) return;
-    SelectResult sel = radix_select<false>(s, n, n_pool, hist, bc);
-    int ties_seen = 0, written = 0;
-    for (int base = 0; base < n; base += SEL_THREADS) {
-        int i = base + threadIdx.x;
-        uint32_t key = i < n ? select_image<false>(s[i]) : 0u;
-        int is_tie = (i < n && key == sel.kth_key) ? 1 : 0;
-        int tie_rank = ties_seen + block_exclusive_scan(is_tie, warp_tot, &tot);
-        ties_seen += tot;
-        int chosen = (i < n && (key > sel.kth_key || (is_tie && tie_rank < sel.take_ties))) ? 1 : 0;
-        int pos = written + block_exclusive_scan(chosen, warp_tot, &tot);
-        written += tot;
-        if (chosen) out[pos] = i;
-    }
+    const SelectResult sel = radix_select<false>(s, n, n_pool, hist, bc);
+    ordered_pass<false>(s, n, sel, true, sc, [&](int i, bool chosen, int pos) { if (chosen) out[pos] = i; });
 }
 
 // Step 3.  grid (U), SEL_THREADS threads.
-__global__ void __launch_bounds__(SEL_THREADS)
+__global__ void __launch_bounds__(SEL_THREADS, 2)
 truncate_kernel(const float* __restrict__ eps, const int32_t* __restrict__ pool_idx, int64_t N, int n_pool,
                 int n_apx, uint8_t* __restrict__ tier, int32_t* __restrict__ ret_idx,
                 int32_t* __restrict__ apx_idx) {
     __shared__ int hist[256];
     __shared__ int bc[2];
-    __shared__ int warp_tot[32];
-    __shared__ int tot;
+    __shared__ OrderedScratch sc;
     const int u = blockIdx.x;
     const float* e = eps + (size_t)u * n_pool;
     const int32_t* pool = pool_idx + (size_t)u * n_pool;
@@ -131,32 +192,21 @@ truncate_kernel(const float* __restrict__ eps, const int32_t* __restrict__ pool_
     const int n_ret = n_pool - n_apx;
     int32_t* ro = ret_idx + (size_t)u * n_ret;
     int32_t* ao = apx_idx + (size_t)u * n_apx;
-    for (int64_t i = threadIdx.x; i < N; i += SEL_THREADS) tr[i] = 0;
+    if ((N & 15) == 0) {
+        for (int64_t i = threadIdx.x; i < N / 16; i += SEL_THREADS) reinterpret_cast<uint4*>(tr)[i] = make_uint4(0, 0, 0, 0);
+    } else {
+        for (int64_t i = threadIdx.x; i < N; i += SEL_THREADS) tr[i] = 0;
+    }
     __syncthreads();
     SelectResult sel;
     sel.kth_key = 0xffffffffu;
     sel.take_ties = 0;
     if (n_apx > 0) sel = radix_select<true>(e, n_pool, n_apx, hist, bc);
-    int ties_seen = 0, n_a_written = 0, n_r_written = 0;
-    for (int base = 0; base < n_pool; base += SEL_THREADS) {
-        int p = base + threadIdx.x;
-        bool in = p < n_pool;
-        uint32_t key = in ? select_image<true>(e[p]) : 0u;
-        int is_tie = (in && n_apx > 0 && key == sel.kth_key) ? 1 : 0;
-        int tie_rank = ties_seen + block_exclusive_scan(is_tie, warp_tot, &tot);
-        ties_seen += tot;
-        int is_apx = (in && n_apx > 0 && (key > sel.kth_key || (is_tie && tie_rank < sel.take_ties))) ? 1 : 0;
-        int a_pos = n_a_written + block_exclusive_scan(is_apx, warp_tot, &tot);
-        n_a_written += tot;
-        int is_ret = (in && !is_apx) ? 1 : 0;
-        int r_pos = n_r_written + block_exclusive_scan(is_ret, warp_tot, &tot);
-        n_r_written += tot;
-        if (in) {
-            int32_t token = pool[p];
-            if (is_apx) { ao[a_pos] = token; tr[token] = 1; }
-            else        { ro[r_pos] = token; tr[token] = 2; }
-        }
-    }
+    ordered_pass<true>(e, n_pool, sel, n_apx > 0, sc, [&](int p, bool is_apx, int pos) {
+        const int32_t token = pool[p];
+        if (is_apx) { ao[pos] = token; tr[token] = 1; }
+        else        { ro[pos] = token; tr[token] = 2; }
+    });
 }
 
 // Step 2 on CUDA cores.  grid (ceil(n_idx / 64), U), 256 threads; W^T staged in
