@@ -242,7 +242,10 @@ static vector_status launch_score_tc(const Dims& dm, const void* Q, const void* 
     stc::score_pass2_tc<<<blocks, stc::THREADS, stc::SMEM_BYTES, st>>>(mapQ, mapK, P, lse2, raw_part, fault);
     VEC_LAUNCH_CHECK();
     dim3 gp((unsigned)((N + stc::POOL_TILE - 1) / stc::POOL_TILE), dm.U);
-    stc::score_pool_parts<<<gp, 256, 0, st>>>(raw_part, 2 * pl.RG, N, dm.w, dm.pool_kernel / 2, raw_out, scores);
+    if ((N & 3) == 0)
+        stc::score_pool_parts_v4<<<gp, 256, 0, st>>>(raw_part, 2 * pl.RG, N, dm.w, dm.pool_kernel / 2, raw_out, scores);
+    else
+        stc::score_pool_parts<<<gp, 256, 0, st>>>(raw_part, 2 * pl.RG, N, dm.w, dm.pool_kernel / 2, raw_out, scores);
     VEC_LAUNCH_CHECK();
     return VECTOR_OK;
 }

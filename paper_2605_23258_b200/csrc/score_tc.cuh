@@ -519,6 +519,53 @@ score_pool_parts(const float* __restrict__ raw_part, int parts, long long N, int
     }
 }
 
+// The same for N a multiple of 4: 16-byte loads and stores, four keys per thread.
+__global__ void __launch_bounds__(256)
+score_pool_parts_v4(const float* __restrict__ raw_part, int parts, long long N, int w, int r, float* __restrict__ raw_out,
+                    float* __restrict__ score) {
+    __shared__ __align__(16) float rs[POOL_TILE + 16];          // keys i0 - 8 .. i0 + POOL_TILE + 8
+    const int u = blockIdx.y;
+    const long long i0 = (long long)blockIdx.x * POOL_TILE;
+    const float* base = raw_part + (size_t)u * parts * N;
+    const long long P = N - w;
+    for (int e4 = threadIdx.x; e4 < (POOL_TILE + 16) / 4; e4 += 256) {
+        const long long i = i0 - 8 + 4 * e4;
+        float4 v = make_float4(-INFINITY, -INFINITY, -INFINITY, -INFINITY);
+        if (i >= 0 && i < N) {
+            v = *reinterpret_cast<const float4*>(base + i);
+            for (int p = 1; p < parts; ++p) {
+                const float4 x = *reinterpret_cast<const float4*>(base + (size_t)p * N + i);
+                v.x += x.x; v.y += x.y; v.z += x.z; v.w += x.w;
+            }
+            if (raw_out && e4 >= 2 && e4 < 2 + POOL_TILE / 4) *reinterpret_cast<float4*>(raw_out + (size_t)u * N + i) = v;
+            if (i + 0 >= P) v.x = -INFINITY;           // pooling looks at the prefix only
+            if (i + 1 >= P) v.y = -INFINITY;
+            if (i + 2 >= P) v.z = -INFINITY;
+            if (i + 3 >= P) v.w = -INFINITY;
+        }
+        *reinterpret_cast<float4*>(rs + 4 * e4) = v;
+    }
+    __syncthreads();
+    const long long i = i0 + 4 * threadIdx.x;
+    if (i >= N) return;
+    float x[20];                                                // keys i - 8 .. i + 11
+#pragma unroll
+    for (int k = 0; k < 5; ++k) {
+        const float4 v = *reinterpret_cast<const float4*>(rs + 4 * threadIdx.x + 4 * k);
+        x[4 * k] = v.x; x[4 * k + 1] = v.y; x[4 * k + 2] = v.z; x[4 * k + 3] = v.w;
+    }
+    float o[4];
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+        float best = x[8 + j];
+#pragma unroll
+        for (int k = 1; k <= 7; ++k)
+            if (k <= r) best = fmaxf(best, fmaxf(x[8 + j - k], x[8 + j + k]));
+        o[j] = i + j < P ? best : INFINITY;
+    }
+    *reinterpret_cast<float4*>(score + (size_t)u * N + i) = make_float4(o[0], o[1], o[2], o[3]);
+}
+
 }  // namespace stc
 }  // namespace vec
 #endif
