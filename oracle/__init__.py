@@ -142,6 +142,16 @@ def score(Q, K, scale: float, pool_kernel: int):
     return raw, sc
 
 
+def score_keydiff(K) -> np.ndarray:
+    """Key-geometry scorer: K [N][d] -> score [N] float64 (minus the cosine to the mean unit key)."""
+    K = _f64(K)
+    N, d = K.shape
+    sc = np.empty(N, dtype=np.float64)
+    rc = lib().oracle_score_keydiff(_p(K), ctypes.c_int32(d), ctypes.c_int64(N), _p(sc))
+    _check(rc, "score_keydiff")
+    return sc
+
+
 def pool_select(score_f32, n_pool: int) -> np.ndarray:
     s = _f32(score_f32)
     out = np.empty(n_pool, dtype=np.int32)

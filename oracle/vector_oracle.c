@@ -207,6 +207,41 @@ int oracle_score(const double* Q, const double* K, int32_t g, int32_t w, int32_t
     return ORACLE_OK;
 }
 
+/*
+ * Query-agnostic base scorer by key geometry (the KeyDiff-style scorer the paper names among
+ * the base scorers of Step 1 and describes as "key geometric diversity"; it gives no formula, so
+ * this follows the published idea): the anchor is the mean of the unit-normalised keys, and a
+ * token is the more important the less its key points along the anchor:
+ *   a = (1/N) sum_j k_j / ||k_j||,   score_i = - <k_i, a> / (||k_i|| ||a||).
+ * No observation window, no pooling.  A zero key has cosine 0 with everything (score 0); if
+ * the anchor itself is zero every score is 0.  K: [N][d]; score_out: [N].
+ */
+int oracle_score_keydiff(const double* K, int32_t d, int64_t N, double* score_out) {
+    if (!K || !score_out || d <= 0 || N <= 0) return ORACLE_ERR_ARG;
+    double* a = (double*)calloc((size_t)d, sizeof(double));
+    double* nrm = (double*)malloc((size_t)N * sizeof(double));
+    if (!a || !nrm) { free(a); free(nrm); return ORACLE_ERR_ARG; }
+    for (int64_t i = 0; i < N; ++i) {
+        const double* k = K + i * d;
+        double n2 = 0.0;
+        for (int c = 0; c < d; ++c) n2 += k[c] * k[c];
+        nrm[i] = sqrt(n2);
+        if (nrm[i] > 0.0)
+            for (int c = 0; c < d; ++c) a[c] += k[c] / nrm[i];
+    }
+    double an2 = 0.0;
+    for (int c = 0; c < d; ++c) { a[c] /= (double)N; an2 += a[c] * a[c]; }
+    double an = sqrt(an2);
+    for (int64_t i = 0; i < N; ++i) {
+        const double* k = K + i * d;
+        double dot = 0.0;
+        for (int c = 0; c < d; ++c) dot += k[c] * a[c];
+        score_out[i] = (nrm[i] > 0.0 && an > 0.0) ? -dot / (nrm[i] * an) : 0.0;
+    }
+    free(a); free(nrm);
+    return ORACLE_OK;
+}
+
 /* ---- routing ---- */
 typedef struct { float key; int32_t idx; } f_item;
 typedef struct { double key; int32_t idx; } d_item;

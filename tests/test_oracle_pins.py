@@ -447,3 +447,34 @@ def test_end_to_end_no_eviction_noise_free_equals_uncompressed(oracle):
     o1, o2 = oracle.attend(q, rk, rv, ak, W, 1 / np.sqrt(d))
     ref = _attn_ref(q, K, V, 1 / np.sqrt(d))
     assert np.allclose(o1, ref, atol=1e-7) and np.allclose(o2, ref, atol=1e-7)
+
+
+def test_keydiff_scorer_pins(oracle):
+    """The key-geometry scorer against what its definition fixes (none of these retypes the formula):
+    identical keys all sit on the anchor; two unit keys at angle t are bisected by it; scores do not
+    change when keys are rescaled or reordered; an isolated direction scores highest; the range is [-1, 1]."""
+    rng = np.random.default_rng(3)
+    d = 16
+    k = rng.standard_normal(d)
+    same = np.tile(k, (9, 1)) * rng.uniform(0.1, 5.0, size=(9, 1))          # same direction, different lengths
+    assert np.allclose(oracle.score_keydiff(same), -1.0, atol=1e-12)
+    for t in (0.3, 1.0, 2.5):
+        two = np.zeros((2, d)); two[0, 0] = 1.0; two[1, 0], two[1, 1] = np.cos(t), np.sin(t)
+        assert np.allclose(oracle.score_keydiff(two), -np.cos(t / 2), atol=1e-12)
+    K = rng.standard_normal((200, d)) + 2.0 * k                              # a cloud around one direction
+    s0 = oracle.score_keydiff(K)
+    assert np.all(s0 >= -1 - 1e-12) and np.all(s0 <= 1 + 1e-12)
+    scale = rng.uniform(0.01, 100.0, size=(200, 1))
+    assert np.allclose(oracle.score_keydiff(K * scale), s0, atol=1e-10)      # lengths do not matter
+    perm = rng.permutation(200)
+    assert np.allclose(oracle.score_keydiff(K[perm]), s0[perm], atol=1e-12)  # order does not matter
+    K2 = K.copy(); K2[17] = -3.0 * k                                         # one key pointing the other way
+    s2 = oracle.score_keydiff(K2)
+    assert int(np.argmax(s2)) == 17 and s2[17] > 0.9
+    # rotating every key by one orthogonal map leaves all cosines unchanged
+    Qm, _ = np.linalg.qr(rng.standard_normal((d, d)))
+    assert np.allclose(oracle.score_keydiff(K @ Qm.T), s0, atol=1e-10)
+    # a zero key is orthogonal to everything; antipodal pairs cancel the anchor
+    K3 = K.copy(); K3[5] = 0.0
+    assert oracle.score_keydiff(K3)[5] == 0.0
+    assert np.all(oracle.score_keydiff(np.stack([k, -k])) == 0.0)
