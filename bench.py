@@ -357,6 +357,21 @@ def main():
         per_tile = {"us_per_step": us, "gbs": step_bytes / us / 1e3,
                     "extra_flop_per_step": 2.0 * U * n_apx * d * d}
 
+    # ---- the query-agnostic base scorer (key geometry), outside the timed step: two HBM passes over K
+    kd_scores = torch.empty(U, N, dtype=torch.float32, device=dev)
+    for _ in range(2):
+        vec.vector_score_keydiff(shape, Kt, N, kd_scores, comp.ws)
+    a, b_ = ev(), ev()
+    torch.cuda.synchronize(); a.record()
+    for _ in range(5):
+        vec.vector_score_keydiff(shape, Kt, N, kd_scores, comp.ws)
+    b_.record(); torch.cuda.synchronize()
+    kd_ms = a.elapsed_time(b_) / 5
+    kd_bytes = U * (2 * N * d * es + 3 * N * 4)
+    keydiff = {"ms": kd_ms, "gbs": kd_bytes / (kd_ms * 1e-3) / 1e9, "frac_of_measured_copy": kd_bytes / (kd_ms * 1e-3) / 1e9 / hbm,
+               "tokens_per_s": wl.batch * N / (kd_ms * 1e-3)}
+    del kd_scores
+
     # ---- end to end through host buffers (rank 0 semantics on every rank; reported from rank 0)
     e2e = None
     if not args.no_e2e:
@@ -434,7 +449,7 @@ def main():
         "decode": {"gbs": decode_bytes / (dec_ms_max * 1e-3) / 1e9, "frac_of_measured_copy": decode_bytes / (dec_ms_max * 1e-3) / 1e9 / hbm,
                    "frac_of_8tbs": decode_bytes / (dec_ms_max * 1e-3) / 1e9 / 8000.0, "us_per_step": dec_ms_max * 1e3 / D,
                    "tokens_per_s": world * wl.batch * D / (dec_ms_max * 1e-3), "bytes_per_step": decode_bytes / D},
-        "decode_per_tile": per_tile, "roofline": roofline, "roofline_kernels": kernels, "cpu_baseline": cpu, "e2e": e2e,
+        "decode_per_tile": per_tile, "score_keydiff": keydiff, "roofline": roofline, "roofline_kernels": kernels, "cpu_baseline": cpu, "e2e": e2e,
         "gpu_launches": kernels_per_step * K_steps, "clocks": clocks,
     }
     print(json.dumps(line))

@@ -151,6 +151,18 @@ VECTOR_API vector_status vector_score(const vector_shape* shape, const void* Q_o
                            float* scores, float* raw_out, void* ws, size_t ws_bytes, void* stream);
 
 /*
+ * Query-agnostic base scorer by key geometry, an alternative to vector_score for Step 1 (the
+ * paper names KeyDiff among the base scorers, Sections 3.2 and 5.1, "key geometric diversity",
+ * without a formula; this is the published idea): with the anchor a = sum_j k_j / ||k_j||,
+ * score_i = - <k_i, a> / (||k_i|| ||a||), in [-1, 1]; higher = less like the average key.  No
+ * observation window and no pooling (shape->window and pool_kernel are not used by this call, but
+ * vector_route still keeps shape->window <= n_pool).  A zero key scores 0.
+ * K: device [U][N][d]; scores: device fp32 [U][N].
+ */
+VECTOR_API vector_status vector_score_keydiff(const vector_shape* shape, const void* K, int64_t N,
+                                   float* scores, void* ws, size_t ws_bytes, void* stream);
+
+/*
  * Step 1, budget relaxation: per unit the n_pool largest scores, ties to the
  * lower index.  scores: device fp32 [U][N]; pool_idx: device [U][n_pool] ascending.
  */

@@ -137,6 +137,8 @@ def load_library() -> ctypes.CDLL:
     lib.vector_workspace_bytes.restype = SZ
     lib.vector_workspace_bytes.argtypes = [SP, BP]
     lib.vector_score.argtypes = [SP, P, P, I64, P, P, P, SZ, P]
+    lib.vector_score_keydiff.argtypes = [SP, P, I64, P, P, SZ, P]
+    lib.vector_score_keydiff.restype = ctypes.c_int
     lib.vector_pool_select.argtypes = [SP, BP, P, P, P, SZ, P]
     lib.vector_residual.argtypes = [SP, P, P, P, I64, P, I64, P, P]
     lib.vector_truncate.argtypes = [SP, BP, P, P, P, P, P, P, SZ, P]
@@ -246,6 +248,13 @@ def vector_score(shape: Shape, Q_obs, K, N: int, scores, raw_out=None, ws=None, 
                                      _dev(K, shape.torch_dtype, "K"), N, _dev(scores, torch.float32, "scores"),
                                      _dev(raw_out, torch.float32, "raw_out"), wp, wn, _stream(stream))
     _check(rc, "vector_score")
+
+
+def vector_score_keydiff(shape: Shape, K, N: int, scores, ws=None, stream=None):
+    wp, wn = _ws(ws)
+    rc = load_library().vector_score_keydiff(ctypes.byref(shape._c()), _dev(K, shape.torch_dtype, "K"), N,
+                                             _dev(scores, torch.float32, "scores"), wp, wn, _stream(stream))
+    _check(rc, "vector_score_keydiff")
 
 
 def vector_pool_select(shape: Shape, budget: Budget, scores, pool_idx, ws=None, stream=None):

@@ -275,8 +275,10 @@ size_t vector_workspace_bytes(const vector_shape* shape, const vector_budget* bu
     size_t a = vec::score_ws_bytes(D, budget->n_tokens, true);
     size_t b = vec::select_ws_bytes(D, *budget);
     size_t c = vec::decode_ws_bytes(D);
+    size_t k = vec::keydiff_ws_bytes(D, budget->n_tokens);
     size_t r = a > b ? a : b;
-    return (r > c ? r : c) + 256;
+    r = r > c ? r : c;
+    return (r > k ? r : k) + 256;
 }
 
 }  // extern "C"

@@ -49,6 +49,7 @@ int decode_num_splits(int U, int64_t rows);
 // Record slots per unit that the persistent bf16 decode kernel may use (two blocks per SM, 148 SMs).
 int decode_stream_slots(int U);
 size_t decode_ws_bytes(const Dims& D);
+size_t keydiff_ws_bytes(const Dims& D, int64_t N);
 
 inline size_t align256(size_t x) { return (x + 255) & ~size_t(255); }
 

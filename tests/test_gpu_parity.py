@@ -70,6 +70,51 @@ def test_score_parity(oracle, base, over):
     assert np.allclose(raw.double().sum(1).cpu().numpy(), mass, rtol=1e-4)
 
 
+KEYDIFF_CASES = [(0, {}), (0, {"N": 333}), (1, {"N": 1000, "n_kv_heads": 2, "n_q_heads": 8}),
+                 (1, {"N": 4096 + 77, "n_kv_heads": 1, "n_q_heads": 4}), (2, {"N": 1500, "n_layers": 20}),
+                 (1, {"N": 900, "head_dim": 64, "n_kv_heads": 1, "n_q_heads": 2}), (1, {"N": 1, "n_kv_heads": 1, "n_q_heads": 4})]
+
+
+@pytest.mark.parametrize("base,over", KEYDIFF_CASES)
+def test_keydiff_score_parity(oracle, base, over):
+    """Key-geometry scorer: cosines in [-1, 1] from fp32 sums over N rows against the fp64 oracle;
+    |g - o| <= 1e-3 max(|o|, 0.05)."""
+    wl = synth.shrink(synth.WORKLOADS[base], **over)
+    K, _, _ = synth.context(wl, DEV)
+    if wl.N > 10:
+        K[0, 7] = 0                                        # a zero key scores 0
+    sh = shape_of(wl)
+    ws = vec.alloc_workspace(sh, vec.vector_plan_budget(wl.N, wl.N, 0, min(wl.window, wl.N)))
+    scores = torch.full((wl.units, wl.N), float("nan"), dtype=torch.float32, device=DEV)
+    vec.vector_score_keydiff(sh, K, wl.N, scores, ws)
+    again = torch.empty_like(scores)
+    vec.vector_score_keydiff(sh, K, wl.N, again, ws)
+    torch.cuda.synchronize()
+    assert torch.equal(scores, again)                      # fixed reduction order: bitwise repeatable
+    got = scores.cpu().double().numpy()
+    for u in range(wl.units):
+        want = oracle.score_keydiff(K[u].cpu())
+        assert np.all(np.abs(got[u] - want) <= 1e-3 * np.maximum(np.abs(want), 0.05)), u
+    if wl.N > 10:
+        assert got[0, 7] == 0.0
+
+
+def test_keydiff_scores_drive_the_routing(oracle):
+    """The second base scorer feeds the same Steps 1-3: end-to-end agreement with the oracle run on its own scores."""
+    wl = synth.shrink(synth.WORKLOADS[1], N=2000, n_kv_heads=2, n_q_heads=8, n_calib=2048, window=8)
+    K, V, _ = synth.context(wl, DEV)
+    W = calibrated_maps(wl).to(DEV)
+    sh = shape_of(wl)
+    b = budget_of(wl, 30)
+    comp = Compressor(sh, b, keep_eps=True)
+    vec.vector_score_keydiff(sh, K, wl.N, comp.scores, comp.ws)
+    comp.route(K, V, W)
+    torch.cuda.synchronize()
+    sc_o = np.stack([oracle.score_keydiff(K[u].cpu()) for u in range(wl.units)])
+    _assert_routing_agrees(oracle, wl, b, comp, K, V, W.cpu(), sc_o, list(range(wl.units)))
+    assert torch.all((comp.tier == 1).sum(1) == b.n_apx) and torch.all((comp.tier == 2).sum(1) == b.n_ret)
+
+
 def _selection_inputs(U, N, seed, ties):
     g = torch.Generator().manual_seed(seed)
     s = torch.rand(U, N, generator=g)
