@@ -433,15 +433,13 @@ def test_decode_long_block_ranges(oracle):
             assert np.max(np.abs(out1[u].cpu().double().numpy() - o_tok)) <= 2e-2, (base, u, "per tile")
 
 
-def test_full_size_bench_configuration_sampled_units(oracle):
-    """Config 2 at full size in the launch shape the benchmark times; the oracle checks sampled units."""
-    wl = synth.WORKLOADS[2]
-    sample = [0, 131, 255]
-    # device pipeline over ALL 256 units; inputs of non-sampled units are the same law
+def _sampled_units_case(oracle, wl, percent, sample):
+    """Whole workload on the device in the launch shape the benchmark times; the oracle checks the
+    sampled units end to end, every unit is checked for the properties that hold at any size."""
     K, V, Q = synth.context(wl, DEV)
     W = calibrated_maps(wl).to(DEV)
     sh = shape_of(wl)
-    b = budget_of(wl, 20)
+    b = budget_of(wl, percent)
     comp = Compressor(sh, b, extra_rows=1, keep_eps=True)
     comp.compress(Q, K, V, W)
     torch.cuda.synchronize()
@@ -459,15 +457,34 @@ def test_full_size_bench_configuration_sampled_units(oracle):
     # sampled units against the oracle end to end
     class _View:            # the slice of the compressor state the agreement check reads
         tier = tier_all[sample]
+    LH = wl.n_layers * wl.n_kv_heads
+    Ws = torch.stack([W[u % LH] for u in sample]).cpu()
     sub = synth.shrink(wl, batch=1, n_layers=1, n_kv_heads=len(sample), n_q_heads=len(sample) * wl.group)
-    _assert_routing_agrees(oracle, sub, b, _View, K[sample], V[sample], W[sample].cpu(), sc_o, list(range(len(sample))))
+    _assert_routing_agrees(oracle, sub, b, _View, K[sample], V[sample], Ws, sc_o, list(range(len(sample))))
     _, sq, _ = synth.all_head_params(wl, DEV)
     q = synth.decode_q(wl, 0, DEV, sq)
     out = torch.empty(wl.units, wl.group, wl.head_dim, dtype=torch.float32, device=DEV)
     comp.decode(q, W, out)
     torch.cuda.synchronize()
+    assert vec.vector_device_fault() == 0
     c = comp.cache
-    for u in sample:
+    for j, u in enumerate(sample):
         _, o = oracle.attend(q[u].cpu(), c.ret_k[u, : c.n_ret].cpu(), c.ret_v[u, : c.n_ret].cpu(),
-                             c.apx_k[u, : c.n_apx].cpu(), W[u].cpu(), 1.0 / np.sqrt(wl.head_dim))
+                             c.apx_k[u, : c.n_apx].cpu(), Ws[j], 1.0 / np.sqrt(wl.head_dim))
         assert np.max(np.abs(out[u].cpu().double().numpy() - o)) <= 2e-2
+
+
+def test_full_size_bench_configuration_sampled_units(oracle):
+    """Config 2 at full size in the launch shape the benchmark times; the oracle checks sampled units."""
+    _sampled_units_case(oracle, synth.WORKLOADS[2], 20, [0, 131, 255])
+
+
+def test_config3_shape_sampled_units(oracle):
+    """Batched serving shape (config 3: N = 16384, budget 10 %, several sequences), cut to 2 sequences x 4 layers."""
+    _sampled_units_case(oracle, synth.shrink(synth.WORKLOADS[3], batch=2, n_layers=4), 10, [3, 40])
+
+
+def test_config4_shape_sampled_unit(oracle):
+    """Long-context shape (config 4: N = 131072, 8 query heads per KV head, window 128, budget 5 %), one layer;
+    the oracle scores one whole unit (1024 window rows x 131072 keys)."""
+    _sampled_units_case(oracle, synth.shrink(synth.WORKLOADS[4], n_layers=1), 5, [5])
