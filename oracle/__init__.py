@@ -200,6 +200,20 @@ def route(score_f32, K, V, W, n_pool: int, n_apx: int, rope: bool = False, theta
     return dict(tier=tier, ret_idx=ret, apx_idx=apx, eps=eps, pool_idx=pool)
 
 
+DIAG_FIELDS = ("E", "r2_approx", "mu_a", "sum_evicted_w", "sum_approximated_w", "w_bar", "w_star", "threshold")
+
+
+def diagnostics(importance, tier, K, V, W) -> dict:
+    """Distortion E, R^2 over the approximated set and the threshold of Proposition 1 for one routed unit."""
+    imp, K, V, W = _f64(importance), _f64(K), _f64(V), _f64(W)
+    t = np.ascontiguousarray(np.asarray(tier, dtype=np.uint8))
+    N, d = K.shape
+    out = np.empty(8, dtype=np.float64)
+    rc = lib().oracle_diagnostics(_p(imp), _p(t), _p(K), _p(V), _p(W), ctypes.c_int64(N), ctypes.c_int32(d), _p(out))
+    _check(rc, "diagnostics")
+    return dict(zip(DIAG_FIELDS, out.tolist()))
+
+
 def gather_rows(src, idx):
     """-> (rows [n_idx][d] float64, pos int32)."""
     src, idx = _f64(src), _i32(idx)

@@ -450,3 +450,66 @@ int oracle_attend(const double* q, int32_t g, int32_t d,
     free(p); free(kt); free(vh); free(acc);
     return ORACLE_OK;
 }
+
+
+/*
+ * Diagnostics of one routed unit (Section 4: the distortion measure E, R^2_approx and the
+ * threshold of Proposition 1).  importance: [N] non-negative weights w_i (normalised here to sum 1);
+ * tier: [N] 0 evicted / 1 approximated / 2 retained; K, V: [N][d]; W: [d][d] (y = W x).
+ *   E            = sum_{evicted} w_i + sum_{approximated} w_i ||v_i - W k_i||^2 / ||v_i||^2
+ *   mu_A         = mean over the approximated tokens of ||v_i - W k_i||^2 / ||v_i||^2
+ *   R2_approx    = 1 - mu_A
+ *   w_bar        = (1 - sum_{evicted} w_i) / (number of tokens kept in the pool)
+ *   w_star       = the largest weight among the evicted tokens (the token at the eviction boundary)
+ *   threshold    = w_bar / (w_star + w_bar)    (approximation pays off when R2_approx exceeds it)
+ * out[8] = { E, R2_approx, mu_A, sum_evicted_w, sum_approximated_w, w_bar, w_star, threshold }.
+ * A token with v = 0 counts a relative error of 0 when its residual is 0 too, else 1.
+ */
+int oracle_diagnostics(const double* importance, const uint8_t* tier, const double* K, const double* V,
+                       const double* W, int64_t N, int32_t d, double* out) {
+    if (!importance || !tier || !K || !V || !W || !out || N <= 0 || d <= 0) return ORACLE_ERR_ARG;
+    double total = 0.0;
+    for (int64_t i = 0; i < N; ++i) {
+        if (!(importance[i] >= 0.0) || isinf(importance[i])) return ORACLE_ERR_ARG;
+        total += importance[i];
+    }
+    if (!(total > 0.0)) return ORACLE_ERR_ARG;
+    double sum_e = 0.0, sum_a = 0.0, sum_a_rel = 0.0, mu = 0.0, w_star = 0.0;
+    int64_t n_a = 0, n_kept = 0;
+    for (int64_t i = 0; i < N; ++i) {
+        const double w = importance[i] / total;
+        if (tier[i] == 0) {
+            sum_e += w;
+            if (w > w_star) w_star = w;
+            continue;
+        }
+        ++n_kept;
+        if (tier[i] == 1) {
+            const double* k = K + i * d;
+            const double* v = V + i * d;
+            double r2 = 0.0, v2 = 0.0;
+            for (int c = 0; c < d; ++c) {
+                double pred = 0.0;
+                for (int j = 0; j < d; ++j) pred += W[(size_t)c * d + j] * k[j];
+                r2 += (v[c] - pred) * (v[c] - pred);
+                v2 += v[c] * v[c];
+            }
+            const double rel = v2 > 0.0 ? r2 / v2 : (r2 > 0.0 ? 1.0 : 0.0);
+            sum_a += w;
+            sum_a_rel += w * rel;
+            mu += rel;
+            ++n_a;
+        }
+    }
+    mu = n_a > 0 ? mu / (double)n_a : 0.0;
+    const double w_bar = n_kept > 0 ? (1.0 - sum_e) / (double)n_kept : 0.0;
+    out[0] = sum_e + sum_a_rel;
+    out[1] = 1.0 - mu;
+    out[2] = mu;
+    out[3] = sum_e;
+    out[4] = sum_a;
+    out[5] = w_bar;
+    out[6] = w_star;
+    out[7] = (w_star + w_bar) > 0.0 ? w_bar / (w_star + w_bar) : 0.0;
+    return ORACLE_OK;
+}

@@ -478,3 +478,34 @@ def test_keydiff_scorer_pins(oracle):
     K3 = K.copy(); K3[5] = 0.0
     assert oracle.score_keydiff(K3)[5] == 0.0
     assert np.all(oracle.score_keydiff(np.stack([k, -k])) == 0.0)
+
+
+def test_diagnostics_pins(oracle):
+    """Distortion measure and Proposition 1's threshold (Section 4) on cases worked by hand."""
+    rng = np.random.default_rng(5)
+    d = 8
+    K = rng.standard_normal((4, d)); Wm = rng.standard_normal((d, d)) / 3
+    w = np.array([0.4, 0.3, 0.2, 0.1])
+    tier = np.array([2, 1, 1, 0], dtype=np.uint8)          # retained, approximated x2, evicted
+    # exact reconstruction: approximated tokens cost nothing
+    r = oracle.diagnostics(w, tier, K, K @ Wm.T, Wm)
+    assert r["E"] == pytest.approx(0.1) and r["r2_approx"] == pytest.approx(1.0) and r["mu_a"] == pytest.approx(0.0, abs=1e-28)
+    assert r["sum_evicted_w"] == pytest.approx(0.1) and r["sum_approximated_w"] == pytest.approx(0.5)
+    assert r["w_bar"] == pytest.approx(0.9 / 3) and r["w_star"] == pytest.approx(0.1)
+    assert r["threshold"] == pytest.approx(0.3 / 0.4)      # w_bar / (w_star + w_bar) = 0.75
+    # a zero map reconstructs nothing: every approximated token counts like an evicted one
+    V = rng.standard_normal((4, d))
+    r0 = oracle.diagnostics(w, tier, K, V, np.zeros((d, d)))
+    assert r0["E"] == pytest.approx(0.1 + 0.5) and r0["r2_approx"] == pytest.approx(0.0) and r0["mu_a"] == pytest.approx(1.0)
+    # one approximated token with a residual of known relative size: v = W k + t * u with u orthogonal to W k
+    k = K[1]; p = Wm @ k
+    u = rng.standard_normal(d); u -= u @ p / (p @ p) * p; u *= np.linalg.norm(p) / np.linalg.norm(u)
+    V2 = K @ Wm.T; V2[1] = p + 0.5 * u                       # ||r||^2 / ||v||^2 = 0.25 / 1.25 = 0.2
+    r2 = oracle.diagnostics(w, tier, K, V2, Wm)
+    assert r2["mu_a"] == pytest.approx(0.1) and r2["E"] == pytest.approx(0.1 + 0.3 * 0.2)
+    # importance is normalised; no approximation tier -> E is the evicted mass; no eviction -> w_star = 0, threshold 1
+    assert oracle.diagnostics(7.0 * w, tier, K, V2, Wm) == pytest.approx(r2)
+    r3 = oracle.diagnostics(w, np.array([2, 2, 0, 0], dtype=np.uint8), K, V, Wm)
+    assert r3["E"] == pytest.approx(0.3) and r3["sum_approximated_w"] == 0.0 and r3["r2_approx"] == 1.0
+    r4 = oracle.diagnostics(w, np.array([2, 1, 1, 2], dtype=np.uint8), K, V2, Wm)
+    assert r4["w_star"] == 0.0 and r4["threshold"] == pytest.approx(1.0) and r4["w_bar"] == pytest.approx(0.25)
