@@ -226,6 +226,22 @@ VECTOR_API vector_status vector_decode_attn(const vector_shape* shape, const voi
                                  void* ws, size_t ws_bytes, void* stream);
 
 /*
+ * Diagnostics of a routed cache (paper Section 4: the distortion measure E, R^2_approx and the
+ * condition of Proposition 1).  importance: device fp32 [U][N], non-negative finite weights w_i,
+ * normalised per unit to sum 1 by the call (pass the un-pooled sums raw_out of vector_score; the
+ * pooled scores carry +inf for the window).  tier, pool_idx, eps: as written by vector_route
+ * (eps_out and pool_idx_out are needed).  V: device [U][N][d].  out: device fp32 [U][8] =
+ *   { E = sum_evicted w + sum_approx w ||v - W k||^2 / ||v||^2,  R2_approx = 1 - mu_A,
+ *     mu_A = mean relative reconstruction error over the approximated tokens,
+ *     sum of evicted w, sum of approximated w,  w_bar = (1 - sum evicted w) / n_pool,
+ *     w_star = largest evicted w,  threshold = w_bar / (w_star + w_bar) }.
+ * Approximation reduces the distortion when R2_approx > threshold (Proposition 1).
+ */
+VECTOR_API vector_status vector_diagnostics(const vector_shape* shape, const vector_budget* budget,
+                                 const float* importance, const uint8_t* tier, const int32_t* pool_idx,
+                                 const float* eps, const void* V, float* out /* [U][8] */, void* stream);
+
+/*
  * Allocation-free variant of vector_decode_attn (the paper has no counterpart:
  * this entry point exists for the integration, not for the method).
  *

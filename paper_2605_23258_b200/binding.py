@@ -144,6 +144,8 @@ def load_library() -> ctypes.CDLL:
     lib.vector_truncate.argtypes = [SP, BP, P, P, P, P, P, P, SZ, P]
     lib.vector_route.argtypes = [SP, BP, P, P, P, P, P, P, P, P, P, P, SZ, P]
     lib.vector_compact.argtypes = [SP, BP, P, P, P, P, CP, P]
+    lib.vector_diagnostics.argtypes = [SP, BP, P, P, P, P, P, P, P]
+    lib.vector_diagnostics.restype = ctypes.c_int
     lib.vector_decode_attn.argtypes = [SP, P, CP, P, P, I32, I32, P, SZ, P]
     lib.vector_decode_scratch_bytes.restype = SZ
     lib.vector_decode_scratch_bytes.argtypes = [SP]
@@ -292,6 +294,18 @@ def vector_route(shape: Shape, budget: Budget, scores, K, V, W, tier, ret_idx, a
                                      _dev(apx_idx, torch.int32, "apx_idx"), _dev(eps_out, torch.float32, "eps_out"),
                                      _dev(pool_idx_out, torch.int32, "pool_idx_out"), wp, wn, _stream(stream))
     _check(rc, "vector_route")
+
+
+DIAG_FIELDS = ("E", "r2_approx", "mu_a", "sum_evicted_w", "sum_approximated_w", "w_bar", "w_star", "threshold")
+
+
+def vector_diagnostics(shape: Shape, budget: Budget, importance, tier, pool_idx, eps, V, out, stream=None):
+    """out [U][8] fp32: the DIAG_FIELDS of every unit."""
+    rc = load_library().vector_diagnostics(ctypes.byref(shape._c()), ctypes.byref(budget._c()),
+                                           _dev(importance, torch.float32, "importance"), _dev(tier, torch.uint8, "tier"),
+                                           _dev(pool_idx, torch.int32, "pool_idx"), _dev(eps, torch.float32, "eps"),
+                                           _dev(V, shape.torch_dtype, "V"), _dev(out, torch.float32, "out"), _stream(stream))
+    _check(rc, "vector_diagnostics")
 
 
 def vector_compact(shape: Shape, budget: Budget, K, V, ret_idx, apx_idx, cache: Cache, stream=None):

@@ -115,6 +115,28 @@ def test_keydiff_scores_drive_the_routing(oracle):
     assert torch.all((comp.tier == 1).sum(1) == b.n_apx) and torch.all((comp.tier == 2).sum(1) == b.n_ret)
 
 
+def test_diagnostics_parity(oracle):
+    """Distortion E, R^2 over the approximated set and Proposition 1's threshold of a routed cache."""
+    wl = synth.shrink(synth.WORKLOADS[1], N=3000, n_kv_heads=2, n_q_heads=8, n_calib=2048)
+    K, V, Q = synth.context(wl, DEV)
+    W = calibrated_maps(wl).to(DEV)
+    sh = shape_of(wl)
+    b = budget_of(wl, 30)
+    comp = Compressor(sh, b, keep_eps=True)
+    raw = torch.empty(wl.units, wl.N, dtype=torch.float32, device=DEV)
+    vec.vector_score(sh, Q, K, wl.N, comp.scores, raw, comp.ws)
+    comp.route(K, V, W)
+    out = torch.empty(wl.units, 8, dtype=torch.float32, device=DEV)
+    vec.vector_diagnostics(sh, b, raw, comp.tier, comp.pool_idx, comp.eps, V, out)
+    torch.cuda.synchronize()
+    for u in range(wl.units):
+        want = oracle.diagnostics(raw[u].cpu(), comp.tier[u].cpu().numpy(), K[u].cpu(), V[u].cpu(), W[u].cpu())
+        got = dict(zip(vec.DIAG_FIELDS, out[u].cpu().double().tolist()))
+        for name in vec.DIAG_FIELDS:          # fp64 sums of fp32 residuals: the residual's own rounding dominates
+            assert got[name] == pytest.approx(want[name], rel=1e-4, abs=1e-7), (u, name, got[name], want[name])
+        assert 0.0 <= got["E"] <= 1.0 and got["mu_a"] < 0.5          # the approximated tokens are the reconstructable ones
+
+
 def _selection_inputs(U, N, seed, ties):
     g = torch.Generator().manual_seed(seed)
     s = torch.rand(U, N, generator=g)
