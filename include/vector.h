@@ -218,7 +218,11 @@ VECTOR_API vector_status vector_compact(const vector_shape* shape, const vector_
  * tokens are rebuilt as W k).  Per query head: p = softmax over the keys of both
  * pools jointly (logit = sm_scale * q.k), then
  *   mode 0 (factored):  o = sum_R p_i v_i + W (sum_A p_i k~_i)
- *   mode 1 (per tile):  o = sum_R p_i v_i + sum_A p_i (W k~_i)
+ *   mode 1 (per tile):  o = sum_R p_i v_i + sum_A p_i (W k~_i), W k formed tile by tile on the tensor
+ *                       cores; bf16, head_dim 128, rope off only (else VECTOR_ERR_UNSUPPORTED); about
+ *                       three times slower than mode 0, which gives the same sum by linearity
+ * With shape->rope_enabled, k~_i is the stored key turned back by cache->apx_pos (required then);
+ * the logit always uses the stored key.
  * q: device [U][g][d] of shape->dtype; out: device [U][g][d] of out_dtype.
  */
 VECTOR_API vector_status vector_decode_attn(const vector_shape* shape, const void* q, const vector_cache* cache,
