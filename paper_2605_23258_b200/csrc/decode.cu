@@ -203,25 +203,30 @@ static vector_status launch_decode(const Dims& dm, const void* q, const vector_c
 // Fault word that bounded waits inside kernels write to (0 = none).
 static __device__ int g_kernel_fault;
 int* kernel_fault_address() {
-    static int* addr = nullptr;           // single-device processes; looked up with the current device
-    if (!addr) {
+    static int* addr[PerDeviceOnce::kMax] = {};      // per device, looked up with that device current
+    static std::mutex mu;
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= PerDeviceOnce::kMax) return nullptr;
+    std::lock_guard<std::mutex> lock(mu);
+    if (!addr[dev]) {
         void* p = nullptr;
-        if (cudaGetSymbolAddress(&p, g_kernel_fault) == cudaSuccess) addr = (int*)p;
+        if (cudaGetSymbolAddress(&p, g_kernel_fault) == cudaSuccess) addr[dev] = (int*)p;
     }
-    return addr;
+    return addr[dev];
 }
 
 // bf16, head_dim 128: persistent TMA + tensor-core streaming kernel and the record merge.
 static vector_status launch_decode_bf16_d128(const Dims& dm, const void* q, const vector_cache* ch, const void* W,
                                              void* out, int out_dtype, int mode, float* partial, cudaStream_t st) {
     using T = __nv_bfloat16;
-    static bool configured = false;
-    if (!configured) {
-        VEC_CUDA_CHECK(cudaFuncSetAttribute(dbf::decode_stream_bf16_d128<false>,
-                                            cudaFuncAttributeMaxDynamicSharedMemorySize, dbf::SMEM_BYTES));
-        VEC_CUDA_CHECK(cudaFuncSetAttribute(dbf::decode_stream_bf16_d128<true>,
-                                            cudaFuncAttributeMaxDynamicSharedMemorySize, dbf::SMEM_BYTES_PER_TILE));
-        configured = true;
+    static PerDeviceOnce once;
+    if (once.first()) {
+        cudaError_t e = cudaFuncSetAttribute(dbf::decode_stream_bf16_d128<false>,
+                                             cudaFuncAttributeMaxDynamicSharedMemorySize, dbf::SMEM_BYTES);
+        if (e == cudaSuccess)
+            e = cudaFuncSetAttribute(dbf::decode_stream_bf16_d128<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                     dbf::SMEM_BYTES_PER_TILE);
+        if (e != cudaSuccess) { once.undo(); VEC_CUDA_CHECK(e); }
     }
     int* fault = kernel_fault_address();
     if (!fault) return VECTOR_ERR_CUDA;

@@ -1,7 +1,9 @@
 // Host-only entry points of libvector: status text, the tier planner and the
 // offline least-squares calibration, plus the argument checks the device entry
-// points share.  No CUDA calls in this file.
+// points share.  The only CUDA call in this file is cudaGetDevice.
 #include <cmath>
+#include <mutex>
+#include <cuda_runtime_api.h>
 #include <cstring>
 #include <vector>
 
@@ -11,6 +13,22 @@ namespace vec {
 
 static thread_local int g_last_cuda_error = 0;
 void set_last_cuda_error(int e) { g_last_cuda_error = e; }
+
+static std::mutex g_once_mu;
+bool PerDeviceOnce::first() {
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMax) return false;
+    std::lock_guard<std::mutex> lock(g_once_mu);
+    if (done[dev]) return false;
+    done[dev] = 1;
+    return true;
+}
+void PerDeviceOnce::undo() {
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMax) return;
+    std::lock_guard<std::mutex> lock(g_once_mu);
+    done[dev] = 0;
+}
 
 vector_status check_shape(const vector_shape* s, Dims* out) {
     if (!s || !out) return VECTOR_ERR_NULL;

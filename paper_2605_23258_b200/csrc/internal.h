@@ -41,8 +41,19 @@ size_t score_ws_bytes(const Dims& D, int64_t N, bool need_raw);
 struct ScoreTcPlan { int RG, nt, tpc, n_chunks, n_items; };
 ScoreTcPlan score_tc_plan(int U, int R, int64_t N);
 inline bool score_uses_tc(const Dims& D) { return D.dtype == VECTOR_BF16 && D.d == 128; }
-// Device address of the word in which bounded waits inside kernels record that they gave up.
+// Device address (on the current device) of the word in which bounded waits inside kernels record
+// that they gave up; NULL if it cannot be resolved.
 int* kernel_fault_address();
+
+// One-time set-up that has to happen once per device (kernel attributes are per device): returns true
+// the first time it is called with the current device for this flag set, false afterwards (and false,
+// doing nothing, if the device index is out of range).  Thread-safe.
+struct PerDeviceOnce {
+    static constexpr int kMax = 64;
+    unsigned char done[kMax] = {};
+    bool first();          // defined in host.cpp
+    void undo();           // the set-up failed: try again on the next call
+};
 size_t select_ws_bytes(const Dims& D, const vector_budget& b);
 // Number of key splits of one unit in decode attention for `rows` logical keys.
 int decode_num_splits(int U, int64_t rows);

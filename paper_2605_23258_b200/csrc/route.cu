@@ -283,10 +283,10 @@ static vector_status launch_residual(const Dims& dm, const void* K, const void* 
 static vector_status launch_residual_tc(const Dims& dm, const void* K, const void* V, const void* W, int64_t N,
                                         const int32_t* idx, int64_t n_idx, float* eps, cudaStream_t st) {
     if (n_idx == 0) return VECTOR_OK;
-    static bool configured = false;
-    if (!configured) {
-        VEC_CUDA_CHECK(cudaFuncSetAttribute(rtc::residual_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, rtc::SMEM_BYTES));
-        configured = true;
+    static PerDeviceOnce once;
+    if (once.first()) {
+        const cudaError_t e = cudaFuncSetAttribute(rtc::residual_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, rtc::SMEM_BYTES);
+        if (e != cudaSuccess) { once.undo(); VEC_CUDA_CHECK(e); }
     }
     int* fault = kernel_fault_address();
     if (!fault) return VECTOR_ERR_CUDA;

@@ -218,11 +218,12 @@ static vector_status launch_score_tc(const Dims& dm, const void* Q, const void* 
     float* lse2 = (float*)ws;
     ws += align256((size_t)dm.U * dm.R * sizeof(float));
     float* raw_part = (float*)ws;
-    static bool configured = false;
-    if (!configured) {
-        VEC_CUDA_CHECK(cudaFuncSetAttribute(stc::score_pass1_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, stc::SMEM_BYTES));
-        VEC_CUDA_CHECK(cudaFuncSetAttribute(stc::score_pass2_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, stc::SMEM_BYTES));
-        configured = true;
+    static PerDeviceOnce once;
+    if (once.first()) {
+        cudaError_t e = cudaFuncSetAttribute(stc::score_pass1_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, stc::SMEM_BYTES);
+        if (e == cudaSuccess)
+            e = cudaFuncSetAttribute(stc::score_pass2_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, stc::SMEM_BYTES);
+        if (e != cudaSuccess) { once.undo(); VEC_CUDA_CHECK(e); }
     }
     int* fault = kernel_fault_address();
     if (!fault) return VECTOR_ERR_CUDA;

@@ -96,6 +96,16 @@ def test_device_calls_validate_before_touching_the_gpu():
     # N shorter than the window; missing workspace
     assert lib.vector_score(ctypes.byref(sh), 1, 1, 16, 1, None, None, 0, None) == -2
     assert lib.vector_score(ctypes.byref(sh), 256, 256, 1024, 256, None, None, 0, None) == -5
+    # the second scorer, the diagnostics and the per-tile decode mode check their arguments the same way
+    assert lib.vector_score_keydiff(ctypes.byref(sh), None, 1024, None, None, 0, None) == -1
+    assert lib.vector_score_keydiff(ctypes.byref(sh), 256, 0, 256, None, 0, None) == -2
+    assert lib.vector_score_keydiff(ctypes.byref(sh), 256, 1024, 256, None, 0, None) == -5
+    assert lib.vector_diagnostics(ctypes.byref(sh), ctypes.byref(bu), *([None] * 6), None) == -1
+    c = binding._Cache(256, 256, 256, 256, 256, 8, 8, 4, 4)
+    assert lib.vector_decode_attn(ctypes.byref(sh), 256, ctypes.byref(c), 256, 256, 0, 1, 256, 1 << 30, None) == -9   # mode 1: bf16/128 only
+    assert lib.vector_decode_attn(ctypes.byref(sh), 256, ctypes.byref(c), 256, 256, 0, 2, 256, 1 << 30, None) == -2
+    rope = _shape(rope_enabled=1, rope_theta=0.5)
+    assert lib.vector_score(ctypes.byref(rope._c()), 1, 1, 1024, 1, None, None, 0, None) == -2                   # theta must exceed 1
     # inconsistent budget
     bad_b = vec.Budget(1024, 256, 128, 999, 256, 128, 640)._c()
     assert lib.vector_pool_select(ctypes.byref(sh), ctypes.byref(bad_b), 256, 256, None, 0, None) == -4
