@@ -146,6 +146,7 @@ decode_stream_bf16_d128(const __nv_bfloat16* __restrict__ q, const __grid_consta
         // ------------------------------------------------------------------ producer
         if (lane == 0) {
             tma::prefetch_map(&maps.ret_k); tma::prefetch_map(&maps.ret_v); tma::prefetch_map(&maps.apx_k);
+            const uint64_t pol = tma::policy_evict_first();      // the cache is read once per step
             int u = u0, t = t0;
             for (int i = 0; i < n_my; ++i) {
                 const int s = i % SLOTS, round = i / SLOTS;
@@ -154,16 +155,16 @@ decode_stream_bf16_d128(const __nv_bfloat16* __restrict__ q, const __grid_consta
                 tma::mbar_expect_tx(&full_bar[s], SLOT_BYTES);
                 if (t < pl.n_rt) {
                     const int row0 = t * KEYS;
-                    tma::load_3d(st, &maps.ret_k, 0, row0, u, &full_bar[s]);
-                    tma::load_3d(st + BOX_BYTES, &maps.ret_k, 64, row0, u, &full_bar[s]);
-                    tma::load_3d(st + HALF_BYTES, &maps.ret_v, 0, row0, u, &full_bar[s]);
-                    tma::load_3d(st + HALF_BYTES + BOX_BYTES, &maps.ret_v, 64, row0, u, &full_bar[s]);
+                    tma::load_3d_hint(st, &maps.ret_k, 0, row0, u, &full_bar[s], pol);
+                    tma::load_3d_hint(st + BOX_BYTES, &maps.ret_k, 64, row0, u, &full_bar[s], pol);
+                    tma::load_3d_hint(st + HALF_BYTES, &maps.ret_v, 0, row0, u, &full_bar[s], pol);
+                    tma::load_3d_hint(st + HALF_BYTES + BOX_BYTES, &maps.ret_v, 64, row0, u, &full_bar[s], pol);
                 } else {
                     const int row0 = (t - pl.n_rt) * 2 * KEYS;
-                    tma::load_3d(st, &maps.apx_k, 0, row0, u, &full_bar[s]);
-                    tma::load_3d(st + BOX_BYTES, &maps.apx_k, 64, row0, u, &full_bar[s]);
-                    tma::load_3d(st + HALF_BYTES, &maps.apx_k, 0, row0 + KEYS, u, &full_bar[s]);
-                    tma::load_3d(st + HALF_BYTES + BOX_BYTES, &maps.apx_k, 64, row0 + KEYS, u, &full_bar[s]);
+                    tma::load_3d_hint(st, &maps.apx_k, 0, row0, u, &full_bar[s], pol);
+                    tma::load_3d_hint(st + BOX_BYTES, &maps.apx_k, 64, row0, u, &full_bar[s], pol);
+                    tma::load_3d_hint(st + HALF_BYTES, &maps.apx_k, 0, row0 + KEYS, u, &full_bar[s], pol);
+                    tma::load_3d_hint(st + HALF_BYTES + BOX_BYTES, &maps.apx_k, 64, row0 + KEYS, u, &full_bar[s], pol);
                 }
                 if (++t == pl.n_tiles) { t = 0; ++u; }
             }
