@@ -8,6 +8,7 @@
 //   split  grid (n_splits, U): online softmax over a slice of the logical key
 //          range [0, n_ret + n_apx); emits (m, l, acc_v[d], acc_k[d]) per head
 //   merge  grid (U): combines the splits, applies W to acc_k, normalises
+#include <cmath>
 #include <mutex>
 
 #include "common.cuh"
@@ -221,10 +222,13 @@ static vector_status launch_decode_bf16_d128(const Dims& dm, const void* q, cons
     using T = __nv_bfloat16;
     static PerDeviceOnce once;
     if (once.first()) {
-        cudaError_t e = cudaFuncSetAttribute(dbf::decode_stream_bf16_d128<false>,
+        cudaError_t e = cudaFuncSetAttribute(dbf::decode_stream_bf16_d128<false, false>,
                                              cudaFuncAttributeMaxDynamicSharedMemorySize, dbf::SMEM_BYTES);
         if (e == cudaSuccess)
-            e = cudaFuncSetAttribute(dbf::decode_stream_bf16_d128<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+            e = cudaFuncSetAttribute(dbf::decode_stream_bf16_d128<false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                     dbf::SMEM_BYTES);
+        if (e == cudaSuccess)
+            e = cudaFuncSetAttribute(dbf::decode_stream_bf16_d128<true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                      dbf::SMEM_BYTES_PER_TILE);
         if (e != cudaSuccess) { once.undo(); VEC_CUDA_CHECK(e); }
     }
@@ -249,12 +253,24 @@ static vector_status launch_decode_bf16_d128(const Dims& dm, const void* q, cons
     if (ch->n_ret == 0) { maps.ret_k = maps.apx_k; maps.ret_v = maps.apx_k; }   // never dereferenced: no such tiles
     if (ch->n_apx == 0) maps.apx_k = maps.ret_k;
     const float c2 = dm.scale * 1.4426950408889634f;
+    dbf::RopePhases ph = {};
+    if (dm.rope) {
+        // turns per position of channel pair c, theta^(-2c/128) / (2 pi), as a 64-bit fraction
+        for (int c = 0; c < 64; ++c) {
+            const long double f = powl((long double)dm.theta, -2.0L * c / 128.0L) / 6.283185307179586476925286766559L;
+            ph.phase[c] = (unsigned long long)ldexpl(f - floorl(f), 64);
+        }
+    }
     if (mode == 1)
-        dbf::decode_stream_bf16_d128<true><<<pl.B, dbf::THREADS, dbf::SMEM_BYTES_PER_TILE, st>>>(
-            (const T*)q, maps, pl, (int)ch->n_ret, (int)ch->n_apx, dm.g, dm.LH, c2, partial, fault);
+        dbf::decode_stream_bf16_d128<true, false><<<pl.B, dbf::THREADS, dbf::SMEM_BYTES_PER_TILE, st>>>(
+            (const T*)q, maps, pl, (int)ch->n_ret, (int)ch->n_apx, dm.g, dm.LH, c2, partial, fault, nullptr, 0, ph);
+    else if (dm.rope)
+        dbf::decode_stream_bf16_d128<false, true><<<pl.B, dbf::ROPE_THREADS, dbf::SMEM_BYTES, st>>>(
+            (const T*)q, maps, pl, (int)ch->n_ret, (int)ch->n_apx, dm.g, dm.LH, c2, partial, fault, ch->apx_pos,
+            (long long)ch->cap_apx, ph);
     else
-        dbf::decode_stream_bf16_d128<false><<<pl.B, dbf::THREADS, dbf::SMEM_BYTES, st>>>(
-            (const T*)q, maps, pl, (int)ch->n_ret, (int)ch->n_apx, dm.g, dm.LH, c2, partial, fault);
+        dbf::decode_stream_bf16_d128<false, false><<<pl.B, dbf::THREADS, dbf::SMEM_BYTES, st>>>(
+            (const T*)q, maps, pl, (int)ch->n_ret, (int)ch->n_apx, dm.g, dm.LH, c2, partial, fault, nullptr, 0, ph);
     VEC_LAUNCH_CHECK();
     // programmatic dependent launch: the merge blocks start while the streaming kernel drains
     cudaLaunchAttribute attr;
@@ -314,9 +330,7 @@ extern "C" vector_status vector_decode_attn(const vector_shape* shape, const voi
         return dm.d == 64 ? launch_decode_g<float, 64>(dm, q, cache, W, out, out_dtype, partial, st)
                           : launch_decode_g<float, 128>(dm, q, cache, W, out, out_dtype, partial, st);
     if (dm.d == 64) return launch_decode_g<__nv_bfloat16, 64>(dm, q, cache, W, out, out_dtype, partial, st);
-    // the de-rotating variant exists on the CUDA-core path only
-    return dm.rope ? launch_decode_g<__nv_bfloat16, 128>(dm, q, cache, W, out, out_dtype, partial, st)
-                   : launch_decode_bf16_d128(dm, q, cache, W, out, out_dtype, mode, partial, st);
+    return launch_decode_bf16_d128(dm, q, cache, W, out, out_dtype, mode, partial, st);
 }
 
 // ---------------------------------------------------------------------------

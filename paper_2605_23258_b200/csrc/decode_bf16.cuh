@@ -23,6 +23,11 @@
 // key-only step the warp first forms V^T = W K^T for its 64 keys on the tensor cores (W of the unit in
 // shared memory, 512 MMAs), then accumulates O^T += V^T P^T with V^T and P split into bf16 hi + lo; the
 // merge step then adds that part without applying W.
+// RoPE decoupling (ROPE): the value of a key-only token is W applied to the key turned back by its
+// original position.  The logits use the stored keys; before the P K product the warp rotates its 64
+// keys in shared memory, channel c with c + 64 by the angle -pos * theta^(-2c/128).  The angle is
+// taken exactly modulo one turn in 64-bit fixed point (pos * phase[c] wraps by itself), its sine and
+// cosine by the fast units.
 // A warp keeps one running state (m, l, O or A) per unit and writes it as its
 // partial record when it leaves the unit; a warp that met no tile of a unit the
 // block touches writes an empty record.  The merge kernel combines a unit's
@@ -43,6 +48,13 @@ constexpr int HALF_BYTES = 16384;            // 64 rows of 256 B as two swizzled
 constexpr int BOX_BYTES = 8192;              // 64 rows x 128 bytes
 constexpr int CONSUMER_WARPS = 3;
 constexpr int THREADS = 32 * (CONSUMER_WARPS + 1);
+// With RoPE decoupling the block carries helper warps that turn a tile's keys back for the warp
+// that owns the tile: a team is that warp plus four helpers (warps 4 + 4 team .. 7 + 4 team), one
+// per warp scheduler (scheduler = warp index modulo 4), since the sine / cosine unit is per scheduler.
+constexpr int ROPE_HELPERS = 4;
+constexpr int ROPE_THREADS = 32 * (CONSUMER_WARPS + 1 + ROPE_HELPERS * CONSUMER_WARPS);
+constexpr int ROPE_TEAM_THREADS = 32 * (1 + ROPE_HELPERS);
+static_assert(CONSUMER_WARPS + 1 == 4 && ROPE_HELPERS == 4, "register hand-over is per warpgroup: owners + producer, then helpers");
 constexpr int REC = 4 + 2 * 128;             // m, l, value-scale, pad, acc_v[128], acc_k[128]
 constexpr int SMEM_BYTES = SLOTS * SLOT_BYTES + 1024;   // + alignment slack; barriers live in static smem
 constexpr int W_BYTES = 32768;               // the unit's map as two swizzled 128 x 128 B boxes (per-tile form only)
@@ -102,7 +114,77 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
     return *reinterpret_cast<uint32_t*>(&v);
 }
 
+// RoPE decoupling: rows 16 member .. 16 member + 15 of the 64 keys at kbase (two swizzled boxes:
+// channels 0-63 | 64-127) are turned back by their positions, in place.  Channel c pairs with
+// c + 64; the angle is position * theta^(-2c/128), taken as the top bits of the 64-bit product of
+// the position and the per-channel phase, so that it is exact modulo one turn.  pos16: lane l
+// holds the position of row 16 member + (l & 15).
+__device__ __forceinline__ void derotate_rows(uint32_t kbase, int nrows, int member, uint32_t pos16,
+                                              const unsigned long long* phase_s, int lane) {
+    const int qc = lane & 7;                                        // 16-byte chunk: channel pairs 8 qc .. 8 qc + 7
+    const uint2* phase2 = reinterpret_cast<const uint2*>(phase_s) + qc * 8;     // (low, high) words
+#pragma unroll 1
+    for (int j = 0; j < 4; j += 2) {
+        // two rows per round, the loads of both ahead of the stores
+        uint32_t off[2], pos[2], xs[2][4], ys[2][4];
+        bool live[2];
+#pragma unroll
+        for (int u = 0; u < 2; ++u) {
+            const int rl = 4 * (j + u) + (lane >> 3), r = 16 * member + rl;
+            pos[u] = __shfl_sync(0xffffffffu, pos16, rl);
+            live[u] = r < nrows;
+            off[u] = (uint32_t)r * 128u + (uint32_t)((qc ^ (r & 7)) << 4);
+            if (live[u]) {
+                asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];\n" : "=r"(xs[u][0]), "=r"(xs[u][1]), "=r"(xs[u][2]), "=r"(xs[u][3]) : "r"(kbase + off[u]));
+                asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];\n" : "=r"(ys[u][0]), "=r"(ys[u][1]), "=r"(ys[u][2]), "=r"(ys[u][3]) : "r"(kbase + BOX_BYTES + off[u]));
+            } else {
+#pragma unroll
+                for (int e = 0; e < 4; ++e) { xs[u][e] = 0u; ys[u][e] = 0u; }
+            }
+        }
+#pragma unroll
+        for (int u = 0; u < 2; ++u) {
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                float xo[2], yo[2];
+#pragma unroll
+                for (int h = 0; h < 2; ++h) {
+                    const float x = __uint_as_float(h ? (xs[u][e] & 0xffff0000u) : (xs[u][e] << 16));
+                    const float y = __uint_as_float(h ? (ys[u][e] & 0xffff0000u) : (ys[u][e] << 16));
+                    // top 32 bits of pos * phase modulo 2^64 (pos < 2^32): turns modulo 1, half a turn ahead
+                    const uint2 f = phase2[2 * e + h];
+                    const uint32_t turns = pos[u] * f.y + __umulhi(pos[u], f.x) + 0x80000000u;
+                    // its top 23 bits as a float in [1, 2); minus 1.5 is the turn count in [-0.5, 0.5)
+                    const float ang = fmaf(__uint_as_float((turns >> 9) | 0x3f800000u), 6.283185307179586f, -9.42477796076938f);
+                    float sn, cs;
+                    __sincosf(ang, &sn, &cs);
+                    xo[h] = fmaf(x, cs, y * sn);
+                    yo[h] = fmaf(y, cs, -x * sn);
+                }
+                xs[u][e] = pack_bf16(xo[0], xo[1]);
+                ys[u][e] = pack_bf16(yo[0], yo[1]);
+            }
+        }
+#pragma unroll
+        for (int u = 0; u < 2; ++u) {
+            if (live[u]) {
+                asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};\n" ::"r"(kbase + off[u]), "r"(xs[u][0]), "r"(xs[u][1]), "r"(xs[u][2]), "r"(xs[u][3]) : "memory");
+                asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};\n" ::"r"(kbase + BOX_BYTES + off[u]), "r"(ys[u][0]), "r"(ys[u][1]), "r"(ys[u][2]), "r"(ys[u][3]) : "memory");
+            }
+        }
+    }
+    // the slot is refilled by a bulk copy once released: order these stores ahead of it
+    asm volatile("fence.proxy.async.shared::cta;\n" ::: "memory");
+}
+// All threads of team `team` (its owner warp and the helpers).
+__device__ __forceinline__ void team_sync(int team) {
+    asm volatile("bar.sync %0, %1;\n" ::"r"(2 + team), "n"(ROPE_TEAM_THREADS) : "memory");
+}
+
 static_assert(SLOTS % CONSUMER_WARPS == 0, "a slot must always be consumed by the same warp");
+
+// phase[c] = frac(theta^(-2c/128) / (2 pi)) * 2^64, c < 64: turns per position, as a 64-bit fraction.
+struct RopePhases { unsigned long long phase[64]; };
 
 struct Maps {
     CUtensorMap ret_k, ret_v, apx_k;     // rank 3: (128 dims, pool rows, U units), box 64 x 64 x 1, 128B swizzle
@@ -111,12 +193,16 @@ struct Maps {
 
 // grid (plan.B), THREADS threads, SMEM_BYTES dynamic shared memory.
 // partial: [U][s_max][CONSUMER_WARPS][g][REC]; slot of (unit u, block b) = b - block_of_tile(first tile of u).
-template <bool PER_TILE>
-__global__ void __launch_bounds__(THREADS, 1)
+template <bool PER_TILE, bool ROPE>
+__global__ void __launch_bounds__(ROPE ? ROPE_THREADS : THREADS, 1)
 decode_stream_bf16_d128(const __nv_bfloat16* __restrict__ q, const __grid_constant__ Maps maps, Plan pl, int n_ret,
                         int n_apx, int g, int LH, float scale_log2e, float* __restrict__ partial,
-                        int* __restrict__ fault) {
+                        int* __restrict__ fault, const int32_t* __restrict__ apx_pos, long long cap_apx,
+                        const __grid_constant__ RopePhases rope) {
     extern __shared__ unsigned char smem_raw[];
+    __shared__ unsigned long long phase_s[ROPE ? 64 : 1];
+    if (ROPE && threadIdx.x < 64) phase_s[threadIdx.x] = rope.phase[threadIdx.x];
+    __shared__ volatile int team_ok[CONSUMER_WARPS];     // RoPE: the owner's go / no-go for the tile at hand
     __shared__ __align__(8) uint64_t full_bar[SLOTS];
     __shared__ __align__(8) uint64_t empty_bar[SLOTS];
     __shared__ __align__(8) uint64_t w_bar;
@@ -142,6 +228,42 @@ decode_stream_bf16_d128(const __nv_bfloat16* __restrict__ q, const __grid_consta
     }
     __syncthreads();
 
+    if (ROPE && wq > CONSUMER_WARPS) {
+        // ------------------------------------------------------------------ helpers (RoPE only)
+        // A helper walks its owner's key-only tiles and turns back its quarter of each 64 keys
+        // between the owner's two team barriers.  It waits on nothing but those barriers, which the
+        // owner reaches for every key-only tile whether or not its own (bounded) waits succeeded.
+        // The block is compiled for 128 registers a thread (512 threads): the three helper
+        // warpgroups hand registers over to the first one (the three owners and the producer).
+        asm volatile("setmaxnreg.dec.sync.aligned.u32 96;\n");
+        const int team = (wq - CONSUMER_WARPS - 1) / ROPE_HELPERS, member = (wq - CONSUMER_WARPS - 1) % ROPE_HELPERS;
+        int i = team;
+        for (int u = u0; u <= u_last; ++u) {
+            const long long unit_end = (long long)(u + 1) * pl.n_tiles - gt_lo;
+            for (; i < n_my && i < unit_end; i += CONSUMER_WARPS) {
+                const int t = (int)(gt_lo + i - (long long)u * pl.n_tiles);
+                if (t < pl.n_rt) continue;
+                const int r0 = (t - pl.n_rt) * 2 * KEYS;
+                const int32_t* pr = apx_pos + (size_t)u * cap_apx + r0 + 16 * member + (lane & 15);
+                const int n0 = min(KEYS, n_apx - r0), n1 = min(KEYS, n_apx - r0 - KEYS);      // n1 <= 0: no second half
+                const uint32_t p0 = 16 * member + (lane & 15) < n0 ? (uint32_t)__ldg(pr) : 0u;
+                const uint32_t p1 = 16 * member + (lane & 15) < n1 ? (uint32_t)__ldg(pr + KEYS) : 0u;
+                team_sync(team);                                   // the owner has published its verdict
+                if (!team_ok[team]) continue;
+                const uint32_t base = tma::smem_u32(smem + (i % SLOTS) * SLOT_BYTES);
+                team_sync(team);                                   // the owner has its scores of half 0
+                derotate_rows(base, n0, member, p0, phase_s, lane);
+                team_sync(team);                                   // ... and of half 1, if there is one
+                if (n1 > 0) {
+                    derotate_rows(base + HALF_BYTES, n1, member, p1, phase_s, lane);
+                    team_sync(team);
+                }
+            }
+        }
+        return;
+    }
+
+    if (ROPE) asm volatile("setmaxnreg.inc.sync.aligned.u32 216;\n");
     if (wq == CONSUMER_WARPS) {
         // ------------------------------------------------------------------ producer
         if (lane == 0) {
@@ -171,7 +293,6 @@ decode_stream_bf16_d128(const __nv_bfloat16* __restrict__ q, const __grid_consta
         }
         return;      // the consumers wait on every tile's full barrier, so no copy outlives the block
     }
-
     // ---------------------------------------------------------------------- consumers
     const int gid = lane >> 2, tig = lane & 3;
     // per-lane ldmatrix geometry (swizzle: 16-byte chunk index XOR (row & 7), rows are 128 bytes)
@@ -237,10 +358,12 @@ decode_stream_bf16_d128(const __nv_bfloat16* __restrict__ q, const __grid_consta
         zero_acc();
         m = -INFINITY; l = 0.f; stash_scale = 1.f; stashed = false;
     };
-    // 64 keys at kbase (two swizzled boxes), "values" at vbase (the keys themselves for a key-only tile).
-    auto step64 = [&](uint32_t kbase, uint32_t vbase, int nrows, bool retained, int unit) {
+    // One softmax step over the 64 keys at kbase (two swizzled boxes), in two parts.  The first
+    // leaves the step's weights p in sc (this thread: head gid, keys 8 n + 2 tig, + 1), brings m, l
+    // and the accumulators to the new running maximum and returns the factor it applied to them.
+    auto scores64 = [&](uint32_t kbase, int nrows, bool retained, int unit, float (&sc)[8][2]) -> float {
         // ---- S = Q K^T: eight 8-key column tiles, each its own accumulator chain over the 8 k-steps
-        float sc[8][2], zz[2];
+        float zz[2];
 #pragma unroll
         for (int n = 0; n < 8; ++n) { sc[n][0] = 0.f; sc[n][1] = 0.f; }
 #pragma unroll
@@ -294,6 +417,10 @@ decode_stream_bf16_d128(const __nv_bfloat16* __restrict__ q, const __grid_consta
                 for (int n = 0; n < 16; ++n) { acc[n][0] *= alpha; acc[n][1] *= alpha; acc[n][2] *= alpha; acc[n][3] *= alpha; }
             }
         }
+        return alpha;
+    };
+    // The second part adds p x (the 64 rows at vbase: values, or the keys themselves for a key-only tile).
+    auto accumulate64 = [&](uint32_t vbase, bool retained, float (&sc)[8][2]) {
         if (PER_TILE && !retained) {
             // ---- P^T as B operands (k = keys, n = heads), bf16 hi and lo, per 16-key k-step
             uint32_t pb_hi[4][2], pb_lo[4][2];
@@ -328,7 +455,7 @@ decode_stream_bf16_d128(const __nv_bfloat16* __restrict__ q, const __grid_consta
 #pragma unroll
                     for (int j = 0; j < 4; ++j) {
                         uint32_t b0, b1, b2, b3;
-                        ldsm_x4(kbase + (ks >> 2) * BOX_BYTES + j * 16 * 128 + qk_row + ((((2 * ks) & 7) << 4) ^ qk_x), b0, b1, b2, b3);
+                        ldsm_x4(vbase + (ks >> 2) * BOX_BYTES + j * 16 * 128 + qk_row + ((((2 * ks) & 7) << 4) ^ qk_x), b0, b1, b2, b3);
 #pragma unroll
                         for (int i = 0; i < 2; ++i) {
                             mma_16(vt[i][2 * j], wa[i][0], wa[i][1], wa[i][2], wa[i][3], b0, b1);
@@ -389,6 +516,31 @@ decode_stream_bf16_d128(const __nv_bfloat16* __restrict__ q, const __grid_consta
         }
     };
 
+    auto step64 = [&](uint32_t kbase, uint32_t vbase, int nrows, bool retained, int unit) {
+        float sc[8][2];
+        scores64(kbase, nrows, retained, unit, sc);
+        accumulate64(vbase, retained, sc);
+    };
+    // A key-only tile under RoPE decoupling.  The scores come from the keys as stored, the key sum
+    // wants them without the rotation: the helpers turn each half back between the two uses, and
+    // the owner forms the second half's scores (then the first half's sum) in the meantime.
+    auto rope_tile = [&](uint32_t base, int n0, int n1, int unit) {
+        float sc0[8][2], sc1[8][2];
+        scores64(base, n0, false, unit, sc0);
+        team_sync(wq);                         // every lane is past its last read of half 0 as stored
+        if (n1 > 0) {
+            const float alpha = scores64(base + HALF_BYTES, n1, false, unit, sc1);
+#pragma unroll
+            for (int n = 0; n < 8; ++n) { sc0[n][0] *= alpha; sc0[n][1] *= alpha; }     // the sums moved to the new maximum
+        }
+        team_sync(wq);                         // half 0 is turned back (and half 1 is free to be)
+        accumulate64(base, false, sc0);
+        if (n1 > 0) {
+            team_sync(wq);                     // half 1 is turned back
+            accumulate64(base + HALF_BYTES, false, sc1);
+        }
+    };
+
     zero_acc();
     // Walk the units the block touches; this warp owns the block's tiles i with i % CONSUMER_WARPS == wq.
     int i = wq;                                        // index into the block's tile sequence
@@ -408,19 +560,29 @@ decode_stream_bf16_d128(const __nv_bfloat16* __restrict__ q, const __grid_consta
         const long long unit_end = (long long)(u + 1) * pl.n_tiles - gt_lo;     // first sequence index past the unit
         bool loaded = false;
         for (; i < n_my && i < unit_end; i += CONSUMER_WARPS) {
-            if (!ok) continue;
-            if (!loaded) { load_q(u); loaded = true; }
             const int s = i % SLOTS, round = i / SLOTS;
             const int t = (int)(gt_lo + i - (long long)u * pl.n_tiles);
-            ok = tma::mbar_wait_warp(&full_bar[s], round & 1, fault, 2);
+            if (ok) {
+                if (!loaded) { load_q(u); loaded = true; }
+                ok = tma::mbar_wait_warp(&full_bar[s], round & 1, fault, 2);
+            }
+            if (ROPE && t >= pl.n_rt) {        // tell the helpers whether this key-only tile is worked on
+                if (lane == 0) team_ok[wq] = ok ? 1 : 0;
+                team_sync(wq);
+            }
             if (!ok) continue;
             const uint32_t base = tma::smem_u32(smem + s * SLOT_BYTES);
             if (t < pl.n_rt) {
                 step64(base, base + HALF_BYTES, min(KEYS, n_ret - t * KEYS), true, u);
             } else {
                 const int r0 = (t - pl.n_rt) * 2 * KEYS;
-                step64(base, base, min(KEYS, n_apx - r0), false, u);
-                if (n_apx - r0 > KEYS) step64(base + HALF_BYTES, base + HALF_BYTES, min(KEYS, n_apx - r0 - KEYS), false, u);
+                if (ROPE) {
+                    rope_tile(base, min(KEYS, n_apx - r0), min(KEYS, n_apx - r0 - KEYS), u);
+                } else {
+                    step64(base, base, min(KEYS, n_apx - r0), false, u);
+                    if (n_apx - r0 > KEYS)
+                        step64(base + HALF_BYTES, base + HALF_BYTES, min(KEYS, n_apx - r0 - KEYS), false, u);
+                }
             }
             __syncwarp();
             if (lane == 0) tma::mbar_arrive(&empty_bar[s]);
