@@ -373,6 +373,36 @@ def main():
                "tokens_per_s": wl.batch * N / (kd_ms * 1e-3)}
     del kd_scores
 
+    # ---- RoPE decoupling (the stored keys taken as post-RoPE: the residual and the reconstruction
+    #      turn them back by position), outside the timed step; same shapes, same budget
+    rope = None
+    if wl.dtype == "bf16" and d == 128:
+        import dataclasses
+        shape_r = dataclasses.replace(shape, rope_enabled=1, rope_theta=500000.0)
+        comp_r = Compressor(shape_r, budget)
+        comp_r.compress(Qt, Kt, Vt, Wm)
+        for _ in range(2):
+            comp_r.route(Kt, Vt, Wm)
+        a, b_ = ev(), ev()
+        torch.cuda.synchronize(); a.record()
+        for _ in range(5):
+            comp_r.route(Kt, Vt, Wm)
+        b_.record(); torch.cuda.synchronize()
+        r_ms = a.elapsed_time(b_) / 5
+        for _ in range(3):
+            comp_r.decode(qs[0], Wm, out)
+        a, b_ = ev(), ev()
+        torch.cuda.synchronize(); a.record()
+        for i in range(10):
+            comp_r.decode(qs[i % n_q], Wm, out)
+        b_.record(); torch.cuda.synchronize()
+        us = a.elapsed_time(b_) * 1e3 / 10
+        step_bytes = U * (2 * n_ret + n_apx) * d * es
+        rope = {"theta": 500000.0, "route_ms": r_ms, "route_gbs": (resid_bytes + U * N * 4 * 2) / (r_ms * 1e-3) / 1e9,
+                "decode_us_per_step": us, "decode_gbs": step_bytes / us / 1e3,
+                "sincos_per_decode_step": 2.0 * U * n_apx * (d // 2), "sincos_per_route": 2.0 * U * n_pool * (d // 2)}
+        del comp_r
+
     # ---- end to end through host buffers (rank 0 semantics on every rank; reported from rank 0)
     e2e = None
     if not args.no_e2e:
@@ -452,7 +482,7 @@ def main():
         "decode": {"gbs": decode_bytes / (dec_ms_max * 1e-3) / 1e9, "frac_of_measured_copy": decode_bytes / (dec_ms_max * 1e-3) / 1e9 / hbm,
                    "frac_of_8tbs": decode_bytes / (dec_ms_max * 1e-3) / 1e9 / 8000.0, "us_per_step": dec_ms_max * 1e3 / D,
                    "tokens_per_s": world * wl.batch * D / (dec_ms_max * 1e-3), "bytes_per_step": decode_bytes / D},
-        "decode_per_tile": per_tile, "score_keydiff": keydiff, "roofline": roofline, "roofline_kernels": kernels, "cpu_baseline": cpu, "e2e": e2e,
+        "decode_per_tile": per_tile, "score_keydiff": keydiff, "rope_decoupled": rope, "roofline": roofline, "roofline_kernels": kernels, "cpu_baseline": cpu, "e2e": e2e,
         "gpu_launches": kernels_per_step * K_steps, "clocks": clocks,
     }
     print(json.dumps(line))

@@ -42,6 +42,15 @@ __device__ __forceinline__ void rope_cos_sin(double pos, double inv_freq, float&
     const double r = fma(-n, 6.283185307179586, ang);
     sincosf((float)r, &sn, &cs);
 }
+// The same for the tuned kernels, from the pair's 64-bit phase (turns per position as a fraction
+// of 2^64, f = its low and high words): the top 32 bits of pos * phase modulo 2^64 are the angle
+// in turns modulo one, exact to 2^-32 of a turn for any 32-bit position; its top 23 bits make a
+// float in [1, 2), shifted by half a turn so that the result lies in [-pi, pi).
+__device__ __forceinline__ void rope_phase_cos_sin(uint32_t pos, uint2 f, float& cs, float& sn) {
+    const uint32_t turns = pos * f.y + __umulhi(pos, f.x) + 0x80000000u;
+    const float ang = fmaf(__uint_as_float((turns >> 9) | 0x3f800000u), 6.283185307179586f, -9.42477796076938f);
+    __sincosf(ang, &sn, &cs);
+}
 // Inverse frequencies theta^(-2c/d), c < d/2, into shared memory (fp64); callers synchronise.
 __device__ __forceinline__ void rope_fill_inv_freq(double* inv_freq, int d, float theta) {
     for (int c = threadIdx.x; c < d / 2; c += blockDim.x) inv_freq[c] = pow((double)theta, -2.0 * (double)c / (double)d);

@@ -253,14 +253,8 @@ static vector_status launch_decode_bf16_d128(const Dims& dm, const void* q, cons
     if (ch->n_ret == 0) { maps.ret_k = maps.apx_k; maps.ret_v = maps.apx_k; }   // never dereferenced: no such tiles
     if (ch->n_apx == 0) maps.apx_k = maps.ret_k;
     const float c2 = dm.scale * 1.4426950408889634f;
-    dbf::RopePhases ph = {};
-    if (dm.rope) {
-        // turns per position of channel pair c, theta^(-2c/128) / (2 pi), as a 64-bit fraction
-        for (int c = 0; c < 64; ++c) {
-            const long double f = powl((long double)dm.theta, -2.0L * c / 128.0L) / 6.283185307179586476925286766559L;
-            ph.phase[c] = (unsigned long long)ldexpl(f - floorl(f), 64);
-        }
-    }
+    RopePhases ph = {};
+    if (dm.rope) rope_phases(dm.theta, 128, &ph);
     if (mode == 1)
         dbf::decode_stream_bf16_d128<true, false><<<pl.B, dbf::THREADS, dbf::SMEM_BYTES_PER_TILE, st>>>(
             (const T*)q, maps, pl, (int)ch->n_ret, (int)ch->n_apx, dm.g, dm.LH, c2, partial, fault, nullptr, 0, ph);

@@ -36,6 +36,7 @@
 #define VECTOR_DECODE_BF16_CUH_
 
 #include "common.cuh"
+#include "internal.h"
 #include "tma.cuh"
 
 namespace vec {
@@ -151,13 +152,8 @@ __device__ __forceinline__ void derotate_rows(uint32_t kbase, int nrows, int mem
                 for (int h = 0; h < 2; ++h) {
                     const float x = __uint_as_float(h ? (xs[u][e] & 0xffff0000u) : (xs[u][e] << 16));
                     const float y = __uint_as_float(h ? (ys[u][e] & 0xffff0000u) : (ys[u][e] << 16));
-                    // top 32 bits of pos * phase modulo 2^64 (pos < 2^32): turns modulo 1, half a turn ahead
-                    const uint2 f = phase2[2 * e + h];
-                    const uint32_t turns = pos[u] * f.y + __umulhi(pos[u], f.x) + 0x80000000u;
-                    // its top 23 bits as a float in [1, 2); minus 1.5 is the turn count in [-0.5, 0.5)
-                    const float ang = fmaf(__uint_as_float((turns >> 9) | 0x3f800000u), 6.283185307179586f, -9.42477796076938f);
                     float sn, cs;
-                    __sincosf(ang, &sn, &cs);
+                    rope_phase_cos_sin(pos[u], phase2[2 * e + h], cs, sn);
                     xo[h] = fmaf(x, cs, y * sn);
                     yo[h] = fmaf(y, cs, -x * sn);
                 }
@@ -182,9 +178,6 @@ __device__ __forceinline__ void team_sync(int team) {
 }
 
 static_assert(SLOTS % CONSUMER_WARPS == 0, "a slot must always be consumed by the same warp");
-
-// phase[c] = frac(theta^(-2c/128) / (2 pi)) * 2^64, c < 64: turns per position, as a 64-bit fraction.
-struct RopePhases { unsigned long long phase[64]; };
 
 struct Maps {
     CUtensorMap ret_k, ret_v, apx_k;     // rank 3: (128 dims, pool rows, U units), box 64 x 64 x 1, 128B swizzle

@@ -14,6 +14,14 @@ namespace vec {
 static thread_local int g_last_cuda_error = 0;
 void set_last_cuda_error(int e) { g_last_cuda_error = e; }
 
+void rope_phases(float theta, int d, RopePhases* out) {
+    for (int c = 0; c < 64; ++c) {
+        if (c >= d / 2) { out->phase[c] = 0ull; continue; }
+        const long double f = powl((long double)theta, -2.0L * c / (long double)d) / 6.283185307179586476925286766559L;
+        out->phase[c] = (unsigned long long)ldexpl(f - floorl(f), 64);
+    }
+}
+
 static std::mutex g_once_mu;
 bool PerDeviceOnce::first() {
     int dev = -1;

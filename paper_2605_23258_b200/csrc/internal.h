@@ -25,6 +25,12 @@ struct Dims {
     float theta;
 };
 
+// phase[c] = frac(theta^(-2c/d) / (2 pi)) * 2^64, c < d/2 <= 64: the turns channel pair c makes per
+// position, as a 64-bit fraction.  The top 32 bits of position * phase (modulo 2^64) are then the
+// rotary angle of that pair, in turns modulo one, to 2^-32 of a turn for any 32-bit position.
+struct RopePhases { unsigned long long phase[64]; };
+void rope_phases(float theta, int d, RopePhases* out);
+
 // Checks a shape against what the kernels support and fills Dims.
 vector_status check_shape(const vector_shape* s, Dims* out);
 // Checks internal consistency of tier sizes (the identities of the planner).

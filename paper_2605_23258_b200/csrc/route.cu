@@ -285,7 +285,9 @@ static vector_status launch_residual_tc(const Dims& dm, const void* K, const voi
     if (n_idx == 0) return VECTOR_OK;
     static PerDeviceOnce once;
     if (once.first()) {
-        const cudaError_t e = cudaFuncSetAttribute(rtc::residual_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, rtc::SMEM_BYTES);
+        cudaError_t e = cudaFuncSetAttribute(rtc::residual_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, rtc::SMEM_BYTES);
+        if (e == cudaSuccess)
+            e = cudaFuncSetAttribute(rtc::residual_tc_rope, cudaFuncAttributeMaxDynamicSharedMemorySize, rtc::R_SMEM_BYTES);
         if (e != cudaSuccess) { once.undo(); VEC_CUDA_CHECK(e); }
     }
     int* fault = kernel_fault_address();
@@ -297,16 +299,22 @@ static vector_status launch_residual_tc(const Dims& dm, const void* K, const voi
     P.tpu = (int)((n_idx + rtc::TILE - 1) / rtc::TILE);
     P.n_tiles = (long long)dm.U * P.tpu;
     const int blocks = (int)(P.n_tiles < 148 ? P.n_tiles : 148);
-    rtc::residual_tc<<<blocks, rtc::THREADS, rtc::SMEM_BYTES, st>>>((const __nv_bfloat16*)K, (const __nv_bfloat16*)V, mapW,
-                                                                    idx, P, eps, fault);
+    if (dm.rope) {
+        RopePhases ph;
+        rope_phases(dm.theta, 128, &ph);
+        rtc::residual_tc_rope<<<blocks, rtc::R_THREADS, rtc::R_SMEM_BYTES, st>>>((const __nv_bfloat16*)K, (const __nv_bfloat16*)V,
+                                                                                 mapW, idx, P, ph, eps, fault);
+    } else {
+        rtc::residual_tc<<<blocks, rtc::THREADS, rtc::SMEM_BYTES, st>>>((const __nv_bfloat16*)K, (const __nv_bfloat16*)V, mapW,
+                                                                        idx, P, eps, fault);
+    }
     VEC_LAUNCH_CHECK();
     return VECTOR_OK;
 }
 
 static vector_status residual_dispatch(const Dims& dm, const void* K, const void* V, const void* W, int64_t N,
                                        const int32_t* idx, int64_t n_idx, float* eps, cudaStream_t st) {
-    // the de-rotating variant exists on the CUDA-core path only
-    if (!dm.rope && dm.dtype == VECTOR_BF16 && dm.d == 128) return launch_residual_tc(dm, K, V, W, N, idx, n_idx, eps, st);
+    if (dm.dtype == VECTOR_BF16 && dm.d == 128) return launch_residual_tc(dm, K, V, W, N, idx, n_idx, eps, st);
     if (dm.dtype == VECTOR_F32)
         return dm.d == 64 ? launch_residual<float, 64>(dm, K, V, W, N, idx, n_idx, eps, st)
                           : launch_residual<float, 128>(dm, K, V, W, N, idx, n_idx, eps, st);

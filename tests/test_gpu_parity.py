@@ -378,7 +378,8 @@ def test_residual_rope_parity(oracle, base, over, theta):
 
 
 def test_decode_rope_large_positions(oracle):
-    """Key-only rows whose original positions reach 10^5: the angle must be formed in fp64."""
+    """Key-only rows whose original positions reach 10^5 (tens of thousands of radians): the angle needs
+    more than fp32 to come out right modulo a turn."""
     wl = synth.shrink(synth.WORKLOADS[1], N=2048, n_kv_heads=2, n_q_heads=8, n_calib=1024)
     K, V, _ = synth.context(wl, DEV)
     W = calibrated_maps(wl).to(DEV)
