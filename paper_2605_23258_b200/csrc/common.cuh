@@ -3,6 +3,7 @@
 #define VECTOR_COMMON_CUH_
 
 #include <cuda_bf16.h>
+#include <cuda_fp16.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
 

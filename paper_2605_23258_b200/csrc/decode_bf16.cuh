@@ -110,13 +110,31 @@ __device__ __forceinline__ void mma_16(float (&c)[4], uint32_t a0, uint32_t a1, 
         : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
         : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
 }
+// The same product with fp16 operands (the keys turned back under RoPE decoupling are held in fp16).
+__device__ __forceinline__ void mma_16_f16(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0,
+                                           uint32_t b1) {
+    asm volatile(
+        "mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};\n"
+        : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+        : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+// Two floats to an fp16 pair, low half first; values beyond the fp16 range go to its largest finite number.
+__device__ __forceinline__ uint32_t pack_f16(float lo, float hi) {
+    uint32_t r;
+    asm("cvt.rn.satfinite.f16x2.f32 %0, %1, %2;\n" : "=r"(r) : "f"(hi), "f"(lo));
+    return r;
+}
+__device__ __forceinline__ float f16_lo(uint32_t v) { return __half2float(__ushort_as_half((unsigned short)(v & 0xffffu))); }
+__device__ __forceinline__ float f16_hi(uint32_t v) { return __half2float(__ushort_as_half((unsigned short)(v >> 16))); }
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
     __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
     return *reinterpret_cast<uint32_t*>(&v);
 }
 
 // RoPE decoupling: rows 16 member .. 16 member + 15 of the 64 keys at kbase (two swizzled boxes:
-// channels 0-63 | 64-127) are turned back by their positions, in place.  Channel c pairs with
+// channels 0-63 | 64-127) are turned back by their positions, in place, and left there as fp16 (a
+// turned key is not a bf16 number; eleven bits keep the key sum within the tolerance of the output,
+// eight do not; |k| beyond 65504 saturates).  Channel c pairs with
 // c + 64; the angle is position * theta^(-2c/128), taken as the top bits of the 64-bit product of
 // the position and the per-channel phase, so that it is exact modulo one turn.  pos16: lane l
 // holds the position of row 16 member + (l & 15).
@@ -157,8 +175,8 @@ __device__ __forceinline__ void derotate_rows(uint32_t kbase, int nrows, int mem
                     xo[h] = fmaf(x, cs, y * sn);
                     yo[h] = fmaf(y, cs, -x * sn);
                 }
-                xs[u][e] = pack_bf16(xo[0], xo[1]);
-                ys[u][e] = pack_bf16(yo[0], yo[1]);
+                xs[u][e] = pack_f16(xo[0], xo[1]);
+                ys[u][e] = pack_f16(yo[0], yo[1]);
             }
         }
 #pragma unroll
@@ -493,6 +511,19 @@ decode_stream_bf16_d128(const __nv_bfloat16* __restrict__ q, const __grid_consta
         for (int kk = 0; kk < 4; ++kk) {
             // P as bf16 hi (MMA rows 0-7) + lo (rows 8-15)
             const float p00 = sc[2 * kk][0], p01 = sc[2 * kk][1], p10 = sc[2 * kk + 1][0], p11 = sc[2 * kk + 1][1];
+            if (ROPE && !retained) {
+                // the turned keys are fp16: so are the weights, again as hi + lo
+                const uint32_t a0 = pack_f16(p00, p01), a2 = pack_f16(p10, p11);
+                const uint32_t a1 = pack_f16(p00 - f16_lo(a0), p01 - f16_hi(a0)), a3 = pack_f16(p10 - f16_lo(a2), p11 - f16_hi(a2));
+#pragma unroll
+                for (int np = 0; np < 8; ++np) {
+                    uint32_t b0, b1, b2, b3;
+                    ldsm_x4_t(vbase + (np >> 2) * BOX_BYTES + kk * 16 * 128 + pv_row + ((((2 * np) & 7) << 4) ^ pv_x), b0, b1, b2, b3);
+                    mma_16_f16(acc[2 * np], a0, a1, a2, a3, b0, b1);
+                    mma_16_f16(acc[2 * np + 1], a0, a1, a2, a3, b2, b3);
+                }
+                continue;
+            }
             const __nv_bfloat16 h00 = __float2bfloat16_rn(p00), h01 = __float2bfloat16_rn(p01);
             const __nv_bfloat16 h10 = __float2bfloat16_rn(p10), h11 = __float2bfloat16_rn(p11);
             const uint32_t a0 = pack_bf16(__bfloat162float(h00), __bfloat162float(h01));

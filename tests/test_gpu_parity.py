@@ -456,12 +456,16 @@ def test_decode_long_block_ranges(oracle):
             assert np.max(np.abs(out1[u].cpu().double().numpy() - o_tok)) <= 2e-2, (base, u, "per tile")
 
 
-def _sampled_units_case(oracle, wl, percent, sample):
+def _sampled_units_case(oracle, wl, percent, sample, theta=None):
     """Whole workload on the device in the launch shape the benchmark times; the oracle checks the
-    sampled units end to end, every unit is checked for the properties that hold at any size."""
+    sampled units end to end, every unit is checked for the properties that hold at any size.
+    With `theta` the stored keys are post-RoPE and RoPE decoupling is on."""
     K, V, Q = synth.context(wl, DEV)
     W = calibrated_maps(wl).to(DEV)
     sh = shape_of(wl)
+    if theta is not None:
+        K = synth.rope_keys(K, theta)
+        sh.rope_enabled, sh.rope_theta = 1, theta
     b = budget_of(wl, percent)
     comp = Compressor(sh, b, extra_rows=1, keep_eps=True)
     comp.compress(Q, K, V, W)
@@ -483,7 +487,7 @@ def _sampled_units_case(oracle, wl, percent, sample):
     LH = wl.n_layers * wl.n_kv_heads
     Ws = torch.stack([W[u % LH] for u in sample]).cpu()
     sub = synth.shrink(wl, batch=1, n_layers=1, n_kv_heads=len(sample), n_q_heads=len(sample) * wl.group)
-    _assert_routing_agrees(oracle, sub, b, _View, K[sample], V[sample], Ws, sc_o, list(range(len(sample))))
+    _assert_routing_agrees(oracle, sub, b, _View, K[sample], V[sample], Ws, sc_o, list(range(len(sample))), theta)
     _, sq, _ = synth.all_head_params(wl, DEV)
     q = synth.decode_q(wl, 0, DEV, sq)
     out = torch.empty(wl.units, wl.group, wl.head_dim, dtype=torch.float32, device=DEV)
@@ -493,8 +497,15 @@ def _sampled_units_case(oracle, wl, percent, sample):
     c = comp.cache
     for j, u in enumerate(sample):
         _, o = oracle.attend(q[u].cpu(), c.ret_k[u, : c.n_ret].cpu(), c.ret_v[u, : c.n_ret].cpu(),
-                             c.apx_k[u, : c.n_apx].cpu(), Ws[j], 1.0 / np.sqrt(wl.head_dim))
+                             c.apx_k[u, : c.n_apx].cpu(), Ws[j], 1.0 / np.sqrt(wl.head_dim),
+                             apx_pos=c.apx_pos[u, : c.n_apx].cpu().numpy(), rope=theta is not None, theta=theta or 10000.0)
         assert np.max(np.abs(out[u].cpu().double().numpy() - o)) <= 2e-2
+
+
+def test_config2_shape_rope_decoupled_sampled_units(oracle):
+    """Config-2 shape (8 of its layers: the decode grid is full, blocks start and end inside units) with
+    post-RoPE keys: the tensor-core residual and decode kernels with RoPE decoupling, sampled units."""
+    _sampled_units_case(oracle, synth.shrink(synth.WORKLOADS[2], n_layers=8), 20, [0, 37, 63], theta=500000.0)
 
 
 def test_full_size_bench_configuration_sampled_units(oracle):
