@@ -3,9 +3,10 @@
 //
 // Both selections are exact top-k with the lower index winning ties, done as a
 // most-significant-digit radix select on an order-preserving 32-bit image of
-// the fp32 value (4 histogram passes of 8 bits find the k-th key and how many
-// ties of it are taken), followed by one ordered pass whose block-wide prefix
-// sums place the chosen indices in ascending order.  One thread block per unit.
+// the fp32 value (3 histogram passes of 11, 11 and 10 bits find the k-th key and
+// how many ties of it are taken; the third runs over a short list of
+// candidates), followed by one ordered walk whose block-wide prefix sums place
+// the chosen indices in ascending order.  One thread block per unit.
 #include "common.cuh"
 #include "internal.h"
 #include "residual_tc.cuh"
@@ -14,11 +15,6 @@ namespace vec {
 
 constexpr int SEL_THREADS = 1024;
 
-struct SelectResult {
-    uint32_t kth_key;   // image of the k-th best value
-    int take_ties;      // how many elements equal to it are taken (lowest indices first)
-};
-
 // Best = largest image.  For "k smallest" the caller passes inverted images.
 template <bool SMALLEST>
 __device__ __forceinline__ uint32_t select_image(float v) {
@@ -26,92 +22,205 @@ __device__ __forceinline__ uint32_t select_image(float v) {
     return SMALLEST ? ~k : k;
 }
 
-// hist[bin] += 1 for every lane with `valid`.  When the whole warp hits one bin (common in the later
-// passes, where the surviving keys share their leading bits) a single lane adds the count.
-// Every lane of the warp must call it.
+// hist[bin] += 1 if `valid`.  With 11-bit digits the lanes of a warp rarely share a bin, so a plain
+// shared-memory atomic per element is cheaper than aggregating equal bins across the warp first;
+// equal bins (many equal values) serialise inside the atomic unit and cost time, not correctness.
 __device__ __forceinline__ void hist_add(int* hist, int bin, bool valid) {
-    const unsigned active = __ballot_sync(0xffffffffu, valid);
-    if (active == 0) return;
-    const int first = __shfl_sync(0xffffffffu, bin, __ffs(active) - 1);
-    if (__ballot_sync(0xffffffffu, valid && bin != first) == 0) {
-        if ((int)(threadIdx.x & 31) == __ffs(active) - 1) atomicAdd(&hist[first], __popc(active));
-    } else if (valid) {
-        atomicAdd(&hist[bin], 1);
+    if (valid) atomicAdd(&hist[bin], 1);
+}
+
+// Scratch of one selection (static shared memory of the block).
+constexpr int CAND_CAP = 6144;
+constexpr int MASK_GROUPS = 1024;   // groups of 32 elements whose selection is kept as bit masks
+struct OrderedScratch { int gt[32], tie[32], out[32], quota[32]; };
+constexpr int SEL_BINS = 2048;      // digits of 11, 11 and 10 bits
+struct SelectScratch {
+    int hist[SEL_BINS];
+    int bc[2];
+    int n_cand, overflow;
+    int32_t cand[CAND_CAP];       // indices of the elements that share the k-th key's leading 11 bits
+    uint32_t sel_mask[MASK_GROUPS];   // per group of 32 elements: those above the k-th key
+    uint32_t tie_mask[MASK_GROUPS];   // ... and those equal to it
+    OrderedScratch os;
+};
+
+// Warp 0: the bin of hist[0..SEL_BINS), counted from the top, in which the cumulative count reaches
+// `remaining` (-> bc[0]) and the rank wanted inside that bin, 1-based (-> bc[1]).
+__device__ __forceinline__ void pick_bin(const int* hist, int remaining, int* bc) {
+    constexpr int PER = SEL_BINS / 32;
+    if (threadIdx.x < 32) {
+        const int top = SEL_BINS - 1 - (int)threadIdx.x * PER;      // this lane's bins: top, top - 1, ..
+        int tot = 0;
+#pragma unroll 8
+        for (int j = 0; j < PER; ++j) tot += hist[top - j];
+        int inc = tot;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const int t = __shfl_up_sync(0xffffffffu, inc, o);
+            if ((int)threadIdx.x >= o) inc += t;
+        }
+        int cum = inc - tot;                            // count in the bins above this lane's
+        if (cum < remaining && inc >= remaining) {      // exactly one lane
+            for (int j = 0; j < PER; ++j) {
+                const int c = hist[top - j];
+                if (cum + c >= remaining) { bc[0] = top - j; bc[1] = remaining - cum; break; }
+                cum += c;
+            }
+        }
     }
 }
 
-// Finds the k-th largest image among vals[0..n) (1 <= k <= n).  All threads of the
-// block call it and all get the result.  hist: 256 ints of shared memory; bc: 2 ints.
+// One histogram pass over all of vals on the digit at `shift`, among the elements whose image
+// matches prefix under mask.  Eight independent loads in flight per thread: the pass is bound by
+// memory latency otherwise.
 template <bool SMALLEST>
-__device__ SelectResult radix_select(const float* __restrict__ vals, int n, int k, int* hist, int* bc) {
-    uint32_t prefix = 0, mask = 0;
-    int remaining = k;
-    for (int shift = 24; shift >= 0; shift -= 8) {
-        for (int b = threadIdx.x; b < 256; b += blockDim.x) hist[b] = 0;
-        __syncthreads();
-        // eight independent loads in flight per thread: the pass is bound by memory latency otherwise
-        for (int base = 0; base < n; base += 8 * blockDim.x) {
-            float v[8];
+__device__ __forceinline__ void hist_pass_all(const float* __restrict__ vals, int n, int shift, uint32_t digit_mask,
+                                              uint32_t prefix, uint32_t mask, int* hist) {
+    for (int base = 0; base < n; base += 8 * blockDim.x) {
+        float v[8];
 #pragma unroll
-            for (int j = 0; j < 8; ++j) {
-                const int i = base + j * blockDim.x + threadIdx.x;
-                v[j] = i < n ? vals[i] : 0.f;
-            }
-#pragma unroll
-            for (int j = 0; j < 8; ++j) {
-                const int i = base + j * blockDim.x + threadIdx.x;
-                const uint32_t key = select_image<SMALLEST>(v[j]);
-                hist_add(hist, (key >> shift) & 255, i < n && (key & mask) == prefix);
-            }
+        for (int j = 0; j < 8; ++j) {
+            const int i = base + j * blockDim.x + threadIdx.x;
+            v[j] = i < n ? vals[i] : 0.f;
         }
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+            const int i = base + j * blockDim.x + threadIdx.x;
+            const uint32_t key = select_image<SMALLEST>(v[j]);
+            hist_add(hist, (key >> shift) & digit_mask, i < n && (key & mask) == prefix);
+        }
+    }
+}
+
+// Piece of the input that warp `wid` owns in the ordered passes: [w0, w1), a multiple of 32 long.
+__device__ __forceinline__ int ordered_chunk(int n, int nw) { return (((n + nw - 1) / nw) + 31) & ~31; }
+
+// Exact top-k of vals[0..n) (largest images; for "k smallest" the images are inverted) with the
+// lower index winning ties, emitted in index order: emit(i, chosen, pos) is called for every element
+// i, pos being its rank among the chosen ones if chosen, else among the others.  1 <= k <= n
+// unless !any (nothing is chosen then).  All threads of the block call it.
+//
+// The k-th key is found by a most-significant-digit radix select with digits of 11, 11 and 10 bits.
+// Pass 1 reads the whole input.  Pass 2 reads it once more, warp by contiguous piece, and on the
+// way (a) notes per group of 32 elements, as a bit mask, those whose leading 11 bits already beat
+// the k-th key's and (b) lists the indices of those that share them (the candidates: a quarter of
+// a binade of values, a few thousand at most).  Pass 3 runs over the list; so does the final
+// classification, which adds the candidates above the k-th key to the masks and marks its ties in
+// a second mask.  The per-piece counts and the emission in index order then need the masks only,
+// not the values.  Two fallbacks read the input again instead: more than CAND_CAP candidates
+// (pass 3 and the classification walk the input), more than 32 MASK_GROUPS elements (the masks are
+// not kept).
+template <bool SMALLEST, typename Emit>
+__device__ __forceinline__ void select_emit(const float* __restrict__ vals, int n, int k, bool any, SelectScratch& S, Emit emit) {
+    const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5, nw = blockDim.x >> 5;
+    const unsigned lt = (1u << lane) - 1u;
+    const int per_w = ordered_chunk(n, nw);
+    const int w0 = min(n, wid * per_w), w1 = min(n, w0 + per_w);
+    const bool masked = n <= 32 * MASK_GROUPS;
+    uint32_t kth = 0xffffffffu;
+    int take_ties = 0;
+    if (threadIdx.x < 32) { S.os.gt[threadIdx.x] = 0; S.os.tie[threadIdx.x] = 0; }
+    if (masked)
+        for (int g = threadIdx.x; g < MASK_GROUPS; g += blockDim.x) { S.sel_mask[g] = 0u; S.tie_mask[g] = 0u; }
+    if (any) {
+        // ---- pass 1: leading 11 bits
+        for (int b = threadIdx.x; b < SEL_BINS; b += blockDim.x) S.hist[b] = 0;
+        if (threadIdx.x == 0) { S.n_cand = 0; S.overflow = 0; }
         __syncthreads();
-        if (threadIdx.x < 32) {
-            // warp 0: the bin, counted from the top, in which the cumulative count reaches `remaining`
-            int c[8], tot = 0;
+        hist_pass_all<SMALLEST>(vals, n, 21, 2047u, 0u, 0u, S.hist);
+        __syncthreads();
+        pick_bin(S.hist, k, S.bc);
+        __syncthreads();
+        const uint32_t bin1 = (uint32_t)S.bc[0];
+        int remaining = S.bc[1];
+        __syncthreads();
+        // ---- pass 2: next 11 bits among the candidates; masks of the sure ones; candidate list
+        for (int b = threadIdx.x; b < SEL_BINS; b += blockDim.x) S.hist[b] = 0;
+        __syncthreads();
+        for (int base = w0; base < w1; base += 128) {
+            float v[4];
 #pragma unroll
-            for (int j = 0; j < 8; ++j) { c[j] = hist[255 - (threadIdx.x * 8 + j)]; tot += c[j]; }
-            int inc = tot;
+            for (int j = 0; j < 4; ++j) v[j] = base + 32 * j + lane < w1 ? vals[base + 32 * j + lane] : 0.f;
 #pragma unroll
-            for (int o = 1; o < 32; o <<= 1) {
-                const int t = __shfl_up_sync(0xffffffffu, inc, o);
-                if ((int)threadIdx.x >= o) inc += t;
-            }
-            int cum = inc - tot;                            // count in the bins above this lane's eight
-            if (cum < remaining && inc >= remaining) {      // exactly one lane
-#pragma unroll
-                for (int j = 0; j < 8; ++j) {
-                    if (cum + c[j] >= remaining) { bc[0] = 255 - (threadIdx.x * 8 + j); bc[1] = remaining - cum; break; }
-                    cum += c[j];
+            for (int j = 0; j < 4; ++j) {
+                const int i = base + 32 * j + lane;
+                const bool in = i < w1;
+                const uint32_t key = select_image<SMALLEST>(v[j]);
+                const uint32_t d1 = key >> 21;
+                if (masked) {
+                    const unsigned gb = __ballot_sync(0xffffffffu, in && d1 > bin1);
+                    if (lane == 0 && base + 32 * j < w1) S.sel_mask[(base >> 5) + j] = gb;
+                }
+                if (in && d1 == bin1) {
+                    atomicAdd(&S.hist[(key >> 10) & 2047], 1);
+                    const int at = atomicAdd(&S.n_cand, 1);
+                    if (at < CAND_CAP) S.cand[at] = i;
+                    else S.overflow = 1;
                 }
             }
         }
         __syncthreads();
-        prefix |= (uint32_t)bc[0] << shift;
-        mask |= 255u << shift;
-        remaining = bc[1];              // rank wanted inside the chosen bin (1-based)
+        pick_bin(S.hist, remaining, S.bc);
         __syncthreads();
+        uint32_t prefix = (bin1 << 21) | ((uint32_t)S.bc[0] << 10);
+        const uint32_t mask = 0xfffffc00u;
+        remaining = S.bc[1];
+        const bool listed = S.overflow == 0;
+        const int n_cand = S.n_cand;
+        __syncthreads();
+        // ---- pass 3: the last 10 bits
+        for (int b = threadIdx.x; b < SEL_BINS; b += blockDim.x) S.hist[b] = 0;
+        __syncthreads();
+        if (listed) {
+            for (int j = threadIdx.x; j < n_cand; j += blockDim.x) {
+                const uint32_t key = select_image<SMALLEST>(vals[S.cand[j]]);
+                hist_add(S.hist, key & 1023, (key & mask) == prefix);
+            }
+        } else {
+            hist_pass_all<SMALLEST>(vals, n, 0, 1023u, prefix, mask, S.hist);
+        }
+        __syncthreads();
+        pick_bin(S.hist, remaining, S.bc);
+        __syncthreads();
+        prefix |= (uint32_t)S.bc[0];
+        remaining = S.bc[1];
+        __syncthreads();
+        kth = prefix;
+        take_ties = remaining;          // all strictly better elements precede; `remaining` ties complete k
+        // ---- the candidates against the k-th key
+        if (masked && listed) {
+            for (int j = threadIdx.x; j < n_cand; j += blockDim.x) {
+                const int i = S.cand[j];
+                const uint32_t key = select_image<SMALLEST>(vals[i]);
+                if (key > kth) atomicOr(&S.sel_mask[i >> 5], 1u << (i & 31));
+                else if (key == kth) atomicOr(&S.tie_mask[i >> 5], 1u << (i & 31));
+            }
+        } else if (masked) {
+            for (int base = w0; base < w1; base += 128) {
+                float v[4];
+#pragma unroll
+                for (int j = 0; j < 4; ++j) v[j] = base + 32 * j + lane < w1 ? vals[base + 32 * j + lane] : 0.f;
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    const bool in = base + 32 * j + lane < w1;
+                    const uint32_t key = select_image<SMALLEST>(v[j]);
+                    const unsigned gb = __ballot_sync(0xffffffffu, in && key > kth);
+                    const unsigned tb = __ballot_sync(0xffffffffu, in && key == kth);
+                    if (lane == 0 && base + 32 * j < w1) { S.sel_mask[(base >> 5) + j] = gb; S.tie_mask[(base >> 5) + j] = tb; }
+                }
+            }
+        }
     }
-    SelectResult r;
-    r.kth_key = prefix;
-    r.take_ties = remaining;   // all strictly better elements precede; `remaining` ties complete k
-    return r;
-}
-
-// The ordered pass both selections end with.  Every warp owns a contiguous piece of the input and
-// walks it 32 elements at a time (coalesced); positions inside a warp come from ballots, the
-// offsets of the warps from one small scan by warp 0.  `emit(i, chosen, pos)` is called for every
-// element i: pos is its rank among the chosen ones if chosen, else among the others.
-struct OrderedScratch { int gt[32], tie[32], out[32], quota[32]; };
-
-template <bool SMALLEST, typename Emit>
-__device__ __forceinline__ void ordered_pass(const float* __restrict__ vals, int n, const SelectResult& sel, bool any,
-                                             OrderedScratch& sc, Emit emit) {
-    const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5, nw = blockDim.x >> 5;
-    const unsigned lt = (1u << lane) - 1u;
-    const int per_w = (((n + nw - 1) / nw) + 31) & ~31;
-    const int w0 = min(n, wid * per_w), w1 = min(n, w0 + per_w);
-    int n_gt = 0, n_tie = 0;
-    if (any) {
+    __syncthreads();
+    // ---- per piece: how many better elements, how many ties
+    if (masked) {
+        int g2 = 0, t2 = 0;
+        for (int g = (w0 >> 5) + lane; g < ((w1 + 31) >> 5); g += 32) { g2 += __popc(S.sel_mask[g]); t2 += __popc(S.tie_mask[g]); }
+        g2 = __reduce_add_sync(0xffffffffu, g2);
+        t2 = __reduce_add_sync(0xffffffffu, t2);
+        if (lane == 0) { S.os.gt[wid] = g2; S.os.tie[wid] = t2; }
+    } else if (any) {
+        int g2 = 0, t2 = 0;
         for (int base = w0; base < w1; base += 128) {
             float v[4];
 #pragma unroll
@@ -120,45 +229,61 @@ __device__ __forceinline__ void ordered_pass(const float* __restrict__ vals, int
             for (int j = 0; j < 4; ++j) {
                 const bool in = base + 32 * j + lane < w1;
                 const uint32_t key = select_image<SMALLEST>(v[j]);
-                n_gt += __popc(__ballot_sync(0xffffffffu, in && key > sel.kth_key));
-                n_tie += __popc(__ballot_sync(0xffffffffu, in && key == sel.kth_key));
+                g2 += __popc(__ballot_sync(0xffffffffu, in && key > kth));
+                t2 += __popc(__ballot_sync(0xffffffffu, in && key == kth));
             }
         }
+        if (lane == 0) { S.os.gt[wid] = g2; S.os.tie[wid] = t2; }
     }
-    if (lane == 0) { sc.gt[wid] = n_gt; sc.tie[wid] = n_tie; }
     __syncthreads();
+    // ---- offsets of the pieces; ties go to the lowest indices
     if (wid == 0) {
-        const int t = lane < nw ? sc.tie[lane] : 0;
+        const int t = lane < nw ? S.os.tie[lane] : 0;
         int inc = t;
 #pragma unroll
         for (int o = 1; o < 32; o <<= 1) { const int x = __shfl_up_sync(0xffffffffu, inc, o); if (lane >= o) inc += x; }
-        const int quota = max(0, min(t, sel.take_ties - (inc - t)));       // ties go to the lowest indices
-        const int c = (lane < nw ? sc.gt[lane] : 0) + quota;
+        const int quota = max(0, min(t, take_ties - (inc - t)));
+        const int c = (lane < nw ? S.os.gt[lane] : 0) + quota;
         int ci = c;
 #pragma unroll
         for (int o = 1; o < 32; o <<= 1) { const int x = __shfl_up_sync(0xffffffffu, ci, o); if (lane >= o) ci += x; }
-        sc.out[lane] = ci - c;
-        sc.quota[lane] = quota;
+        S.os.out[lane] = ci - c;
+        S.os.quota[lane] = quota;
     }
     __syncthreads();
-    int pos = sc.out[wid], ties_left = sc.quota[wid];
-    for (int base = w0; base < w1; base += 128) {
-        float v[4];
-#pragma unroll
-        for (int j = 0; j < 4; ++j) v[j] = base + 32 * j + lane < w1 ? vals[base + 32 * j + lane] : 0.f;
-#pragma unroll
-        for (int j = 0; j < 4; ++j) {
-            const int i = base + 32 * j + lane;
-            const bool in = i < w1;
-            const uint32_t key = select_image<SMALLEST>(v[j]);
-            const bool tie = any && in && key == sel.kth_key;
-            const unsigned tb = __ballot_sync(0xffffffffu, tie);
-            const bool chosen = any && in && (key > sel.kth_key || (tie && __popc(tb & lt) < ties_left));
+    // ---- emission in index order
+    int pos = S.os.out[wid], ties_left = S.os.quota[wid];
+    if (masked) {
+        for (int base = w0; base < w1; base += 32) {
+            const int i = base + lane;
+            const unsigned gb = S.sel_mask[base >> 5], tb = S.tie_mask[base >> 5];
+            const int take = min(ties_left, __popc(tb));
+            const bool chosen = ((gb >> lane) & 1u) || (((tb >> lane) & 1u) && __popc(tb & lt) < take);
             const unsigned cb = __ballot_sync(0xffffffffu, chosen);
             const int before = pos + __popc(cb & lt);               // chosen elements before this one in the unit
-            if (in) emit(i, chosen, chosen ? before : i - before);
+            if (i < w1) emit(i, chosen, chosen ? before : i - before);
             pos += __popc(cb);
-            ties_left -= min(ties_left, __popc(tb));
+            ties_left -= take;
+        }
+    } else {
+        for (int base = w0; base < w1; base += 128) {
+            float v[4];
+#pragma unroll
+            for (int j = 0; j < 4; ++j) v[j] = base + 32 * j + lane < w1 ? vals[base + 32 * j + lane] : 0.f;
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                const int i = base + 32 * j + lane;
+                const bool in = i < w1;
+                const uint32_t key = select_image<SMALLEST>(v[j]);
+                const bool tie = any && in && key == kth;
+                const unsigned tb = __ballot_sync(0xffffffffu, tie);
+                const bool chosen = any && in && (key > kth || (tie && __popc(tb & lt) < ties_left));
+                const unsigned cb = __ballot_sync(0xffffffffu, chosen);
+                const int before = pos + __popc(cb & lt);
+                if (in) emit(i, chosen, chosen ? before : i - before);
+                pos += __popc(cb);
+                ties_left -= min(ties_left, __popc(tb));
+            }
         }
     }
 }
@@ -166,15 +291,12 @@ __device__ __forceinline__ void ordered_pass(const float* __restrict__ vals, int
 // Step 1.  grid (U), SEL_THREADS threads.
 __global__ void __launch_bounds__(SEL_THREADS, 2)
 pool_select_kernel(const float* __restrict__ scores, int64_t N, int n_pool, int32_t* __restrict__ pool_idx) {
-    __shared__ int hist[256];
-    __shared__ int bc[2];
-    __shared__ OrderedScratch sc;
+    __shared__ SelectScratch S;
     const int u = blockIdx.x, n = (int)N;
     const float* s = scores + (size_t)u * N;
     int32_t* out = pool_idx + (size_t)u * n_pool;
     if (n_pool <= 0) return;
-    const SelectResult sel = radix_select<false>(s, n, n_pool, hist, bc);
-    ordered_pass<false>(s, n, sel, true, sc, [&](int i, bool chosen, int pos) { if (chosen) out[pos] = i; });
+    select_emit<false>(s, n, n_pool, true, S, [&](int i, bool chosen, int pos) { if (chosen) out[pos] = i; });
 }
 
 // Step 3.  grid (U), SEL_THREADS threads.
@@ -182,9 +304,7 @@ __global__ void __launch_bounds__(SEL_THREADS, 2)
 truncate_kernel(const float* __restrict__ eps, const int32_t* __restrict__ pool_idx, int64_t N, int n_pool,
                 int n_apx, uint8_t* __restrict__ tier, int32_t* __restrict__ ret_idx,
                 int32_t* __restrict__ apx_idx) {
-    __shared__ int hist[256];
-    __shared__ int bc[2];
-    __shared__ OrderedScratch sc;
+    __shared__ SelectScratch S;
     const int u = blockIdx.x;
     const float* e = eps + (size_t)u * n_pool;
     const int32_t* pool = pool_idx + (size_t)u * n_pool;
@@ -198,11 +318,7 @@ truncate_kernel(const float* __restrict__ eps, const int32_t* __restrict__ pool_
         for (int64_t i = threadIdx.x; i < N; i += SEL_THREADS) tr[i] = 0;
     }
     __syncthreads();
-    SelectResult sel;
-    sel.kth_key = 0xffffffffu;
-    sel.take_ties = 0;
-    if (n_apx > 0) sel = radix_select<true>(e, n_pool, n_apx, hist, bc);
-    ordered_pass<true>(e, n_pool, sel, n_apx > 0, sc, [&](int p, bool is_apx, int pos) {
+    select_emit<true>(e, n_pool, n_apx, n_apx > 0, S, [&](int p, bool is_apx, int pos) {
         const int32_t token = pool[p];
         if (is_apx) { ao[pos] = token; tr[token] = 1; }
         else        { ro[pos] = token; tr[token] = 2; }

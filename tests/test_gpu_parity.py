@@ -140,7 +140,11 @@ def test_diagnostics_parity(oracle):
 def _selection_inputs(U, N, seed, ties):
     g = torch.Generator().manual_seed(seed)
     s = torch.rand(U, N, generator=g)
-    if ties:
+    if ties == "narrow":
+        s = 1.0 + 0.01 * s                              # all values share their leading 11 bits
+    elif ties == "equal":
+        s = torch.full_like(s, 0.25)
+    elif ties:
         s = torch.round(s * 16) / 16                    # many exact ties
     s[:, -8:] = float("inf")
     s[0, : N // 3] = 0.0
@@ -149,7 +153,11 @@ def _selection_inputs(U, N, seed, ties):
 
 @pytest.mark.parametrize("N,n_pool,ties", [(1000, 300, False), (1000, 300, True), (5000, 4999, True),
                                            (4096, 8, True), (70000, 20000, True), (2048, 2048, False),
-                                           (131072, 9829, False)])
+                                           (131072, 9829, False),
+                                           # more candidates after the first digit than the list holds, with
+                                           # and without the bit masks (N above 32768), and nothing but ties
+                                           (20000, 7000, "narrow"), (70000, 20000, "narrow"), (32768, 11000, "equal"),
+                                           (40000, 100, "equal")])
 def test_pool_select_bit_exact(oracle, N, n_pool, ties):
     U = 3
     s = _selection_inputs(U, N, N + n_pool, ties)
@@ -187,13 +195,16 @@ def test_residual_parity(oracle, base, over, n_idx):
 
 @pytest.mark.parametrize("N,n_pool,n_apx,ties", [(1024, 384, 256, False), (1024, 384, 256, True),
                                                  (4000, 1501, 0, True), (4000, 1500, 1500, True),
-                                                 (131072, 9829, 6552, False), (50, 20, 2, True)])
+                                                 (131072, 9829, 6552, False), (50, 20, 2, True),
+                                                 (32768, 11468, 6552, "narrow"), (131072, 45000, 30000, "narrow")])
 def test_truncate_bit_exact(oracle, N, n_pool, n_apx, ties):
     U = 3
     g = torch.Generator().manual_seed(N + n_apx)
     pool = torch.stack([torch.randperm(N, generator=g)[:n_pool].sort().values for _ in range(U)]).to(torch.int32)
     eps = torch.rand(U, n_pool, generator=g) * 3
-    if ties:
+    if ties == "narrow":
+        eps = 2.0 + eps * 0.01                           # one quarter-binade: the candidate list overflows
+    elif ties:
         eps = torch.round(eps * 8) / 8
     wl = synth.shrink(synth.WORKLOADS[0], N=N, window=1, n_kv_heads=U, n_q_heads=U)
     n_a = n_apx // 2
