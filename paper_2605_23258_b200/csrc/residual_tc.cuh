@@ -1,15 +1,24 @@
 // Reconstruction residual of Step 2 on the tensor cores (bf16, head_dim 128):
-//   eps[p] = || v_i - W k_i ||^2,  i = idx[p].
+//   eps[p] = || v_i - W k~_i ||^2,  i = idx[p],  k~ = the key, or under RoPE decoupling the key
+//   turned back by its position (the token index itself), channel c pairing with c + 64.
 // The gather of the listed K and V rows is what costs (64 flop per byte: HBM-bound), so the
-// kernel is built around keeping row loads in flight.  Per 128-row tile the accumulator is
-//   D = K_tile W^T + V_tile (-I)      one chain of 16 tcgen05.mma (k = 256) in tensor memory,
-// i.e. minus the residual itself; the epilogue only squares and adds along each TMEM lane.
+// kernel is built around keeping row loads in flight.  Per 128-row tile the accumulator in tensor
+// memory is D = K_tile W^T (one chain of 8 tcgen05.mma); the epilogue subtracts the value row,
+// which it reads from the tile's copy in shared memory, squares and adds along its TMEM lane.
 //
 // Persistent blocks (one per SM) own equal contiguous ranges of the global tile sequence.
-//   warps 0-3  loaders: cp.async gathers of K and V rows into two stages, written directly in the
-//              128-byte-swizzled layout the MMA reads; row indices are fetched one tile ahead
-//   warp  4    MMA issuer, TMEM owner; also TMA-loads the unit's W when the range enters a new unit
-//   warps 5-8  epilogue: thread = row, sum of squares of its 128 accumulator columns
+//   warps 0-7   loaders: cp.async gathers of K and V rows into the stages, written directly in the
+//               128-byte-swizzled layout the MMA reads; row indices are fetched one tile ahead.
+//               Each thread gathers, for its rows, the 16-byte chunk qc of both key halves
+//               (channels 8 qc.. and 64 + 8 qc..) and the same two chunks of V.
+//   warp  8     MMA issuer, TMEM owner; also TMA-loads the unit's W when the range enters a new unit
+//   warps 9-12  epilogue: thread = row
+// Without RoPE: three stages of K | V (64 KB each), tiles published two behind the one being issued.
+// With RoPE: the turned key is no longer a bf16 number, so it goes to the tensor cores as a bf16
+// pair hi + lo (two chains over the same W), which keeps it to 2^-17 relative; two stages of
+// K hi | K lo | V (96 KB each).  A loader thread turns its own eight channel pairs of each of its
+// rows back once its own copies of the previous tile have landed (no cross-thread hand-over),
+// writes hi in place and lo into the second operand tile.
 #ifndef VECTOR_RESIDUAL_TC_CUH_
 #define VECTOR_RESIDUAL_TC_CUH_
 
@@ -23,23 +32,12 @@ namespace rtc {
 
 constexpr int BOX_BYTES = 16384;                           // 128 rows x 128 bytes
 constexpr int TILE = 128;
-constexpr int STAGES = 2;
 constexpr int OPERAND_BYTES = 2 * BOX_BYTES;               // 128 rows x 256 B as two swizzled halves
-constexpr int STAGE_BYTES = 2 * OPERAND_BYTES;             // K tile | V tile
-constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 2 * OPERAND_BYTES + 1024;   // + W + (-I)
-constexpr int LOADER_WARPS = 4, EPI_WARPS = 4;
-constexpr int THREADS = 32 * (LOADER_WARPS + 1 + EPI_WARPS);
-constexpr int TMEM_COLS = 256;
+constexpr int EPI_WARPS = 4;
 
 struct Params {
     int U, LH, n_idx, tpu;       // units, maps, rows per unit, tiles per unit
     long long N, n_tiles;        // keys per unit, U * tpu
-};
-
-struct Sync {
-    uint64_t full[STAGES], done[STAGES], empty[STAGES];
-    uint64_t w_full, w_empty;
-    uint32_t tmem_base;
 };
 
 __device__ __forceinline__ void cp_async16(uint32_t dst, const void* src, uint32_t src_bytes) {
@@ -55,205 +53,30 @@ __device__ __forceinline__ uint32_t pack2_bf16(float lo, float hi) {
 }
 __device__ __forceinline__ long long range_begin(int b, long long n_tiles, int B) { return (long long)b * n_tiles / B; }
 
-// grid: min(148, n_tiles) blocks.
-__global__ void __launch_bounds__(THREADS, 1)
-residual_tc(const __nv_bfloat16* __restrict__ K, const __nv_bfloat16* __restrict__ V,
-            const __grid_constant__ CUtensorMap mapW, const int32_t* __restrict__ idx, const Params P,
-            float* __restrict__ eps, int* __restrict__ fault) {
-    extern __shared__ unsigned char smem_raw[];
-    __shared__ Sync sy;
-    unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-    unsigned char* stage0 = smem;
-    unsigned char* Ws = smem + STAGES * STAGE_BYTES;
-    unsigned char* Is = Ws + OPERAND_BYTES;
-    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const long long gt_lo = range_begin(blockIdx.x, P.n_tiles, gridDim.x);
-    const long long gt_hi = range_begin(blockIdx.x + 1, P.n_tiles, gridDim.x);
-    const int n_my = (int)(gt_hi - gt_lo);
-
-    // minus identity in the operand layout: row j, column j -> half j / 64, 16-byte chunk swizzled by the row
-    for (int e = tid; e < OPERAND_BYTES / 16; e += THREADS) reinterpret_cast<uint4*>(Is)[e] = make_uint4(0, 0, 0, 0);
-    __syncthreads();
-    if (tid < 128) {
-        const int j = tid;
-        const uint32_t off = (j >> 6) * BOX_BYTES + j * 128 + ((((j & 63) >> 3) ^ (j & 7)) << 4) + (j & 7) * 2;
-        *reinterpret_cast<uint16_t*>(Is + off) = 0xBF80;     // bf16 -1
-    }
-    fence_async_proxy();
-    if (tid == 0) {
-#pragma unroll
-        for (int s = 0; s < STAGES; ++s) {
-            tma::mbar_init(&sy.full[s], 32 * LOADER_WARPS);
-            tma::mbar_init(&sy.done[s], 1);
-            tma::mbar_init(&sy.empty[s], EPI_WARPS);
-        }
-        tma::mbar_init(&sy.w_full, 1);
-        tma::mbar_init(&sy.w_empty, 1);
-        tma::mbar_fence_init();
-    }
-    if (warp == LOADER_WARPS) {
-        tc::tmem_alloc(&sy.tmem_base, TMEM_COLS);
-        tc::tmem_relinquish();
-    }
-    tc::fence_before_sync();
-    __syncthreads();
-    tc::fence_after_sync();
-
-    if (warp < LOADER_WARPS) {
-        // ------------------------------------------------------------------ loaders
-        const int rsub = tid >> 4, c = tid & 15;                    // row inside a pass of 8 rows, 16-byte chunk of the row
-        const uint32_t dst_thread = (c >> 3) * BOX_BYTES + rsub * 128 + (((c & 7) ^ rsub) << 4);
-        int32_t cur[16], nxt[16];
-        auto fetch_idx = [&](int i, int32_t (&out)[16]) {
-            const long long gt = gt_lo + i;
-            const int u = (int)(gt / P.tpu), t = (int)(gt - (long long)u * P.tpu);
-#pragma unroll
-            for (int p = 0; p < 16; ++p) {
-                const int row = t * TILE + p * 8 + rsub;
-                out[p] = row < P.n_idx ? idx[(size_t)u * P.n_idx + row] : -1;
-            }
-        };
-        bool ok = true;
-        if (n_my > 0) fetch_idx(0, cur);
-        for (int i = 0; i < n_my && ok; ++i) {
-            const int s = i % STAGES, round = i / STAGES;
-            if (i + 1 < n_my) fetch_idx(i + 1, nxt);
-            if (round > 0 && !tma::mbar_wait(&sy.empty[s], (round - 1) & 1, fault, 41)) { ok = false; break; }
-            const int u = (int)((gt_lo + i) / P.tpu);
-            const uint32_t kdst = tma::smem_u32(stage0 + s * STAGE_BYTES) + dst_thread;
-            const uint32_t vdst = kdst + OPERAND_BYTES;
-            const __nv_bfloat16* Ku = K + (size_t)u * P.N * 128 + c * 8;
-            const __nv_bfloat16* Vu = V + (size_t)u * P.N * 128 + c * 8;
-#pragma unroll
-            for (int p = 0; p < 16; ++p) {
-                const bool valid = cur[p] >= 0;
-                const size_t ro = valid ? (size_t)cur[p] * 128 : 0;
-                cp_async16(kdst + p * 1024, Ku + ro, valid ? 16u : 0u);     // zero fill past the end of the list
-                cp_async16(vdst + p * 1024, Vu + ro, valid ? 16u : 0u);
-            }
-            cp_async_commit();
-            if (i > 0) {                                 // the previous tile has landed: publish it to the MMA
-                cp_async_wait<1>();
-                fence_async_proxy();
-                tma::mbar_arrive(&sy.full[(i - 1) % STAGES]);
-            }
-#pragma unroll
-            for (int p = 0; p < 16; ++p) cur[p] = nxt[p];
-        }
-        cp_async_wait<0>();
-        if (ok && n_my > 0) {
-            fence_async_proxy();
-            tma::mbar_arrive(&sy.full[(n_my - 1) % STAGES]);
-        }
-    } else if (warp == LOADER_WARPS) {
-        // ------------------------------------------------------------------ W loads and MMA issue
-        if (lane == 0) {
-            tma::prefetch_map(&mapW);
-            const uint32_t w_addr = tma::smem_u32(Ws), i_addr = tma::smem_u32(Is);
-            const uint32_t idesc = tc::instr_desc(128, 128);
-            int cur_u = -1;
-            uint32_t n_units = 0;
-            for (int i = 0; i < n_my; ++i) {
-                const int s = i % STAGES, round = i / STAGES;
-                const long long gt = gt_lo + i;
-                const int u = (int)(gt / P.tpu);
-                if (u != cur_u) {
-                    // the previous unit's MMAs must have read W before it is replaced
-                    if (n_units > 0 && !tma::mbar_wait(&sy.w_empty, (n_units - 1) & 1, fault, 42)) break;
-                    tma::mbar_expect_tx(&sy.w_full, OPERAND_BYTES);
-                    tma::load_3d(Ws, &mapW, 0, 0, u % P.LH, &sy.w_full);
-                    tma::load_3d(Ws + BOX_BYTES, &mapW, 64, 0, u % P.LH, &sy.w_full);
-                    if (!tma::mbar_wait(&sy.w_full, n_units & 1, fault, 43)) break;
-                    cur_u = u;
-                    ++n_units;
-                }
-                if (!tma::mbar_wait(&sy.full[s], round & 1, fault, 44)) break;
-                tc::fence_after_sync();
-                const uint32_t k_addr = tma::smem_u32(stage0 + s * STAGE_BYTES), v_addr = k_addr + OPERAND_BYTES;
-                const uint32_t d = sy.tmem_base + s * 128;
-#pragma unroll
-                for (int ks = 0; ks < 8; ++ks) {
-                    const uint32_t o = (ks >> 2) * BOX_BYTES + (ks & 3) * 32;
-                    tc::mma_bf16(d, tc::smem_desc(v_addr + o), tc::smem_desc(i_addr + o), idesc, ks > 0);
-                }
-#pragma unroll
-                for (int ks = 0; ks < 8; ++ks) {
-                    const uint32_t o = (ks >> 2) * BOX_BYTES + (ks & 3) * 32;
-                    tc::mma_bf16(d, tc::smem_desc(k_addr + o), tc::smem_desc(w_addr + o), idesc, 1u);
-                }
-                tc::mma_commit(&sy.done[s]);
-                const bool last_of_unit = (i + 1 == n_my) || (int)((gt + 1) / P.tpu) != u;
-                if (last_of_unit) tc::mma_commit(&sy.w_empty);
-            }
-        }
-    } else {
-        // ------------------------------------------------------------------ epilogue
-        const int quarter = warp & 3;                       // TMEM lanes this warp may read: 32 (warp % 4) ..
-        const int r = quarter * 32 + lane;
-        const uint32_t lane_addr = sy.tmem_base + ((uint32_t)(quarter * 32) << 16);
-        for (int i = 0; i < n_my; ++i) {
-            const int s = i % STAGES, round = i / STAGES;
-            if (!tma::mbar_wait_warp(&sy.done[s], round & 1, fault, 45)) break;
-            tc::fence_after_sync();
-            const long long gt = gt_lo + i;
-            const int u = (int)(gt / P.tpu), t = (int)(gt - (long long)u * P.tpu);
-            uint32_t ra[32], rb[32];
-            const uint32_t taddr = lane_addr + s * 128;
-            tc::tmem_ld32(taddr, ra);
-            float e0 = 0.f, e1 = 0.f, e2 = 0.f, e3 = 0.f;
-#pragma unroll
-            for (int ch = 0; ch < 4; ++ch) {
-                uint32_t (&cur)[32] = (ch & 1) ? rb : ra;
-                uint32_t (&nxt)[32] = (ch & 1) ? ra : rb;
-                tc::tmem_ld_wait(cur);
-                if (ch < 3) tc::tmem_ld32(taddr + (ch + 1) * 32, nxt);
-#pragma unroll
-                for (int j = 0; j < 32; j += 4) {
-                    const float a = __uint_as_float(cur[j]), b = __uint_as_float(cur[j + 1]);
-                    const float c2 = __uint_as_float(cur[j + 2]), d2 = __uint_as_float(cur[j + 3]);
-                    e0 = fmaf(a, a, e0); e1 = fmaf(b, b, e1); e2 = fmaf(c2, c2, e2); e3 = fmaf(d2, d2, e3);
-                }
-            }
-            tc::fence_before_sync();
-            __syncwarp();
-            if (lane == 0) tma::mbar_arrive(&sy.empty[s]);
-            const int row = t * TILE + r;
-            if (row < P.n_idx) eps[(size_t)u * P.n_idx + row] = (e0 + e1) + (e2 + e3);
-        }
-    }
-    tc::fence_before_sync();
-    __syncthreads();
-    if (warp == LOADER_WARPS) {
-        __syncwarp();
-        tc::fence_after_sync();
-        tc::tmem_dealloc(sy.tmem_base, TMEM_COLS);
-    }
-}
-
-// ---------------------------------------------------------------------------------------------
-// The same residual with RoPE decoupling: the regressor sees the key turned back by its position
-// (the token index itself), channel c pairing with c + 64.  The turned key is no longer a bf16
-// number, so it goes to the tensor cores as a bf16 pair hi + lo (two chains over the same W),
-// which keeps it to 2^-17 relative; the value rows stay out of the MMA and are subtracted in the
-// epilogue.  Per 128-row tile:  D = K_hi W^T + K_lo W^T,  eps = sum_n (D[.][n] - v[n])^2.
-//   warps 0-7   loaders: each thread gathers, for its rows, the 16-byte chunk qc of both key halves
-//               (channels 8 qc.. and 64 + 8 qc..: the eight pairs it will turn) and two chunks of V,
-//               and, once its own copies of the previous tile have landed, turns the pairs back and
-//               writes hi in place and lo into the second operand tile
-//   warp  8     MMA issuer, TMEM owner, W loads
-//   warps 9-12  epilogue: thread = row; reads its accumulator row from TMEM and its value row from
-//               shared memory
 constexpr int R_LOADER_WARPS = 8;
 constexpr int R_THREADS = 32 * (R_LOADER_WARPS + 1 + EPI_WARPS);
-constexpr int R_STAGE_BYTES = 3 * OPERAND_BYTES;            // K hi | K lo | V
-constexpr int R_SMEM_BYTES = STAGES * R_STAGE_BYTES + OPERAND_BYTES + 1024;     // + W
+template <bool ROPE> struct RCfg {
+    static constexpr int STAGES = ROPE ? 2 : 3;
+    static constexpr int STAGE_BYTES = (ROPE ? 3 : 2) * OPERAND_BYTES;
+    static constexpr int V_OFFSET = (ROPE ? 2 : 1) * OPERAND_BYTES;
+    static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + OPERAND_BYTES + 1024;     // + W
+    static constexpr int TMEM_COLS = ROPE ? 256 : 512;          // one 128-column accumulator per stage
+};
+struct RSync {
+    uint64_t full[3], done[3], empty[3];
+    uint64_t w_full, w_empty;
+    uint32_t tmem_base;
+};
 
+// grid: min(148, n_tiles) blocks, R_THREADS threads, RCfg<ROPE>::SMEM_BYTES dynamic shared memory.
+template <bool ROPE>
 __global__ void __launch_bounds__(R_THREADS, 1)
-residual_tc_rope(const __nv_bfloat16* __restrict__ K, const __nv_bfloat16* __restrict__ V,
+residual_tc(const __nv_bfloat16* __restrict__ K, const __nv_bfloat16* __restrict__ V,
                  const __grid_constant__ CUtensorMap mapW, const int32_t* __restrict__ idx, const Params P,
                  const __grid_constant__ RopePhases rope, float* __restrict__ eps, int* __restrict__ fault) {
     extern __shared__ unsigned char smem_raw[];
-    __shared__ Sync sy;
+    __shared__ RSync sy;
+    constexpr int STAGES = RCfg<ROPE>::STAGES, R_STAGE_BYTES = RCfg<ROPE>::STAGE_BYTES, TMEM_COLS = RCfg<ROPE>::TMEM_COLS;
     __shared__ unsigned long long phase_s[64];
     unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     unsigned char* stage0 = smem;
@@ -346,7 +169,7 @@ residual_tc_rope(const __nv_bfloat16* __restrict__ K, const __nv_bfloat16* __res
             if (round > 0 && !tma::mbar_wait(&sy.empty[s], (round - 1) & 1, fault, 46)) { ok = false; break; }
             const int u = (int)((gt_lo + i) / P.tpu);
             const uint32_t kdst = tma::smem_u32(stage0 + s * R_STAGE_BYTES) + dst_thread;
-            const uint32_t vdst = kdst + 2 * OPERAND_BYTES;
+            const uint32_t vdst = kdst + RCfg<ROPE>::V_OFFSET;
             const __nv_bfloat16* Ku = K + (size_t)u * P.N * 128 + qc * 8;
             const __nv_bfloat16* Vu = V + (size_t)u * P.N * 128 + qc * 8;
 #pragma unroll
@@ -360,15 +183,29 @@ residual_tc_rope(const __nv_bfloat16* __restrict__ K, const __nv_bfloat16* __res
                 cp_async16(vdst + BOX_BYTES + p * 4096, Vu + ro + 64, nb);
             }
             cp_async_commit();
-            if (i > 0) {                                 // this thread's copies of the previous tile have landed
-                cp_async_wait<1>();
-                turn_back((i - 1) % STAGES, prev);
+            if (ROPE) {
+                if (i > 0) {                             // this thread's copies of the previous tile have landed
+                    cp_async_wait<1>();
+                    turn_back((i - 1) % STAGES, prev);
+                }
+            } else if (i >= 2) {                         // ... of the tile before the previous one
+                cp_async_wait<2>();
+                fence_async_proxy();
+                tma::mbar_arrive(&sy.full[(i - 2) % STAGES]);
             }
 #pragma unroll
             for (int p = 0; p < 4; ++p) { prev[p] = cur[p]; cur[p] = nxt[p]; }
         }
-        cp_async_wait<0>();
-        if (ok && n_my > 0) turn_back((n_my - 1) % STAGES, prev);
+        if (ROPE) {
+            cp_async_wait<0>();
+            if (ok && n_my > 0) turn_back((n_my - 1) % STAGES, prev);
+        } else if (ok) {
+            if (n_my > 1) { cp_async_wait<1>(); fence_async_proxy(); tma::mbar_arrive(&sy.full[(n_my - 2) % STAGES]); }
+            cp_async_wait<0>();
+            if (n_my > 0) { fence_async_proxy(); tma::mbar_arrive(&sy.full[(n_my - 1) % STAGES]); }
+        } else {
+            cp_async_wait<0>();
+        }
     } else if (warp == R_LOADER_WARPS) {
         // ------------------------------------------------------------------ W loads and MMA issue
         if (lane == 0) {
@@ -399,10 +236,12 @@ residual_tc_rope(const __nv_bfloat16* __restrict__ K, const __nv_bfloat16* __res
                     const uint32_t o = (ks >> 2) * BOX_BYTES + (ks & 3) * 32;
                     tc::mma_bf16(d, tc::smem_desc(hi_addr + o), tc::smem_desc(w_addr + o), idesc, ks > 0);
                 }
+                if (ROPE) {
 #pragma unroll
-                for (int ks = 0; ks < 8; ++ks) {
-                    const uint32_t o = (ks >> 2) * BOX_BYTES + (ks & 3) * 32;
-                    tc::mma_bf16(d, tc::smem_desc(lo_addr + o), tc::smem_desc(w_addr + o), idesc, 1u);
+                    for (int ks = 0; ks < 8; ++ks) {
+                        const uint32_t o = (ks >> 2) * BOX_BYTES + (ks & 3) * 32;
+                        tc::mma_bf16(d, tc::smem_desc(lo_addr + o), tc::smem_desc(w_addr + o), idesc, 1u);
+                    }
                 }
                 tc::mma_commit(&sy.done[s]);
                 const bool last_of_unit = (i + 1 == n_my) || (int)((gt + 1) / P.tpu) != u;
@@ -423,7 +262,7 @@ residual_tc_rope(const __nv_bfloat16* __restrict__ K, const __nv_bfloat16* __res
             tc::fence_after_sync();
             const long long gt = gt_lo + i;
             const int u = (int)(gt / P.tpu), t = (int)(gt - (long long)u * P.tpu);
-            const uint32_t v_addr = tma::smem_u32(stage0 + s * R_STAGE_BYTES) + 2 * OPERAND_BYTES + v_thread;
+            const uint32_t v_addr = tma::smem_u32(stage0 + s * R_STAGE_BYTES) + RCfg<ROPE>::V_OFFSET + v_thread;
             uint32_t ra[32], rb[32];
             const uint32_t taddr = lane_addr + s * 128;
             tc::tmem_ld32(taddr, ra);

@@ -401,9 +401,11 @@ static vector_status launch_residual_tc(const Dims& dm, const void* K, const voi
     if (n_idx == 0) return VECTOR_OK;
     static PerDeviceOnce once;
     if (once.first()) {
-        cudaError_t e = cudaFuncSetAttribute(rtc::residual_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, rtc::SMEM_BYTES);
+        cudaError_t e = cudaFuncSetAttribute(rtc::residual_tc<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                             rtc::RCfg<false>::SMEM_BYTES);
         if (e == cudaSuccess)
-            e = cudaFuncSetAttribute(rtc::residual_tc_rope, cudaFuncAttributeMaxDynamicSharedMemorySize, rtc::R_SMEM_BYTES);
+            e = cudaFuncSetAttribute(rtc::residual_tc<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                     rtc::RCfg<true>::SMEM_BYTES);
         if (e != cudaSuccess) { once.undo(); VEC_CUDA_CHECK(e); }
     }
     int* fault = kernel_fault_address();
@@ -415,14 +417,14 @@ static vector_status launch_residual_tc(const Dims& dm, const void* K, const voi
     P.tpu = (int)((n_idx + rtc::TILE - 1) / rtc::TILE);
     P.n_tiles = (long long)dm.U * P.tpu;
     const int blocks = (int)(P.n_tiles < 148 ? P.n_tiles : 148);
+    RopePhases ph = {};
     if (dm.rope) {
-        RopePhases ph;
         rope_phases(dm.theta, 128, &ph);
-        rtc::residual_tc_rope<<<blocks, rtc::R_THREADS, rtc::R_SMEM_BYTES, st>>>((const __nv_bfloat16*)K, (const __nv_bfloat16*)V,
-                                                                                 mapW, idx, P, ph, eps, fault);
+        rtc::residual_tc<true><<<blocks, rtc::R_THREADS, rtc::RCfg<true>::SMEM_BYTES, st>>>(
+            (const __nv_bfloat16*)K, (const __nv_bfloat16*)V, mapW, idx, P, ph, eps, fault);
     } else {
-        rtc::residual_tc<<<blocks, rtc::THREADS, rtc::SMEM_BYTES, st>>>((const __nv_bfloat16*)K, (const __nv_bfloat16*)V, mapW,
-                                                                        idx, P, eps, fault);
+        rtc::residual_tc<false><<<blocks, rtc::R_THREADS, rtc::RCfg<false>::SMEM_BYTES, st>>>(
+            (const __nv_bfloat16*)K, (const __nv_bfloat16*)V, mapW, idx, P, ph, eps, fault);
     }
     VEC_LAUNCH_CHECK();
     return VECTOR_OK;
