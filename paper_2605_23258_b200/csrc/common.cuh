@@ -45,11 +45,19 @@ __device__ __forceinline__ void rope_cos_sin(double pos, double inv_freq, float&
 }
 // The same for the tuned kernels, from the pair's 64-bit phase (turns per position as a fraction
 // of 2^64, f = its low and high words): the top 32 bits of pos * phase modulo 2^64 are the angle
-// in turns modulo one, exact to 2^-32 of a turn for any 32-bit position; its top 23 bits make a
-// float in [1, 2), shifted by half a turn so that the result lies in [-pi, pi).
+// in turns modulo one, exact to 2^-32 of a turn for any 32-bit position; read as a signed number
+// they lie in [-1/2, 1/2), so the angle handed to sine and cosine lies in [-pi, pi).
 __device__ __forceinline__ void rope_phase_cos_sin(uint32_t pos, uint2 f, float& cs, float& sn) {
-    const uint32_t turns = pos * f.y + __umulhi(pos, f.x) + 0x80000000u;
-    const float ang = fmaf(__uint_as_float((turns >> 9) | 0x3f800000u), 6.283185307179586f, -9.42477796076938f);
+    const uint32_t turns = pos * f.y + __umulhi(pos, f.x);
+    const float ang = (float)(int)turns * 1.4629180792671596e-9f;      // 2 pi / 2^32
+    __sincosf(ang, &sn, &cs);
+}
+// A shorter form for where issue slots are what costs (decode): the phase rounded to 32 bits.  The
+// 32-bit product pos * phase32 is the angle in turns modulo one, taken as a signed number in
+// [-1/2, 1/2); the phase's rounding leaves pos * 2^-33 of a turn (1e-4 rad at position 131072,
+// 8e-4 rad at 2^20), well under the fp16 spacing of the turned key.
+__device__ __forceinline__ void rope_phase32_cos_sin(uint32_t pos, uint32_t phase32, float& cs, float& sn) {
+    const float ang = (float)(int)(pos * phase32) * 1.4629180792671596e-9f;      // 2 pi / 2^32
     __sincosf(ang, &sn, &cs);
 }
 // Inverse frequencies theta^(-2c/d), c < d/2, into shared memory (fp64); callers synchronise.

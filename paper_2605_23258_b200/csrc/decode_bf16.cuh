@@ -135,13 +135,13 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
 // channels 0-63 | 64-127) are turned back by their positions, in place, and left there as fp16 (a
 // turned key is not a bf16 number; eleven bits keep the key sum within the tolerance of the output,
 // eight do not; |k| beyond 65504 saturates).  Channel c pairs with
-// c + 64; the angle is position * theta^(-2c/128), taken as the top bits of the 64-bit product of
-// the position and the per-channel phase, so that it is exact modulo one turn.  pos16: lane l
+// c + 64; the angle is position * theta^(-2c/128), taken as the 32-bit product of the position and
+// the per-channel phase (turns per position as a fraction of 2^32), which is the angle modulo one turn.  pos16: lane l
 // holds the position of row 16 member + (l & 15).
 __device__ __forceinline__ void derotate_rows(uint32_t kbase, int nrows, int member, uint32_t pos16,
-                                              const unsigned long long* phase_s, int lane) {
+                                              const uint32_t* phase_s, int lane) {
     const int qc = lane & 7;                                        // 16-byte chunk: channel pairs 8 qc .. 8 qc + 7
-    const uint2* phase2 = reinterpret_cast<const uint2*>(phase_s) + qc * 8;     // (low, high) words
+    const uint32_t* phase = phase_s + qc * 8;
 #pragma unroll 1
     for (int j = 0; j < 4; j += 2) {
         // two rows per round, the loads of both ahead of the stores
@@ -171,7 +171,7 @@ __device__ __forceinline__ void derotate_rows(uint32_t kbase, int nrows, int mem
                     const float x = __uint_as_float(h ? (xs[u][e] & 0xffff0000u) : (xs[u][e] << 16));
                     const float y = __uint_as_float(h ? (ys[u][e] & 0xffff0000u) : (ys[u][e] << 16));
                     float sn, cs;
-                    rope_phase_cos_sin(pos[u], phase2[2 * e + h], cs, sn);
+                    rope_phase32_cos_sin(pos[u], phase[2 * e + h], cs, sn);
                     xo[h] = fmaf(x, cs, y * sn);
                     yo[h] = fmaf(y, cs, -x * sn);
                 }
@@ -211,8 +211,8 @@ decode_stream_bf16_d128(const __nv_bfloat16* __restrict__ q, const __grid_consta
                         int* __restrict__ fault, const int32_t* __restrict__ apx_pos, long long cap_apx,
                         const __grid_constant__ RopePhases rope) {
     extern __shared__ unsigned char smem_raw[];
-    __shared__ unsigned long long phase_s[ROPE ? 64 : 1];
-    if (ROPE && threadIdx.x < 64) phase_s[threadIdx.x] = rope.phase[threadIdx.x];
+    __shared__ uint32_t phase_s[ROPE ? 64 : 1];          // the phases rounded to 32 bits
+    if (ROPE && threadIdx.x < 64) phase_s[threadIdx.x] = (uint32_t)((rope.phase[threadIdx.x] + 0x80000000ull) >> 32);
     __shared__ volatile int team_ok[CONSUMER_WARPS];     // RoPE: the owner's go / no-go for the tile at hand
     __shared__ __align__(8) uint64_t full_bar[SLOTS];
     __shared__ __align__(8) uint64_t empty_bar[SLOTS];

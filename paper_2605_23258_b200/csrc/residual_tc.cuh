@@ -134,7 +134,7 @@ residual_tc(const __nv_bfloat16* __restrict__ K, const __nv_bfloat16* __restrict
                 const uint32_t tok = pos[p] >= 0 ? (uint32_t)pos[p] : 0u;      // rows past the list are zeros
 #pragma unroll
                 for (int e = 0; e < 4; ++e) {
-                    float xo[2], yo[2], xh[2], yh[2];
+                    float xo[2], yo[2];
 #pragma unroll
                     for (int h = 0; h < 2; ++h) {
                         const float x = __uint_as_float(h ? (xs[e] & 0xffff0000u) : (xs[e] << 16));
@@ -143,13 +143,12 @@ residual_tc(const __nv_bfloat16* __restrict__ K, const __nv_bfloat16* __restrict
                         rope_phase_cos_sin(tok, fr[2 * e + h], cs, sn);
                         xo[h] = fmaf(x, cs, y * sn);
                         yo[h] = fmaf(y, cs, -x * sn);
-                        xh[h] = __bfloat162float(__float2bfloat16_rn(xo[h]));
-                        yh[h] = __bfloat162float(__float2bfloat16_rn(yo[h]));
                     }
-                    xs[e] = pack2_bf16(xh[0], xh[1]);
-                    ys[e] = pack2_bf16(yh[0], yh[1]);
-                    xl[e] = pack2_bf16(xo[0] - xh[0], xo[1] - xh[1]);
-                    yl[e] = pack2_bf16(yo[0] - yh[0], yo[1] - yh[1]);
+                    // hi = the pair rounded to bf16, lo = what the rounding left, again as bf16
+                    xs[e] = pack2_bf16(xo[0], xo[1]);
+                    ys[e] = pack2_bf16(yo[0], yo[1]);
+                    xl[e] = pack2_bf16(xo[0] - __uint_as_float(xs[e] << 16), xo[1] - __uint_as_float(xs[e] & 0xffff0000u));
+                    yl[e] = pack2_bf16(yo[0] - __uint_as_float(ys[e] << 16), yo[1] - __uint_as_float(ys[e] & 0xffff0000u));
                 }
                 asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};\n" ::"r"(hi0 + p * 4096), "r"(xs[0]), "r"(xs[1]), "r"(xs[2]), "r"(xs[3]) : "memory");
                 asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};\n" ::"r"(hi0 + BOX_BYTES + p * 4096), "r"(ys[0]), "r"(ys[1]), "r"(ys[2]), "r"(ys[3]) : "memory");
