@@ -37,6 +37,7 @@
 
 #include "common.cuh"
 #include "internal.h"
+#include "tcgen05.cuh"
 #include "tma.cuh"
 
 namespace vec {
@@ -141,7 +142,9 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
 __device__ __forceinline__ void derotate_rows(uint32_t kbase, int nrows, int member, uint32_t pos16,
                                               const uint32_t* phase_s, int lane) {
     const int qc = lane & 7;                                        // 16-byte chunk: channel pairs 8 qc .. 8 qc + 7
-    const uint32_t* phase = phase_s + qc * 8;
+    uint32_t phase[8];                                              // this lane's eight channel pairs
+#pragma unroll
+    for (int c = 0; c < 8; ++c) phase[c] = phase_s[qc * 8 + c];
 #pragma unroll 1
     for (int j = 0; j < 4; j += 2) {
         // two rows per round, the loads of both ahead of the stores
@@ -165,16 +168,18 @@ __device__ __forceinline__ void derotate_rows(uint32_t kbase, int nrows, int mem
         for (int u = 0; u < 2; ++u) {
 #pragma unroll
             for (int e = 0; e < 4; ++e) {
-                float xo[2], yo[2];
+                float x[2], y[2], cs[2], sn[2], xo[2], yo[2];
 #pragma unroll
                 for (int h = 0; h < 2; ++h) {
-                    const float x = __uint_as_float(h ? (xs[u][e] & 0xffff0000u) : (xs[u][e] << 16));
-                    const float y = __uint_as_float(h ? (ys[u][e] & 0xffff0000u) : (ys[u][e] << 16));
-                    float sn, cs;
-                    rope_phase32_cos_sin(pos[u], phase[2 * e + h], cs, sn);
-                    xo[h] = fmaf(x, cs, y * sn);
-                    yo[h] = fmaf(y, cs, -x * sn);
+                    x[h] = __uint_as_float(h ? (xs[u][e] & 0xffff0000u) : (xs[u][e] << 16));
+                    y[h] = __uint_as_float(h ? (ys[u][e] & 0xffff0000u) : (ys[u][e] << 16));
+                    rope_phase32_cos_sin(pos[u], phase[2 * e + h], cs[h], sn[h]);
                 }
+                // both pairs of the word at once on the packed FMA path
+                const uint64_t x2 = tc::pack2(x[0], x[1]), y2 = tc::pack2(y[0], y[1]);
+                const uint64_t c2 = tc::pack2(cs[0], cs[1]), s2 = tc::pack2(sn[0], sn[1]);
+                tc::unpack2(tc::fma2(x2, c2, tc::mul2(y2, s2)), xo[0], xo[1]);
+                tc::unpack2(tc::fma2(y2, c2, tc::mul2(x2, tc::pack2(-sn[0], -sn[1]))), yo[0], yo[1]);
                 xs[u][e] = pack_f16(xo[0], xo[1]);
                 ys[u][e] = pack_f16(yo[0], yo[1]);
             }

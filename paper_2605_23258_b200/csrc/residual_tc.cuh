@@ -134,16 +134,18 @@ residual_tc(const __nv_bfloat16* __restrict__ K, const __nv_bfloat16* __restrict
                 const uint32_t tok = pos[p] >= 0 ? (uint32_t)pos[p] : 0u;      // rows past the list are zeros
 #pragma unroll
                 for (int e = 0; e < 4; ++e) {
-                    float xo[2], yo[2];
+                    float x[2], y[2], cs[2], sn[2], xo[2], yo[2];
 #pragma unroll
                     for (int h = 0; h < 2; ++h) {
-                        const float x = __uint_as_float(h ? (xs[e] & 0xffff0000u) : (xs[e] << 16));
-                        const float y = __uint_as_float(h ? (ys[e] & 0xffff0000u) : (ys[e] << 16));
-                        float cs, sn;
-                        rope_phase_cos_sin(tok, fr[2 * e + h], cs, sn);
-                        xo[h] = fmaf(x, cs, y * sn);
-                        yo[h] = fmaf(y, cs, -x * sn);
+                        x[h] = __uint_as_float(h ? (xs[e] & 0xffff0000u) : (xs[e] << 16));
+                        y[h] = __uint_as_float(h ? (ys[e] & 0xffff0000u) : (ys[e] << 16));
+                        rope_phase_cos_sin(tok, fr[2 * e + h], cs[h], sn[h]);
                     }
+                    // both pairs of the word at once on the packed FMA path
+                    const uint64_t x2 = tc::pack2(x[0], x[1]), y2 = tc::pack2(y[0], y[1]);
+                    const uint64_t c2 = tc::pack2(cs[0], cs[1]), s2 = tc::pack2(sn[0], sn[1]);
+                    tc::unpack2(tc::fma2(x2, c2, tc::mul2(y2, s2)), xo[0], xo[1]);
+                    tc::unpack2(tc::fma2(y2, c2, tc::mul2(x2, tc::pack2(-sn[0], -sn[1]))), yo[0], yo[1]);
                     // hi = the pair rounded to bf16, lo = what the rounding left, again as bf16
                     xs[e] = pack2_bf16(xo[0], xo[1]);
                     ys[e] = pack2_bf16(yo[0], yo[1]);
