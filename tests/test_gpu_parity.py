@@ -360,6 +360,10 @@ def test_pipeline_with_rotary_keys(oracle):
     wl = synth.shrink(synth.WORKLOADS[1], N=1200, n_kv_heads=2, n_q_heads=8, n_calib=2048)
     _run_pipeline_case(oracle, wl, 30, theta=10000.0)
     _run_pipeline_case(oracle, synth.shrink(synth.WORKLOADS[0], N=700), 25, decode_steps=2, theta=500.0)    # fp32, d = 64
+    # eight query heads per KV head, window 128, pools that end inside a 64-key half
+    wl8 = synth.shrink(synth.WORKLOADS[4], N=3000, n_layers=2, n_kv_heads=1, n_q_heads=8, n_calib=2048)
+    _run_pipeline_case(oracle, wl8, 12, theta=500000.0)
+    _run_pipeline_case(oracle, wl8, 31, theta=500000.0)
 
 
 @pytest.mark.parametrize("base,over,theta", [(1, {"N": 3000, "n_kv_heads": 2, "n_q_heads": 8}, 10000.0),
