@@ -37,6 +37,7 @@ constexpr int SEL_BINS = 2048;      // digits of 11, 11 and 10 bits
 struct SelectScratch {
     int hist[SEL_BINS];
     int bc[2];
+    int part[32];                 // per-warp bin sums of pick_bin
     int n_cand, overflow;
     int32_t cand[CAND_CAP];       // indices of the elements that share the k-th key's leading 11 bits
     uint32_t sel_mask[MASK_GROUPS];   // per group of 32 elements: those above the k-th key
@@ -44,29 +45,35 @@ struct SelectScratch {
     OrderedScratch os;
 };
 
-// Warp 0: the bin of hist[0..SEL_BINS), counted from the top, in which the cumulative count reaches
-// `remaining` (-> bc[0]) and the rank wanted inside that bin, 1-based (-> bc[1]).
-__device__ __forceinline__ void pick_bin(const int* hist, int remaining, int* bc) {
-    constexpr int PER = SEL_BINS / 32;
-    if (threadIdx.x < 32) {
-        const int top = SEL_BINS - 1 - (int)threadIdx.x * PER;      // this lane's bins: top, top - 1, ..
-        int tot = 0;
-#pragma unroll 8
-        for (int j = 0; j < PER; ++j) tot += hist[top - j];
-        int inc = tot;
+// The bin of hist[0..SEL_BINS), counted from the top, in which the cumulative count reaches
+// `remaining` (-> bc[0]) and the rank wanted inside that bin, 1-based (-> bc[1]).  Every thread of
+// the block calls it (one block barrier inside; the caller synchronises before and after): warp w
+// sums the 64 bins below SEL_BINS - 64 w, every warp scans the 32 sums, and the one warp whose
+// range holds the answer finds the bin with two lane scans.
+static_assert(SEL_THREADS == 1024 && SEL_BINS == 2048, "one warp per 64 bins");
+__device__ __forceinline__ int lane_scan_incl(int v, int lane) {
 #pragma unroll
-        for (int o = 1; o < 32; o <<= 1) {
-            const int t = __shfl_up_sync(0xffffffffu, inc, o);
-            if ((int)threadIdx.x >= o) inc += t;
-        }
-        int cum = inc - tot;                            // count in the bins above this lane's
-        if (cum < remaining && inc >= remaining) {      // exactly one lane
-            for (int j = 0; j < PER; ++j) {
-                const int c = hist[top - j];
-                if (cum + c >= remaining) { bc[0] = top - j; bc[1] = remaining - cum; break; }
-                cum += c;
-            }
-        }
+    for (int o = 1; o < 32; o <<= 1) {
+        const int t = __shfl_up_sync(0xffffffffu, v, o);
+        if (lane >= o) v += t;
+    }
+    return v;
+}
+__device__ __forceinline__ void pick_bin(const int* hist, int remaining, int* bc, int* part) {
+    const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
+    const int top = SEL_BINS - 1 - wid * 64;                // this warp's bins: top, top - 1, .., top - 63
+    const int c0 = hist[top - lane], c1 = hist[top - 32 - lane];
+    const int tot = __reduce_add_sync(0xffffffffu, c0 + c1);
+    if (lane == 0) part[wid] = tot;
+    __syncthreads();
+    const int p = part[lane];
+    const int above = __shfl_sync(0xffffffffu, lane_scan_incl(p, lane) - p, wid);      // count in the warps above this one
+    if (above < remaining && above + tot >= remaining) {     // exactly one warp
+        const int r = remaining - above;
+        const int s0 = lane_scan_incl(c0, lane), tot0 = __shfl_sync(0xffffffffu, s0, 31);
+        const int s1 = tot0 + lane_scan_incl(c1, lane);
+        if (s0 - c0 < r && s0 >= r) { bc[0] = top - lane; bc[1] = r - (s0 - c0); }
+        if (s1 - c1 < r && s1 >= r) { bc[0] = top - 32 - lane; bc[1] = r - (s1 - c1); }
     }
 }
 
@@ -75,7 +82,7 @@ __device__ __forceinline__ void pick_bin(const int* hist, int remaining, int* bc
 // memory latency otherwise.
 template <bool SMALLEST>
 __device__ __forceinline__ void hist_pass_all(const float* __restrict__ vals, int n, int shift, uint32_t digit_mask,
-                                              uint32_t prefix, uint32_t mask, int* hist) {
+                                              uint32_t prefix, uint32_t mask, int* hist, uint32_t* stage = nullptr) {
     for (int base = 0; base < n; base += 8 * blockDim.x) {
         float v[8];
 #pragma unroll
@@ -87,6 +94,7 @@ __device__ __forceinline__ void hist_pass_all(const float* __restrict__ vals, in
         for (int j = 0; j < 8; ++j) {
             const int i = base + j * blockDim.x + threadIdx.x;
             const uint32_t key = select_image<SMALLEST>(v[j]);
+            if (stage && i < n) stage[i] = key;          // keep the image for the later passes
             hist_add(hist, (key >> shift) & digit_mask, i < n && (key & mask) == prefix);
         }
     }
@@ -109,9 +117,11 @@ __device__ __forceinline__ int ordered_chunk(int n, int nw) { return (((n + nw -
 // a second mask.  The per-piece counts and the emission in index order then need the masks only,
 // not the values.  Two fallbacks read the input again instead: more than CAND_CAP candidates
 // (pass 3 and the classification walk the input), more than 32 MASK_GROUPS elements (the masks are
-// not kept).
+// not kept).  With `stage` (n words of shared memory) pass 1 also keeps the images there and the
+// later passes never go back to global memory.
 template <bool SMALLEST, typename Emit>
-__device__ __forceinline__ void select_emit(const float* __restrict__ vals, int n, int k, bool any, SelectScratch& S, Emit emit) {
+__device__ __forceinline__ void select_emit(const float* __restrict__ vals, int n, int k, bool any, SelectScratch& S, Emit emit,
+                                            uint32_t* stage = nullptr) {
     const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5, nw = blockDim.x >> 5;
     const unsigned lt = (1u << lane) - 1u;
     const int per_w = ordered_chunk(n, nw);
@@ -127,9 +137,9 @@ __device__ __forceinline__ void select_emit(const float* __restrict__ vals, int 
         for (int b = threadIdx.x; b < SEL_BINS; b += blockDim.x) S.hist[b] = 0;
         if (threadIdx.x == 0) { S.n_cand = 0; S.overflow = 0; }
         __syncthreads();
-        hist_pass_all<SMALLEST>(vals, n, 21, 2047u, 0u, 0u, S.hist);
+        hist_pass_all<SMALLEST>(vals, n, 21, 2047u, 0u, 0u, S.hist, stage);
         __syncthreads();
-        pick_bin(S.hist, k, S.bc);
+        pick_bin(S.hist, k, S.bc, S.part);
         __syncthreads();
         const uint32_t bin1 = (uint32_t)S.bc[0];
         int remaining = S.bc[1];
@@ -138,14 +148,17 @@ __device__ __forceinline__ void select_emit(const float* __restrict__ vals, int 
         for (int b = threadIdx.x; b < SEL_BINS; b += blockDim.x) S.hist[b] = 0;
         __syncthreads();
         for (int base = w0; base < w1; base += 128) {
-            float v[4];
+            uint32_t kv[4];
 #pragma unroll
-            for (int j = 0; j < 4; ++j) v[j] = base + 32 * j + lane < w1 ? vals[base + 32 * j + lane] : 0.f;
+            for (int j = 0; j < 4; ++j) {
+                const int i = base + 32 * j + lane;
+                kv[j] = i >= w1 ? 0u : stage ? stage[i] : select_image<SMALLEST>(vals[i]);
+            }
 #pragma unroll
             for (int j = 0; j < 4; ++j) {
                 const int i = base + 32 * j + lane;
                 const bool in = i < w1;
-                const uint32_t key = select_image<SMALLEST>(v[j]);
+                const uint32_t key = kv[j];
                 const uint32_t d1 = key >> 21;
                 if (masked) {
                     const unsigned gb = __ballot_sync(0xffffffffu, in && d1 > bin1);
@@ -160,7 +173,7 @@ __device__ __forceinline__ void select_emit(const float* __restrict__ vals, int 
             }
         }
         __syncthreads();
-        pick_bin(S.hist, remaining, S.bc);
+        pick_bin(S.hist, remaining, S.bc, S.part);
         __syncthreads();
         uint32_t prefix = (bin1 << 21) | ((uint32_t)S.bc[0] << 10);
         const uint32_t mask = 0xfffffc00u;
@@ -173,14 +186,14 @@ __device__ __forceinline__ void select_emit(const float* __restrict__ vals, int 
         __syncthreads();
         if (listed) {
             for (int j = threadIdx.x; j < n_cand; j += blockDim.x) {
-                const uint32_t key = select_image<SMALLEST>(vals[S.cand[j]]);
+                const uint32_t key = stage ? stage[S.cand[j]] : select_image<SMALLEST>(vals[S.cand[j]]);
                 hist_add(S.hist, key & 1023, (key & mask) == prefix);
             }
         } else {
             hist_pass_all<SMALLEST>(vals, n, 0, 1023u, prefix, mask, S.hist);
         }
         __syncthreads();
-        pick_bin(S.hist, remaining, S.bc);
+        pick_bin(S.hist, remaining, S.bc, S.part);
         __syncthreads();
         prefix |= (uint32_t)S.bc[0];
         remaining = S.bc[1];
@@ -191,7 +204,7 @@ __device__ __forceinline__ void select_emit(const float* __restrict__ vals, int 
         if (masked && listed) {
             for (int j = threadIdx.x; j < n_cand; j += blockDim.x) {
                 const int i = S.cand[j];
-                const uint32_t key = select_image<SMALLEST>(vals[i]);
+                const uint32_t key = stage ? stage[i] : select_image<SMALLEST>(vals[i]);
                 if (key > kth) atomicOr(&S.sel_mask[i >> 5], 1u << (i & 31));
                 else if (key == kth) atomicOr(&S.tie_mask[i >> 5], 1u << (i & 31));
             }
@@ -299,12 +312,13 @@ pool_select_kernel(const float* __restrict__ scores, int64_t N, int n_pool, int3
     select_emit<false>(s, n, n_pool, true, S, [&](int i, bool chosen, int pos) { if (chosen) out[pos] = i; });
 }
 
-// Step 3.  grid (U), SEL_THREADS threads.
+// Step 3.  grid (U), SEL_THREADS threads; dynamic shared memory: n_pool words (stage = 1) or none.
 __global__ void __launch_bounds__(SEL_THREADS, 2)
 truncate_kernel(const float* __restrict__ eps, const int32_t* __restrict__ pool_idx, int64_t N, int n_pool,
                 int n_apx, uint8_t* __restrict__ tier, int32_t* __restrict__ ret_idx,
-                int32_t* __restrict__ apx_idx) {
+                int32_t* __restrict__ apx_idx, int stage) {
     __shared__ SelectScratch S;
+    extern __shared__ uint32_t staged_keys[];        // n_pool words when the launch gave them, else none
     const int u = blockIdx.x;
     const float* e = eps + (size_t)u * n_pool;
     const int32_t* pool = pool_idx + (size_t)u * n_pool;
@@ -322,7 +336,7 @@ truncate_kernel(const float* __restrict__ eps, const int32_t* __restrict__ pool_
         const int32_t token = pool[p];
         if (is_apx) { ao[pos] = token; tr[token] = 1; }
         else        { ro[pos] = token; tr[token] = 2; }
-    });
+    }, stage ? staged_keys : nullptr);
 }
 
 // Step 2 on CUDA cores.  grid (ceil(n_idx / 64), U), 256 threads; W^T staged in
@@ -440,6 +454,25 @@ static vector_status residual_dispatch(const Dims& dm, const void* K, const void
                       : launch_residual<__nv_bfloat16, 128>(dm, K, V, W, N, idx, n_idx, eps, st);
 }
 
+// Residual lists up to this length are kept in shared memory by the truncation kernel (two blocks
+// per SM stay resident).
+constexpr int TRUNC_STAGE_MAX = 16384;
+static vector_status launch_truncate(const Dims& dm, const vector_budget* budget, const float* eps, const int32_t* pool,
+                                     uint8_t* tier, int32_t* ret_idx, int32_t* apx_idx, cudaStream_t st) {
+    const int stage = budget->n_pool <= TRUNC_STAGE_MAX ? 1 : 0;
+    const size_t smem = stage ? (size_t)budget->n_pool * sizeof(uint32_t) : 0;
+    static PerDeviceOnce once;
+    if (once.first()) {
+        const cudaError_t e = cudaFuncSetAttribute(truncate_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                                   TRUNC_STAGE_MAX * (int)sizeof(uint32_t));
+        if (e != cudaSuccess) { once.undo(); VEC_CUDA_CHECK(e); }
+    }
+    truncate_kernel<<<dm.U, SEL_THREADS, smem, st>>>(eps, pool, budget->n_tokens, (int)budget->n_pool, (int)budget->n_apx,
+                                                     tier, ret_idx, apx_idx, stage);
+    VEC_LAUNCH_CHECK();
+    return VECTOR_OK;
+}
+
 }  // namespace vec
 
 using namespace vec;
@@ -479,10 +512,7 @@ extern "C" vector_status vector_truncate(const vector_shape* shape, const vector
     if ((rc = check_budget(budget, dm.w)) != VECTOR_OK) return rc;
     if (!eps || !pool_idx || !tier) return VECTOR_ERR_NULL;
     if ((budget->n_ret > 0 && !ret_idx) || (budget->n_apx > 0 && !apx_idx)) return VECTOR_ERR_NULL;
-    truncate_kernel<<<dm.U, SEL_THREADS, 0, (cudaStream_t)stream>>>(
-        eps, pool_idx, budget->n_tokens, (int)budget->n_pool, (int)budget->n_apx, tier, ret_idx, apx_idx);
-    VEC_LAUNCH_CHECK();
-    return VECTOR_OK;
+    return launch_truncate(dm, budget, eps, pool_idx, tier, ret_idx, apx_idx, (cudaStream_t)stream);
 }
 
 extern "C" vector_status vector_route(const vector_shape* shape, const vector_budget* budget, const float* scores,
@@ -505,8 +535,5 @@ extern "C" vector_status vector_route(const vector_shape* shape, const vector_bu
     VEC_LAUNCH_CHECK();
     rc = residual_dispatch(dm, K, V, W, budget->n_tokens, pool, budget->n_pool, eps, st);
     if (rc != VECTOR_OK) return rc;
-    truncate_kernel<<<dm.U, SEL_THREADS, 0, st>>>(eps, pool, budget->n_tokens, (int)budget->n_pool,
-                                                  (int)budget->n_apx, tier, ret_idx, apx_idx);
-    VEC_LAUNCH_CHECK();
-    return VECTOR_OK;
+    return launch_truncate(dm, budget, eps, pool, tier, ret_idx, apx_idx, st);
 }
