@@ -86,6 +86,10 @@ residual_tc(const __nv_bfloat16* __restrict__ K, const __nv_bfloat16* __restrict
     const long long gt_hi = range_begin(blockIdx.x + 1, P.n_tiles, gridDim.x);
     const int n_my = (int)(gt_hi - gt_lo);
 
+    // Programmatic launches on both sides (inside vector_route): the kernel after this one may be
+    // scheduled as blocks here finish, and this one may have started before the kernel that writes
+    // idx has drained -- the loaders, the only readers of idx, wait for it below.
+    asm volatile("griddepcontrol.launch_dependents;\n" ::: "memory");
     if (tid < 64) phase_s[tid] = rope.phase[tid];
     if (tid == 0) {
 #pragma unroll
@@ -161,6 +165,7 @@ residual_tc(const __nv_bfloat16* __restrict__ K, const __nv_bfloat16* __restrict
             tma::mbar_arrive(&sy.full[s]);
         };
         bool ok = true;
+        asm volatile("griddepcontrol.wait;\n" ::: "memory");      // idx is complete and visible from here on
         if (n_my > 0) fetch_idx(0, cur);
 #pragma unroll
         for (int p = 0; p < 4; ++p) prev[p] = -1;

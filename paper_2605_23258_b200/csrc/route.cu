@@ -305,6 +305,9 @@ __device__ __forceinline__ void select_emit(const float* __restrict__ vals, int 
 __global__ void __launch_bounds__(SEL_THREADS, 2)
 pool_select_kernel(const float* __restrict__ scores, int64_t N, int n_pool, int32_t* __restrict__ pool_idx) {
     __shared__ SelectScratch S;
+    // inside vector_route the residual kernel is launched as a programmatic dependent: its blocks may
+    // take SMs as this grid's blocks leave them; it reads the index lists only after its own wait
+    asm volatile("griddepcontrol.launch_dependents;\n" ::: "memory");
     const int u = blockIdx.x, n = (int)N;
     const float* s = scores + (size_t)u * N;
     int32_t* out = pool_idx + (size_t)u * n_pool;
@@ -331,6 +334,9 @@ truncate_kernel(const float* __restrict__ eps, const int32_t* __restrict__ pool_
     } else {
         for (int64_t i = threadIdx.x; i < N; i += SEL_THREADS) tr[i] = 0;
     }
+    // everything above touches only the tier map; the residuals and the pool list belong to the
+    // kernels before this one (a no-op unless launched as a programmatic dependent)
+    asm volatile("griddepcontrol.wait;\n" ::: "memory");
     __syncthreads();
     select_emit<true>(e, n_pool, n_apx, n_apx > 0, S, [&](int p, bool is_apx, int pos) {
         const int32_t token = pool[p];
@@ -411,7 +417,7 @@ static vector_status launch_residual(const Dims& dm, const void* K, const void* 
 
 // bf16, head_dim 128: gather + tcgen05 residual kernel.
 static vector_status launch_residual_tc(const Dims& dm, const void* K, const void* V, const void* W, int64_t N,
-                                        const int32_t* idx, int64_t n_idx, float* eps, cudaStream_t st) {
+                                        const int32_t* idx, int64_t n_idx, float* eps, cudaStream_t st, bool dependent) {
     if (n_idx == 0) return VECTOR_OK;
     static PerDeviceOnce once;
     if (once.first()) {
@@ -432,21 +438,29 @@ static vector_status launch_residual_tc(const Dims& dm, const void* K, const voi
     P.n_tiles = (long long)dm.U * P.tpu;
     const int blocks = (int)(P.n_tiles < 148 ? P.n_tiles : 148);
     RopePhases ph = {};
-    if (dm.rope) {
-        rope_phases(dm.theta, 128, &ph);
-        rtc::residual_tc<true><<<blocks, rtc::R_THREADS, rtc::RCfg<true>::SMEM_BYTES, st>>>(
-            (const __nv_bfloat16*)K, (const __nv_bfloat16*)V, mapW, idx, P, ph, eps, fault);
-    } else {
-        rtc::residual_tc<false><<<blocks, rtc::R_THREADS, rtc::RCfg<false>::SMEM_BYTES, st>>>(
-            (const __nv_bfloat16*)K, (const __nv_bfloat16*)V, mapW, idx, P, ph, eps, fault);
-    }
-    VEC_LAUNCH_CHECK();
+    if (dm.rope) rope_phases(dm.theta, 128, &ph);
+    // dependent: blocks may take SMs while the kernel that writes idx drains; the loaders wait for it
+    cudaLaunchAttribute attr;
+    attr.id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr.val.programmaticStreamSerializationAllowed = dependent ? 1 : 0;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(blocks);
+    cfg.blockDim = dim3(rtc::R_THREADS);
+    cfg.dynamicSmemBytes = dm.rope ? rtc::RCfg<true>::SMEM_BYTES : rtc::RCfg<false>::SMEM_BYTES;
+    cfg.stream = st;
+    cfg.attrs = &attr;
+    cfg.numAttrs = 1;
+    const __nv_bfloat16* Kp = (const __nv_bfloat16*)K;
+    const __nv_bfloat16* Vp = (const __nv_bfloat16*)V;
+    if (dm.rope) VEC_CUDA_CHECK(cudaLaunchKernelEx(&cfg, rtc::residual_tc<true>, Kp, Vp, mapW, idx, P, ph, eps, fault));
+    else VEC_CUDA_CHECK(cudaLaunchKernelEx(&cfg, rtc::residual_tc<false>, Kp, Vp, mapW, idx, P, ph, eps, fault));
     return VECTOR_OK;
 }
 
 static vector_status residual_dispatch(const Dims& dm, const void* K, const void* V, const void* W, int64_t N,
-                                       const int32_t* idx, int64_t n_idx, float* eps, cudaStream_t st) {
-    if (dm.dtype == VECTOR_BF16 && dm.d == 128) return launch_residual_tc(dm, K, V, W, N, idx, n_idx, eps, st);
+                                       const int32_t* idx, int64_t n_idx, float* eps, cudaStream_t st,
+                                       bool dependent = false) {
+    if (dm.dtype == VECTOR_BF16 && dm.d == 128) return launch_residual_tc(dm, K, V, W, N, idx, n_idx, eps, st, dependent);
     if (dm.dtype == VECTOR_F32)
         return dm.d == 64 ? launch_residual<float, 64>(dm, K, V, W, N, idx, n_idx, eps, st)
                           : launch_residual<float, 128>(dm, K, V, W, N, idx, n_idx, eps, st);
@@ -458,7 +472,8 @@ static vector_status residual_dispatch(const Dims& dm, const void* K, const void
 // per SM stay resident).
 constexpr int TRUNC_STAGE_MAX = 16384;
 static vector_status launch_truncate(const Dims& dm, const vector_budget* budget, const float* eps, const int32_t* pool,
-                                     uint8_t* tier, int32_t* ret_idx, int32_t* apx_idx, cudaStream_t st) {
+                                     uint8_t* tier, int32_t* ret_idx, int32_t* apx_idx, cudaStream_t st,
+                                     bool dependent = false) {
     const int stage = budget->n_pool <= TRUNC_STAGE_MAX ? 1 : 0;
     const size_t smem = stage ? (size_t)budget->n_pool * sizeof(uint32_t) : 0;
     static PerDeviceOnce once;
@@ -467,9 +482,19 @@ static vector_status launch_truncate(const Dims& dm, const vector_budget* budget
                                                    TRUNC_STAGE_MAX * (int)sizeof(uint32_t));
         if (e != cudaSuccess) { once.undo(); VEC_CUDA_CHECK(e); }
     }
-    truncate_kernel<<<dm.U, SEL_THREADS, smem, st>>>(eps, pool, budget->n_tokens, (int)budget->n_pool, (int)budget->n_apx,
-                                                     tier, ret_idx, apx_idx, stage);
-    VEC_LAUNCH_CHECK();
+    // dependent: may start (and clear the tier map) while the kernel before it in the stream drains
+    cudaLaunchAttribute attr;
+    attr.id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr.val.programmaticStreamSerializationAllowed = dependent ? 1 : 0;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(dm.U);
+    cfg.blockDim = dim3(SEL_THREADS);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cfg.attrs = &attr;
+    cfg.numAttrs = 1;
+    VEC_CUDA_CHECK(cudaLaunchKernelEx(&cfg, truncate_kernel, eps, pool, (int64_t)budget->n_tokens, (int)budget->n_pool,
+                                      (int)budget->n_apx, tier, ret_idx, apx_idx, stage));
     return VECTOR_OK;
 }
 
@@ -533,7 +558,7 @@ extern "C" vector_status vector_route(const vector_shape* shape, const vector_bu
     cudaStream_t st = (cudaStream_t)stream;
     pool_select_kernel<<<dm.U, SEL_THREADS, 0, st>>>(scores, budget->n_tokens, (int)budget->n_pool, pool);
     VEC_LAUNCH_CHECK();
-    rc = residual_dispatch(dm, K, V, W, budget->n_tokens, pool, budget->n_pool, eps, st);
+    rc = residual_dispatch(dm, K, V, W, budget->n_tokens, pool, budget->n_pool, eps, st, true);
     if (rc != VECTOR_OK) return rc;
-    return launch_truncate(dm, budget, eps, pool, tier, ret_idx, apx_idx, st);
+    return launch_truncate(dm, budget, eps, pool, tier, ret_idx, apx_idx, st, true);
 }
