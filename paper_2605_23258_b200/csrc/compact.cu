@@ -1,40 +1,60 @@
 // Compaction into the mixed cache (paper Section 3.2, Step 3): retained tokens
 // keep key and value, approximated tokens keep the key only.  Pure data
-// movement: every thread moves one 16-byte piece of one row.
+// movement: a thread moves one 16-byte piece of each of four rows, the four
+// loads in flight together.
 #include "common.cuh"
 #include "internal.h"
 
 namespace vec {
 
+constexpr int COMPACT_THREADS = 256;
+constexpr int COMPACT_PASSES = 4;
+
 // Logical row r of a unit: [0, n_ret) K -> ret_k ; [n_ret, 2 n_ret) V -> ret_v ;
-// [2 n_ret, 2 n_ret + n_apx) K -> apx_k.   grid-stride over U * rows * pieces.
-__global__ void __launch_bounds__(256)
-compact_kernel(const uint4* __restrict__ K, const uint4* __restrict__ V, int64_t N, int pieces,
+// [2 n_ret, 2 n_ret + n_apx) K -> apx_k.  A row is `pieces` = 2^lp pieces of 16 bytes; a block owns
+// COMPACT_PASSES * (COMPACT_THREADS >> lp) consecutive rows of one unit.  grid: U * chunks blocks.
+__global__ void __launch_bounds__(COMPACT_THREADS)
+compact_kernel(const uint4* __restrict__ K, const uint4* __restrict__ V, int64_t N, int lp,
                const int32_t* __restrict__ ret_idx, const int32_t* __restrict__ apx_idx, int n_ret, int n_apx,
                uint4* __restrict__ ret_k, uint4* __restrict__ ret_v, uint4* __restrict__ apx_k,
                int32_t* __restrict__ ret_pos, int32_t* __restrict__ apx_pos, int64_t cap_ret, int64_t cap_apx,
-               int64_t total) {
-    const int rows = 2 * n_ret + n_apx;
-    for (int64_t t = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; t < total;
-         t += (int64_t)gridDim.x * blockDim.x) {
-        int piece = (int)(t % pieces);
-        int64_t rr = t / pieces;
-        int r = (int)(rr % rows);
-        int64_t u = rr / rows;
+               int chunks) {
+    const int rows = 2 * n_ret + n_apx, pieces = 1 << lp;
+    const int u = blockIdx.x / chunks, chunk = blockIdx.x - u * chunks;
+    const int piece = threadIdx.x & (pieces - 1), rsub = threadIdx.x >> lp, per_pass = COMPACT_THREADS >> lp;
+    const uint4* src[COMPACT_PASSES];
+    uint4* dst[COMPACT_PASSES];
+    int32_t* pos[COMPACT_PASSES];
+    int32_t tok[COMPACT_PASSES];
+#pragma unroll
+    for (int p = 0; p < COMPACT_PASSES; ++p) {
+        const int r = (chunk * COMPACT_PASSES + p) * per_pass + rsub;
+        src[p] = nullptr; dst[p] = nullptr; pos[p] = nullptr; tok[p] = 0;
+        if (r >= rows) continue;
         if (r < n_ret) {
-            int32_t tok = ret_idx[u * n_ret + r];
-            ret_k[(u * cap_ret + r) * pieces + piece] = K[(u * N + tok) * pieces + piece];
-            if (piece == 0) ret_pos[u * cap_ret + r] = tok;
+            tok[p] = ret_idx[(size_t)u * n_ret + r];
+            src[p] = K; dst[p] = ret_k + (((size_t)u * cap_ret + r) << lp) + piece;
+            pos[p] = ret_pos + (size_t)u * cap_ret + r;
         } else if (r < 2 * n_ret) {
-            int q = r - n_ret;
-            int32_t tok = ret_idx[u * n_ret + q];
-            ret_v[(u * cap_ret + q) * pieces + piece] = V[(u * N + tok) * pieces + piece];
+            const int q = r - n_ret;
+            tok[p] = ret_idx[(size_t)u * n_ret + q];
+            src[p] = V; dst[p] = ret_v + (((size_t)u * cap_ret + q) << lp) + piece;
         } else {
-            int q = r - 2 * n_ret;
-            int32_t tok = apx_idx[u * n_apx + q];
-            apx_k[(u * cap_apx + q) * pieces + piece] = K[(u * N + tok) * pieces + piece];
-            if (piece == 0) apx_pos[u * cap_apx + q] = tok;
+            const int q = r - 2 * n_ret;
+            tok[p] = apx_idx[(size_t)u * n_apx + q];
+            src[p] = K; dst[p] = apx_k + (((size_t)u * cap_apx + q) << lp) + piece;
+            pos[p] = apx_pos + (size_t)u * cap_apx + q;
         }
+    }
+    uint4 v[COMPACT_PASSES];
+#pragma unroll
+    for (int p = 0; p < COMPACT_PASSES; ++p)
+        if (src[p]) v[p] = src[p][(((size_t)u * N + tok[p]) << lp) + piece];
+#pragma unroll
+    for (int p = 0; p < COMPACT_PASSES; ++p) {
+        if (!src[p]) continue;
+        *dst[p] = v[p];
+        if (piece == 0 && pos[p]) *pos[p] = tok[p];
     }
 }
 
@@ -57,14 +77,17 @@ extern "C" vector_status vector_compact(const vector_shape* shape, const vector_
     if (budget->n_apx > 0 && (!apx_idx || !cache->apx_k || !cache->apx_pos)) return VECTOR_ERR_NULL;
     const int pieces = dm.d * dm.esize / 16;
     const int64_t rows = 2 * budget->n_ret + budget->n_apx;
-    const int64_t total = (int64_t)dm.U * rows * pieces;
-    if (total == 0) return VECTOR_OK;
-    int64_t blocks = (total + 255) / 256;
-    if (blocks > 148 * 32) blocks = 148 * 32;
-    compact_kernel<<<(unsigned)blocks, 256, 0, (cudaStream_t)stream>>>(
-        (const uint4*)K, (const uint4*)V, budget->n_tokens, pieces, ret_idx, apx_idx, (int)budget->n_ret,
+    if (rows == 0) return VECTOR_OK;
+    int lp = 0;
+    while ((1 << lp) < pieces) ++lp;                  // pieces is 8, 16 or 32 for the supported shapes
+    const int rows_per_block = COMPACT_PASSES * (COMPACT_THREADS >> lp);
+    const int64_t chunks = (rows + rows_per_block - 1) / rows_per_block;
+    const int64_t blocks = (int64_t)dm.U * chunks;
+    if (blocks > 0x7fffffffLL) return VECTOR_ERR_SHAPE;
+    compact_kernel<<<(unsigned)blocks, COMPACT_THREADS, 0, (cudaStream_t)stream>>>(
+        (const uint4*)K, (const uint4*)V, budget->n_tokens, lp, ret_idx, apx_idx, (int)budget->n_ret,
         (int)budget->n_apx, (uint4*)cache->ret_k, (uint4*)cache->ret_v, (uint4*)cache->apx_k, cache->ret_pos,
-        cache->apx_pos, cache->cap_ret, cache->cap_apx, total);
+        cache->apx_pos, cache->cap_ret, cache->cap_apx, (int)chunks);
     VEC_LAUNCH_CHECK();
     return VECTOR_OK;
 }
