@@ -265,8 +265,8 @@ __device__ __forceinline__ float max32(const uint32_t (&v)[32]) {
 // One accumulator tile of pass 1 for this thread's row: 128 columns in four TMEM loads.  The
 // buffer is handed back to the MMA warp as soon as the last load has completed.  The running sum l
 // is kept against a reference m that lags behind the true maximum: the exponentials of a chunk do
-// not wait for the chunk's maximum, and only when a logit exceeds the reference by more than 2^64
-// (always on an item's first chunk, where m = -inf) is the reference moved and the chunk summed again.
+// not wait for the chunk's maximum, and only when their sum exceeds 2^64 (always on an item's first
+// chunk, where m = -inf) is the maximum taken, the reference moved and the chunk summed again.
 template <bool MASKED>
 __device__ __forceinline__ void softmax_tile_pass1(uint32_t taddr, float c, long long key0, long long last_visible,
                                                    float& m, float& l, uint64_t& empty_bar, int lane) {
@@ -285,15 +285,15 @@ __device__ __forceinline__ void softmax_tile_pass1(uint32_t taddr, float c, long
             if (lane == 0) tma::mbar_arrive(&empty_bar);
         }
         if (!MASKED) {
-            const float cm = max32(cur) * c;
-            float s;
-            bool again;
-#pragma unroll 1
-            do {
+            // the sum itself tells whether a logit ran far ahead of the reference: only then is the
+            // chunk's maximum looked for and the chunk summed again against it
+            float s = exp2_sum32(cur, c, -m);
+            if (!(s <= 1.8446744e19f)) {           // above 2^64, infinite (first chunk: m = -inf) or not a number
+                const float cm = max32(cur) * c;
+                l *= ex2(m - cm);
+                m = cm;
                 s = exp2_sum32(cur, c, -m);
-                again = cm > m + 64.f;
-                if (again) { l *= ex2(m - cm); m = cm; }
-            } while (again);
+            }
             l += s;
         } else {
             float v[32];
