@@ -15,8 +15,8 @@ namespace vec {
 template <typename T> struct Piece;
 template <> struct Piece<__nv_bfloat16> {
     static constexpr int EPP = 8;
-    static __device__ __forceinline__ void load(const __nv_bfloat16* p, float (&o)[8]) {
-        const uint4 v = *reinterpret_cast<const uint4*>(p);
+    static __device__ __forceinline__ uint4 load_raw(const __nv_bfloat16* p) { return *reinterpret_cast<const uint4*>(p); }
+    static __device__ __forceinline__ void expand(const uint4 v, float (&o)[8]) {
         o[0] = __uint_as_float(v.x << 16); o[1] = __uint_as_float(v.x & 0xffff0000u);
         o[2] = __uint_as_float(v.y << 16); o[3] = __uint_as_float(v.y & 0xffff0000u);
         o[4] = __uint_as_float(v.z << 16); o[5] = __uint_as_float(v.z & 0xffff0000u);
@@ -25,8 +25,9 @@ template <> struct Piece<__nv_bfloat16> {
 };
 template <> struct Piece<float> {
     static constexpr int EPP = 4;
-    static __device__ __forceinline__ void load(const float* p, float (&o)[4]) {
-        const float4 v = *reinterpret_cast<const float4*>(p);
+    static __device__ __forceinline__ uint4 load_raw(const float* p) { return *reinterpret_cast<const uint4*>(p); }
+    static __device__ __forceinline__ void expand(const uint4 r, float (&o)[4]) {
+        const float4 v = make_float4(__uint_as_float(r.x), __uint_as_float(r.y), __uint_as_float(r.z), __uint_as_float(r.w));
         o[0] = v.x; o[1] = v.y; o[2] = v.z; o[3] = v.w;
     }
 };
@@ -39,7 +40,7 @@ __device__ __forceinline__ float sum8(float v) {        // over the eight lanes 
 
 constexpr int KD_WARPS = 8;
 constexpr int KD_ROWS = 4;        // rows per warp and load
-constexpr int KD_BATCH = 4;       // loads a warp has in flight
+constexpr int KD_BATCH = 8;       // row groups a warp has in flight (kept as raw 16-byte pieces until used)
 
 // grid (chunks, U), 256 threads.  partial[(u * chunks + chunk) * D + c], rinv[u * N + i].
 template <typename T, int D>
@@ -58,31 +59,31 @@ keydiff_anchor_partial(const T* __restrict__ K, int64_t N, int64_t chunk_len, fl
 #pragma unroll
         for (int e = 0; e < EPP; ++e) acc[p][e] = 0.f;
     for (int64_t base = r0 + wid * KD_ROWS * KD_BATCH; base < r1; base += KD_WARPS * KD_ROWS * KD_BATCH) {
-        float x[KD_BATCH][PPL][EPP];
+        uint4 raw[KD_BATCH][PPL];
 #pragma unroll
         for (int b = 0; b < KD_BATCH; ++b) {
             const int64_t row = base + b * KD_ROWS + rsub;
 #pragma unroll
-            for (int p = 0; p < PPL; ++p) {
-#pragma unroll
-                for (int e = 0; e < EPP; ++e) x[b][p][e] = 0.f;
-                if (row < r1) Piece<T>::load(Ku + (size_t)row * D + (p * 8 + seg) * EPP, x[b][p]);
-            }
+            for (int p = 0; p < PPL; ++p)
+                raw[b][p] = row < r1 ? Piece<T>::load_raw(Ku + (size_t)row * D + (p * 8 + seg) * EPP) : make_uint4(0, 0, 0, 0);
         }
 #pragma unroll
         for (int b = 0; b < KD_BATCH; ++b) {
             const int64_t row = base + b * KD_ROWS + rsub;
+            float x[PPL][EPP];
+#pragma unroll
+            for (int p = 0; p < PPL; ++p) Piece<T>::expand(raw[b][p], x[p]);
             float s = 0.f;
 #pragma unroll
             for (int p = 0; p < PPL; ++p)
 #pragma unroll
-                for (int e = 0; e < EPP; ++e) s = fmaf(x[b][p][e], x[b][p][e], s);
+                for (int e = 0; e < EPP; ++e) s = fmaf(x[p][e], x[p][e], s);
             s = sum8(s);
             const float ri = s > 0.f ? 1.0f / sqrtf(s) : 0.f;        // a zero key adds nothing
 #pragma unroll
             for (int p = 0; p < PPL; ++p)
 #pragma unroll
-                for (int e = 0; e < EPP; ++e) acc[p][e] = fmaf(x[b][p][e], ri, acc[p][e]);
+                for (int e = 0; e < EPP; ++e) acc[p][e] = fmaf(x[p][e], ri, acc[p][e]);
             if (seg == 0 && row < r1) rinv[(size_t)u * N + row] = ri;
         }
     }
@@ -132,26 +133,27 @@ keydiff_cosine(const T* __restrict__ K, int64_t N, int64_t chunk_len, const floa
     const T* Ku = K + (size_t)u * N * D;
     const int64_t r0 = (int64_t)chunk * chunk_len, r1 = min(N, r0 + chunk_len);
     for (int64_t base = r0 + wid * KD_ROWS * KD_BATCH; base < r1; base += KD_WARPS * KD_ROWS * KD_BATCH) {
-        float x[KD_BATCH][PPL][EPP], ri[KD_BATCH];
+        uint4 raw[KD_BATCH][PPL];
+        float ri[KD_BATCH];
 #pragma unroll
         for (int b = 0; b < KD_BATCH; ++b) {
             const int64_t row = base + b * KD_ROWS + rsub;
 #pragma unroll
-            for (int p = 0; p < PPL; ++p) {
-#pragma unroll
-                for (int e = 0; e < EPP; ++e) x[b][p][e] = 0.f;
-                if (row < r1) Piece<T>::load(Ku + (size_t)row * D + (p * 8 + seg) * EPP, x[b][p]);
-            }
+            for (int p = 0; p < PPL; ++p)
+                raw[b][p] = row < r1 ? Piece<T>::load_raw(Ku + (size_t)row * D + (p * 8 + seg) * EPP) : make_uint4(0, 0, 0, 0);
             ri[b] = (seg == 0 && row < r1) ? rinv[(size_t)u * N + row] : 0.f;
         }
 #pragma unroll
         for (int b = 0; b < KD_BATCH; ++b) {
             const int64_t row = base + b * KD_ROWS + rsub;
+            float x[PPL][EPP];
+#pragma unroll
+            for (int p = 0; p < PPL; ++p) Piece<T>::expand(raw[b][p], x[p]);
             float s = 0.f;
 #pragma unroll
             for (int p = 0; p < PPL; ++p)
 #pragma unroll
-                for (int e = 0; e < EPP; ++e) s = fmaf(x[b][p][e], a[p][e], s);
+                for (int e = 0; e < EPP; ++e) s = fmaf(x[p][e], a[p][e], s);
             s = sum8(s);
             if (seg == 0 && row < r1) scores[(size_t)u * N + row] = -s * ri[b] * inv_an;
         }
