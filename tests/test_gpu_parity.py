@@ -471,6 +471,31 @@ def test_decode_long_block_ranges(oracle):
             assert np.max(np.abs(out1[u].cpu().double().numpy() - o_tok)) <= 2e-2, (base, u, "per tile")
 
 
+def test_back_to_back_calls_repeat_bitwise(oracle):
+    """The calls of the path are asynchronous and partly overlap (programmatic dependent launches inside
+    route and decode): issued back to back without a host synchronisation, on the same buffers, they
+    must leave bit-identical results every time."""
+    wl = synth.shrink(synth.WORKLOADS[2], n_layers=8)
+    K, V, Q = synth.context(wl, DEV)
+    W = calibrated_maps(wl).to(DEV)
+    sh, b = shape_of(wl), budget_of(wl, 20)
+    comp = Compressor(sh, b, extra_rows=1, keep_eps=True)
+    _, sq, _ = synth.all_head_params(wl, DEV)
+    q = synth.decode_q(wl, 0, DEV, sq)
+    out = torch.empty(wl.units, wl.group, wl.head_dim, dtype=torch.float32, device=DEV)
+    snaps = []
+    for _ in range(4):
+        comp.compress(Q, K, V, W)
+        comp.decode(q, W, out)
+        snaps.append([t.clone() for t in (comp.scores, comp.pool_idx, comp.eps, comp.tier, comp.ret_idx, comp.apx_idx,
+                                          comp.cache.ret_k, comp.cache.ret_v, comp.cache.apx_k, out)])
+    torch.cuda.synchronize()
+    assert vec.vector_device_fault() == 0
+    for later in snaps[1:]:
+        for first, again in zip(snaps[0], later):
+            assert torch.equal(first, again)
+
+
 def _sampled_units_case(oracle, wl, percent, sample, theta=None):
     """Whole workload on the device in the launch shape the benchmark times; the oracle checks the
     sampled units end to end, every unit is checked for the properties that hold at any size.
