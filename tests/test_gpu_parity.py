@@ -471,6 +471,33 @@ def test_decode_long_block_ranges(oracle):
             assert np.max(np.abs(out1[u].cpu().double().numpy() - o_tok)) <= 2e-2, (base, u, "per tile")
 
 
+@pytest.mark.parametrize("base,head_dim,N,Bp,n_a", [(0, 64, 777, 230, 100), (0, 128, 500, 61, 0), (1, 64, 900, 167, 167),
+                                                    (1, 128, 1500, 514, 257)])
+def test_compact_bit_exact(oracle, base, head_dim, N, Bp, n_a):
+    """Compaction alone, every element type and head size (8, 16 and 32 pieces of 16 bytes per row), ragged
+    and empty pools: the gathered rows and positions are copies, so the comparison is exact."""
+    wl = synth.shrink(synth.WORKLOADS[base], N=N, head_dim=head_dim, n_kv_heads=3, n_q_heads=6, window=8)
+    K, V, _ = synth.context(wl, DEV)
+    sh = shape_of(wl)
+    n_ret, n_apx, n_pool = Bp - n_a, 2 * n_a, Bp + n_a          # the planner's identities
+    b = vec.Budget(N, Bp, n_a, n_pool, n_apx, n_ret, N - n_pool)
+    g = torch.Generator().manual_seed(N)
+    ret_idx = torch.stack([torch.randperm(N, generator=g)[:n_ret].sort().values for _ in range(wl.units)]).to(torch.int32)
+    apx_idx = torch.stack([torch.randperm(N, generator=g)[:n_apx].sort().values for _ in range(wl.units)]).to(torch.int32)
+    cache = vec.alloc_cache(sh, b, 2, DEV)
+    vec.vector_compact(sh, b, K, V, ret_idx.to(DEV).reshape(wl.units, -1), apx_idx.to(DEV).reshape(wl.units, -1), cache)
+    torch.cuda.synchronize()
+    for u in range(wl.units):
+        rk, rpos = oracle.gather_rows(K[u].cpu(), ret_idx[u].numpy())
+        rv, _ = oracle.gather_rows(V[u].cpu(), ret_idx[u].numpy())
+        ak, apos = oracle.gather_rows(K[u].cpu(), apx_idx[u].numpy())
+        assert np.array_equal(cache.ret_k[u, :n_ret].cpu().double().numpy(), rk)
+        assert np.array_equal(cache.ret_v[u, :n_ret].cpu().double().numpy(), rv)
+        assert np.array_equal(cache.apx_k[u, :n_apx].cpu().double().numpy(), ak)
+        assert np.array_equal(cache.ret_pos[u, :n_ret].cpu().numpy(), rpos)
+        assert np.array_equal(cache.apx_pos[u, :n_apx].cpu().numpy(), apos)
+
+
 def test_back_to_back_calls_repeat_bitwise(oracle):
     """The calls of the path are asynchronous and partly overlap (programmatic dependent launches inside
     route and decode): issued back to back without a host synchronisation, on the same buffers, they
