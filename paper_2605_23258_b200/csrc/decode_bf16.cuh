@@ -646,6 +646,16 @@ decode_merge_bf16_d128(const float* __restrict__ partial, const __nv_bfloat16* _
     const int first = block_of_tile((long long)u * pl.n_tiles, pl);
     const int n_rec = (block_of_tile((long long)(u + 1) * pl.n_tiles - 1, pl) - first + 1) * CONSUMER_WARPS;   // <= 36
     const float* base = partial + (size_t)u * pl.s_max * CONSUMER_WARPS * g * REC;
+    // The first twelve records' sums are requested before the headers are looked at, so that the
+    // two loads share one memory latency (a unit has at most a dozen records unless it is very long).
+    float rv[12], rk[12];
+#pragma unroll
+    for (int k = 0; k < 12; ++k) {
+        const int j = min(k, n_rec - 1);
+        const float* r = base + ((size_t)j * g + a) * REC + 4;
+        rv[k] = r[c];
+        rk[k] = r[128 + c];
+    }
     if (c < 32) {
         // first warp of head a: headers of records lane and lane + 32
         float mj[2], lj[2], sj[2];
@@ -672,17 +682,18 @@ decode_merge_bf16_d128(const float* __restrict__ partial, const __nv_bfloat16* _
     }
     __syncthreads();
     float av = 0.f, ak = 0.f;
-    for (int j0 = 0; j0 < n_rec; j0 += 6) {
-        float rv[6], rk[6];
+    for (int j0 = 0; j0 < n_rec; j0 += 12) {
+        if (j0 > 0) {
 #pragma unroll
-        for (int k = 0; k < 6; ++k) {
-            const int j = min(j0 + k, n_rec - 1);
-            const float* r = base + ((size_t)j * g + a) * REC + 4;
-            rv[k] = r[c];
-            rk[k] = r[128 + c];
+            for (int k = 0; k < 12; ++k) {
+                const int j = min(j0 + k, n_rec - 1);
+                const float* r = base + ((size_t)j * g + a) * REC + 4;
+                rv[k] = r[c];
+                rk[k] = r[128 + c];
+            }
         }
 #pragma unroll
-        for (int k = 0; k < 6; ++k) {
+        for (int k = 0; k < 12; ++k) {
             if (j0 + k < n_rec) {
                 av = fmaf(fv[a][j0 + k], rv[k], av);
                 ak = fmaf(fk[a][j0 + k], rk[k], ak);
