@@ -7,7 +7,7 @@
 
 namespace vec {
 
-constexpr int COMPACT_THREADS = 256;
+constexpr int COMPACT_THREADS = 64;      // small blocks: many independent gathers in flight per SM, even tail
 constexpr int COMPACT_PASSES = 4;
 
 // Logical row r of a unit: [0, n_ret) K -> ret_k ; [n_ret, 2 n_ret) V -> ret_v ;
