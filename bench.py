@@ -325,7 +325,7 @@ def main():
     # workloads and for kernels changed since the capture.
     ncu_traffic_per_unit = {"vector_score (logit passes)": (541.3e6 + 5.6e6 + 541.4e6 + 17.3e6 + 16.8e6) / 64,
                             "vector_route (select + residual + truncate)": (8.4e6 + 328.4e6 + 5.5e6 + 5.1e6) / 64,
-                            "vector_compact": (217.3e6 + 171.1e6) / 64,
+                            "vector_compact": (217.3e6 + 169.8e6) / 64,
                             "vector_decode_attn (split + merge)": (215.0e6 + 4.3e6 + 4.7e6) / 64}
     exps = 2.0 * g * w * N * U                                  # one exp2 per logit and pass
     xu_peak = 16.0 * 148 * (clocks_hint_mhz * 1e6)              # MUFU results per second at the sampled SM clock
