@@ -65,5 +65,25 @@ __device__ __forceinline__ void rope_fill_inv_freq(double* inv_freq, int d, floa
     for (int c = threadIdx.x; c < d / 2; c += blockDim.x) inv_freq[c] = pow((double)theta, -2.0 * (double)c / (double)d);
 }
 
+// Kernel launch that may carry the programmatic-dependent attribute: with `dependent` the kernel may
+// be scheduled while the kernel before it in the stream drains (once every block of that one has
+// executed griddepcontrol.launch_dependents, or exited); it must execute griddepcontrol.wait before
+// it touches that kernel's output.
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_maybe_dependent(bool dependent, void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem,
+                                          cudaStream_t st, Args... args) {
+    cudaLaunchAttribute attr;
+    attr.id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr.val.programmaticStreamSerializationAllowed = dependent ? 1 : 0;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cfg.attrs = &attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+
 }  // namespace vec
 #endif

@@ -267,23 +267,15 @@ static vector_status launch_decode_bf16_d128(const Dims& dm, const void* q, cons
             (const T*)q, maps, pl, (int)ch->n_ret, (int)ch->n_apx, dm.g, dm.LH, c2, partial, fault, nullptr, 0, ph);
     VEC_LAUNCH_CHECK();
     // programmatic dependent launch: the merge blocks start while the streaming kernel drains
-    cudaLaunchAttribute attr;
-    attr.id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    attr.val.programmaticStreamSerializationAllowed = 1;
-    cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3(dm.U);
-    cfg.blockDim = dim3(128 * dm.g);
-    cfg.dynamicSmemBytes = 0;
-    cfg.stream = st;
-    cfg.attrs = &attr;
-    cfg.numAttrs = 1;
     const float* rec = partial;
     const int apply_w = mode == 1 ? 0 : 1;
     const T* Wp = (const T*)W;
     if (out_dtype == VECTOR_F32)
-        VEC_CUDA_CHECK(cudaLaunchKernelEx(&cfg, dbf::decode_merge_bf16_d128<float>, rec, Wp, dm.LH, dm.g, pl, apply_w, (float*)out));
+        VEC_CUDA_CHECK(launch_maybe_dependent(true, dbf::decode_merge_bf16_d128<float>, dim3(dm.U), dim3(128 * dm.g), 0, st, rec,
+                                              Wp, dm.LH, dm.g, pl, apply_w, (float*)out));
     else
-        VEC_CUDA_CHECK(cudaLaunchKernelEx(&cfg, dbf::decode_merge_bf16_d128<T>, rec, Wp, dm.LH, dm.g, pl, apply_w, (T*)out));
+        VEC_CUDA_CHECK(launch_maybe_dependent(true, dbf::decode_merge_bf16_d128<T>, dim3(dm.U), dim3(128 * dm.g), 0, st, rec, Wp,
+                                              dm.LH, dm.g, pl, apply_w, (T*)out));
     return VECTOR_OK;
 }
 

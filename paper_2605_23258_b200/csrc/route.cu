@@ -440,20 +440,14 @@ static vector_status launch_residual_tc(const Dims& dm, const void* K, const voi
     RopePhases ph = {};
     if (dm.rope) rope_phases(dm.theta, 128, &ph);
     // dependent: blocks may take SMs while the kernel that writes idx drains; the loaders wait for it
-    cudaLaunchAttribute attr;
-    attr.id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    attr.val.programmaticStreamSerializationAllowed = dependent ? 1 : 0;
-    cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3(blocks);
-    cfg.blockDim = dim3(rtc::R_THREADS);
-    cfg.dynamicSmemBytes = dm.rope ? rtc::RCfg<true>::SMEM_BYTES : rtc::RCfg<false>::SMEM_BYTES;
-    cfg.stream = st;
-    cfg.attrs = &attr;
-    cfg.numAttrs = 1;
     const __nv_bfloat16* Kp = (const __nv_bfloat16*)K;
     const __nv_bfloat16* Vp = (const __nv_bfloat16*)V;
-    if (dm.rope) VEC_CUDA_CHECK(cudaLaunchKernelEx(&cfg, rtc::residual_tc<true>, Kp, Vp, mapW, idx, P, ph, eps, fault));
-    else VEC_CUDA_CHECK(cudaLaunchKernelEx(&cfg, rtc::residual_tc<false>, Kp, Vp, mapW, idx, P, ph, eps, fault));
+    if (dm.rope)
+        VEC_CUDA_CHECK(launch_maybe_dependent(dependent, rtc::residual_tc<true>, dim3(blocks), dim3(rtc::R_THREADS),
+                                              rtc::RCfg<true>::SMEM_BYTES, st, Kp, Vp, mapW, idx, P, ph, eps, fault));
+    else
+        VEC_CUDA_CHECK(launch_maybe_dependent(dependent, rtc::residual_tc<false>, dim3(blocks), dim3(rtc::R_THREADS),
+                                              rtc::RCfg<false>::SMEM_BYTES, st, Kp, Vp, mapW, idx, P, ph, eps, fault));
     return VECTOR_OK;
 }
 
@@ -483,18 +477,9 @@ static vector_status launch_truncate(const Dims& dm, const vector_budget* budget
         if (e != cudaSuccess) { once.undo(); VEC_CUDA_CHECK(e); }
     }
     // dependent: may start (and clear the tier map) while the kernel before it in the stream drains
-    cudaLaunchAttribute attr;
-    attr.id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    attr.val.programmaticStreamSerializationAllowed = dependent ? 1 : 0;
-    cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3(dm.U);
-    cfg.blockDim = dim3(SEL_THREADS);
-    cfg.dynamicSmemBytes = smem;
-    cfg.stream = st;
-    cfg.attrs = &attr;
-    cfg.numAttrs = 1;
-    VEC_CUDA_CHECK(cudaLaunchKernelEx(&cfg, truncate_kernel, eps, pool, (int64_t)budget->n_tokens, (int)budget->n_pool,
-                                      (int)budget->n_apx, tier, ret_idx, apx_idx, stage));
+    VEC_CUDA_CHECK(launch_maybe_dependent(dependent, truncate_kernel, dim3(dm.U), dim3(SEL_THREADS), smem, st, eps, pool,
+                                          (int64_t)budget->n_tokens, (int)budget->n_pool, (int)budget->n_apx, tier, ret_idx,
+                                          apx_idx, stage));
     return VECTOR_OK;
 }
 
