@@ -12,6 +12,11 @@ the timed region; `e2e` repeats the measurement through host buffers.
 
   python bench.py [--gpus N] [--steps K] [--warmup W] [--config C] [--impl reference]
 
+Without --config the headline is the largest workload that fits one GPU (the 80-layer,
+131072-token long-context case), and the 32-layer and the batched-serving workloads are
+measured after it in the same process and reported under "configs".  --config C runs one
+workload only.
+
 With --gpus N > 1 (under torchrun) every rank runs an independent replica of the
 workload on its own GPU: the path has no exchange step, so there is no collective
 on the data path and the aggregate is the sum over replicas (weak scaling).
@@ -19,6 +24,9 @@ on the data path and the aggregate is the sum over replicas (weak scaling).
 from __future__ import annotations
 
 import argparse
+import dataclasses
+import gc
+import hashlib
 import json
 import os
 import statistics
@@ -33,6 +41,9 @@ sys.path.insert(0, ROOT)
 METRIC = "compressed tokens/s (score+route+compact); decode-attn HBM GB/s vs peak"
 UNIT = "tokens/s"
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+HEADLINE_CONFIG = 4
+SIDE_CONFIGS = (2, 3)
+XU_PER_CLK_PER_SM = 16.0            # exp2 results of the special-function unit per clock and multiprocessor
 
 
 def load_peaks():
@@ -45,6 +56,36 @@ def load_peaks():
     d = dict(FALLBACK_PEAKS)
     d["source"] = "fallback"
     return d
+
+
+def _sources_digest(files):
+    h = hashlib.sha1()
+    for f in sorted(files):
+        with open(os.path.join(ROOT, "paper_2605_23258_b200", "csrc", f), "rb") as fh:
+            h.update(fh.read())
+    return h.hexdigest()[:16]
+
+
+def load_ncu_traffic():
+    """DRAM bytes per launch from the ncu capture summarised under profiles/ (a small workload of
+    `units` units; these kernels' traffic grows in proportion to the unit count).  An entry is used
+    only while the source files it names still hash to the digest recorded with the capture."""
+    p = os.path.join(ROOT, "profiles", "ncu_dram_bytes.json")
+    if not os.path.exists(p):
+        return {}
+    with open(p) as f:
+        d = json.load(f)
+    out = {}
+    for wl_name, entry in d.get("workloads", {}).items():
+        calls = {}
+        for call, rec in entry["calls"].items():
+            try:
+                if _sources_digest(rec["sources"]) == rec["digest"]:
+                    calls[call] = rec["dram_bytes"]
+            except OSError:
+                pass
+        out[wl_name] = {"units": entry["units"], "calls": calls}
+    return out
 
 
 # --------------------------------------------------------------------------- clocks
@@ -102,11 +143,16 @@ class ClockSampler:
         return out
 
 
+def default_percent(cfg, wl):
+    return 20 if cfg == 1 else wl.budget_percents[0]
+
+
 # ------------------------------------------------------------------- oracle (CPU) arm
 def oracle_sample(wl, percent, n_units=1, decode_steps=2, device="cpu"):
     """Times the oracle, as it stands, single-threaded, on `n_units` units of the workload.
     Returns seconds per unit for compression and per decode step, and what the sample was."""
     import numpy as np
+    import torch
     import oracle
     from paper_2605_23258_b200 import synth
     oracle.build()
@@ -123,7 +169,7 @@ def oracle_sample(wl, percent, n_units=1, decode_steps=2, device="cpu"):
         Q = synth.unit_qobs(wl, bb, l, h, device, params)
         kc, vc = synth.calib_kv(wl, l, h, device, params)
         W = oracle.calibrate(kc.cpu(), vc.cpu(), wl.lam)             # offline, not timed
-        W = np.asarray(__import__("torch").from_numpy(W).to(wl.torch_dtype).double().numpy())
+        W = np.asarray(torch.from_numpy(W).to(wl.torch_dtype).double().numpy())
         Kc, Vc, Qc = K.cpu(), V.cpu(), Q.cpu()
         t0 = time.perf_counter()
         _, sc = oracle.score(Qc, Kc, scale, wl.pool_kernel)
@@ -133,9 +179,9 @@ def oracle_sample(wl, percent, n_units=1, decode_steps=2, device="cpu"):
         ak, _ = oracle.gather_rows(Kc, r["apx_idx"])
         t_comp.append(time.perf_counter() - t0)
         _, sq, _ = params
-        g = __import__("torch").Generator().manual_seed(u)
+        g = torch.Generator().manual_seed(u)
         for _ in range(decode_steps):
-            q = (__import__("torch").randn(wl.group, d, generator=g) * sq.cpu()).to(wl.torch_dtype)
+            q = (torch.randn(wl.group, d, generator=g) * sq.cpu()).to(wl.torch_dtype)
             t0 = time.perf_counter()
             oracle.attend(q, rk, rv, ak, W, scale)
             t_dec.append(time.perf_counter() - t0)
@@ -143,16 +189,25 @@ def oracle_sample(wl, percent, n_units=1, decode_steps=2, device="cpu"):
             "units": units, "budget": b}
 
 
-def run_reference(args, wl, percent):
+def oracle_units_per_sample(wl):
+    """How many units one oracle sample covers: the score of one unit costs 2 g w N d multiply-adds in
+    plain fp64 loops (about a second per 10^9), so long contexts get one unit, short ones a few."""
+    macs = 2.0 * wl.group * wl.window * wl.N * wl.head_dim
+    return max(1, min(wl.units, 4, int(12e9 // macs)))
+
+
+def run_reference(args, cfg, wl, percent):
     """--impl reference: the CPU oracle, timed on the host cores, same metric and config."""
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return 0
-    steps = max(args.steps, 1)
-    for _ in range(min(args.warmup, 1)):
+    n_u = oracle_units_per_sample(wl)
+    steps = max(1, min(args.steps, 3 if n_u > 1 else 2))
+    warm = min(args.warmup, 1)
+    for _ in range(warm):
         oracle_sample(wl, percent, 1, 1)
     t0 = time.perf_counter()
-    res = [oracle_sample(wl, percent, min(wl.units, 4), 2) for _ in range(min(steps, 3))]
+    res = [oracle_sample(wl, percent, n_u, 2) for _ in range(steps)]
     wall = time.perf_counter() - t0
     per_unit = statistics.mean(r["compress_s_per_unit"] for r in res)
     dec_unit = statistics.mean(r["decode_s_per_unit_step"] for r in res)
@@ -160,14 +215,15 @@ def run_reference(args, wl, percent):
     value = wl.batch * wl.N / t_compress_all
     b = res[0]["budget"]
     dec_bytes = wl.units * (2 * b.n_ret + b.n_apx) * wl.head_dim * (2 if wl.dtype == "bf16" else 4)
-    sample = (f"units {res[0]['units']} of {wl.units} per step ({min(steps, 3)} timed samples): "
-              f"score+route+compact and 2 decode steps, single thread; whole-workload time = per-unit time x {wl.units}")
+    sample = (f"units {res[0]['units']} of {wl.units} per step ({steps} timed samples): "
+              f"score+route+compact ({per_unit:.1f} s per unit) and 2 decode steps, single thread; "
+              f"whole-workload time = per-unit time x {wl.units}")
     line = {
-        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": 0, "steps": min(steps, 3),
-        "warmup": min(args.warmup, 1), "ms_per_step": 1e3 * (t_compress_all + dec_unit * wl.units * wl.decode_steps),
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": 0, "steps": steps,
+        "warmup": warm, "ms_per_step": 1e3 * (t_compress_all + dec_unit * wl.units * wl.decode_steps),
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
         "config": {"workload": wl.name, "budget_percent": percent, "batch": wl.batch, "N": wl.N,
-                   "units": wl.units, "extrapolated_from_units": min(wl.units, 4)},
+                   "units": wl.units, "extrapolated_from_units": n_u},
         "cpu_baseline": {"value": value, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": sample},
         "decode": {"gbs": dec_bytes / (dec_unit * wl.units) / 1e9, "s_per_step": dec_unit * wl.units},
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
@@ -178,44 +234,45 @@ def run_reference(args, wl, percent):
 
 
 # ----------------------------------------------------------------------------- GPU arm
-def main():
-    ap = argparse.ArgumentParser()
-    ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=5)
-    ap.add_argument("--warmup", type=int, default=3)
-    ap.add_argument("--config", type=int, default=2, help="workload 1..4 (default 2: 32-layer Llama-3-8B shape)")
-    ap.add_argument("--budget", type=int, default=None, help="budget percent (default: the workload's)")
-    ap.add_argument("--decode-steps", type=int, default=None)
-    ap.add_argument("--layers", type=int, default=None, help="shrink the workload to this many layers (profiling)")
-    ap.add_argument("--impl", default="vector", choices=["vector", "reference"])
-    ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--no-e2e", action="store_true")
-    args = ap.parse_args()
+class Env:
+    """Process-wide state of the GPU arm: device, ranks, peaks."""
 
-    from paper_2605_23258_b200 import synth
-    wl = synth.WORKLOADS[args.config]
-    if args.layers is not None:
-        wl = synth.shrink(wl, n_layers=args.layers, name=f"{wl.name}_first{args.layers}layers")
-    percent = args.budget if args.budget is not None else (20 if args.config == 1 else wl.budget_percents[0])
-    if args.impl == "reference":
-        return run_reference(args, wl, percent)
+    def __init__(self):
+        import torch
+        self.rank = int(os.environ.get("RANK", "0"))
+        self.world = int(os.environ.get("WORLD_SIZE", "1"))
+        self.local = int(os.environ.get("LOCAL_RANK", "0"))
+        torch.cuda.set_device(self.local)
+        self.dev = f"cuda:{self.local}"
+        if self.world > 1:
+            import torch.distributed as dist
+            dist.init_process_group("nccl", device_id=torch.device(self.dev))
+        self.peaks = load_peaks()
+        self.traffic = load_ncu_traffic()
+        self.sm_count = torch.cuda.get_device_properties(self.local).multi_processor_count
 
+    def barrier(self):
+        import torch
+        if self.world > 1:
+            import torch.distributed as dist
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    def close(self):
+        if self.world > 1:
+            import torch.distributed as dist
+            dist.destroy_process_group()
+
+
+def run_workload(env, cfg, wl, percent, steps, warmup, D, extras=True, want_e2e=True, want_cpu=True):
+    """One workload on this rank's GPU: W warm-up steps, K timed steps, the side measurements, and
+    (rank 0, one GPU) the oracle's sample.  Returns the fields of the JSON line."""
     import torch
     import paper_2605_23258_b200 as vec
+    from paper_2605_23258_b200 import replicas, synth
     from paper_2605_23258_b200.pipeline import Compressor, calibrate_maps
 
-    rank = int(os.environ.get("RANK", "0"))
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    local = int(os.environ.get("LOCAL_RANK", "0"))
-    torch.cuda.set_device(local)
-    dev = f"cuda:{local}"
-    if world > 1:
-        import torch.distributed as dist
-        dist.init_process_group("nccl", device_id=torch.device(dev))
-    vec.load_library()
-    W_warm = max(args.warmup, 3)
-    K_steps = max(args.steps, 1)
-    D = args.decode_steps if args.decode_steps is not None else wl.decode_steps
+    dev, world = env.dev, env.world
     es = 2 if wl.dtype == "bf16" else 4
     U, N, d, g, w = wl.units, wl.N, wl.head_dim, wl.group, wl.window
 
@@ -266,28 +323,25 @@ def main():
         if marks is not None:
             marks.append(ev()); marks[-1].record()
 
-    def barrier():
-        if world > 1:
-            import torch.distributed as dist
-            dist.barrier()
-        torch.cuda.synchronize()
-
-    for _ in range(W_warm):
+    for _ in range(warmup):
         one_step()
-    barrier()
-    sampler = ClockSampler(local)
+    env.barrier()
+    sampler = ClockSampler(env.local)
     sampler.start()
     all_marks = []
     t_begin, t_end = ev(), ev()
-    barrier()
+    env.barrier()
+    launches0 = vec.vector_kernel_launches()
     t_begin.record()
-    for _ in range(K_steps):
+    for _ in range(steps):
         m = []
         one_step(m)
         all_marks.append(m)
     t_end.record()
-    barrier()
+    launches = vec.vector_kernel_launches() - launches0
+    env.barrier()
     clocks = sampler.stop()
+    fault = vec.vector_device_fault()
     clocks_hint_mhz = clocks["sm_mhz"] or 1965.0
     total_ms = t_begin.elapsed_time(t_end)
     phase = {"score": [], "route": [], "compact": [], "decode": []}
@@ -297,7 +351,6 @@ def main():
     ms = {k: statistics.mean(v) for k, v in phase.items()}
     compress_ms = ms["score"] + ms["route"] + ms["compact"]
     # every rank is an independent replica: the job's time is the slowest replica's
-    from paper_2605_23258_b200 import replicas
     total_ms, compress_ms, dec_ms_max = replicas.slowest([total_ms, compress_ms, ms["decode"]], dev)
 
     # ---- algorithmic work (per step, one replica)
@@ -305,160 +358,170 @@ def main():
     score_flops = 4.0 * g * w * N * d * U
     score_bytes = U * (N * d * es + N * 4)
     resid_bytes = U * (2 * n_pool * d * es) + U * d * d * es
+    route_bytes = resid_bytes + U * N * 4 * 2
     compact_bytes = 2 * U * (2 * n_ret + n_apx) * d * es
     dec_rows = sum(2 * (n_ret + t) + n_apx for t in range(D))
     decode_bytes = U * dec_rows * d * es + D * (Wm.numel() * es + 2 * U * g * d * es)
-    peaks = load_peaks()
-    hbm, tf = peaks["hbm_gbs"], peaks["bf16_tflops_sustained"]
+    hbm, tf = env.peaks["hbm_gbs"], env.peaks["bf16_tflops_sustained"]
     kernels = [
-        {"kernel": "vector_score (logit passes)", "bound": "tensor", "achieved": score_flops / (ms["score"] * 1e-3) / 1e12,
-         "peak": tf, "unit": "TFLOP/s", "ms": ms["score"], "hbm_gbs": score_bytes / (ms["score"] * 1e-3) / 1e9},
-        {"kernel": "vector_route (select + residual + truncate)", "bound": "hbm",
-         "achieved": (resid_bytes + U * N * 4 * 2) / (ms["route"] * 1e-3) / 1e9, "peak": hbm, "unit": "GB/s", "ms": ms["route"]},
-        {"kernel": "vector_compact", "bound": "hbm", "achieved": compact_bytes / (ms["compact"] * 1e-3) / 1e9,
-         "peak": hbm, "unit": "GB/s", "ms": ms["compact"]},
-        {"kernel": "vector_decode_attn (split + merge)", "bound": "hbm",
+        {"kernel": "vector_score (logit passes)", "call": "score", "bound": "tensor",
+         "achieved": score_flops / (ms["score"] * 1e-3) / 1e12, "peak": tf, "unit": "TFLOP/s", "ms": ms["score"],
+         "hbm_gbs": score_bytes / (ms["score"] * 1e-3) / 1e9},
+        {"kernel": "vector_route (select + residual + truncate)", "call": "route", "bound": "hbm",
+         "achieved": route_bytes / (ms["route"] * 1e-3) / 1e9, "peak": hbm, "unit": "GB/s", "ms": ms["route"]},
+        {"kernel": "vector_compact", "call": "compact", "bound": "hbm",
+         "achieved": compact_bytes / (ms["compact"] * 1e-3) / 1e9, "peak": hbm, "unit": "GB/s", "ms": ms["compact"]},
+        {"kernel": "vector_decode_attn", "call": "decode", "bound": "hbm",
          "achieved": decode_bytes / (ms["decode"] * 1e-3) / 1e9, "peak": hbm, "unit": "GB/s", "ms": ms["decode"]},
     ]
-    # DRAM bytes per call from the ncu capture summarised under profiles/ (64 units of this workload,
-    # scaled by the unit count: traffic of these kernels grows in proportion to it); None for other
-    # workloads and for kernels changed since the capture.
-    ncu_traffic_per_unit = {"vector_score (logit passes)": (541.3e6 + 5.6e6 + 541.4e6 + 17.3e6 + 16.8e6) / 64,
-                            "vector_route (select + residual + truncate)": (8.4e6 + 328.4e6 + 5.5e6 + 5.1e6) / 64,
-                            "vector_compact": (217.3e6 + 169.8e6) / 64,
-                            "vector_decode_attn (split + merge)": (215.0e6 + 4.3e6 + 4.7e6) / 64}
+    captured = env.traffic.get(wl.name.split("_first")[0], None)
     exps = 2.0 * g * w * N * U                                  # one exp2 per logit and pass
-    xu_peak = 16.0 * 148 * (clocks_hint_mhz * 1e6)              # MUFU results per second at the sampled SM clock
+    xu_peak = XU_PER_CLK_PER_SM * env.sm_count * (clocks_hint_mhz * 1e6)
     for k in kernels:
         k["frac"] = k["achieved"] / k["peak"]
         k["traffic"] = None
-        if args.config == 2 and args.budget is None and k["kernel"] in ncu_traffic_per_unit:
-            per_call = ncu_traffic_per_unit[k["kernel"]] * U
-            k["traffic"] = per_call * (D if k["kernel"].startswith("vector_decode") else 1)
-    kernels[0]["xu_exp_per_s"] = exps / (ms["score"] * 1e-3)
-    kernels[0]["xu_frac_of_16_per_clk_per_sm"] = kernels[0]["xu_exp_per_s"] / xu_peak
+        if captured and k["call"] in captured["calls"]:
+            per_call = captured["calls"][k["call"]] * U / captured["units"]
+            k["traffic"] = per_call * (D if k["call"] == "decode" else 1)
+    from paper_2605_23258_b200.binding import score_poly_share
+    poly = score_poly_share()
+    kernels[0]["exp2_per_s"] = exps / (ms["score"] * 1e-3)
+    kernels[0]["exp2_share_on_fma_pipe"] = poly
+    kernels[0]["xu_frac_of_16_per_clk_per_sm"] = (1.0 - poly) * kernels[0]["exp2_per_s"] / xu_peak
     dominant = max(kernels, key=lambda k: k["ms"])
     roofline = {k: dominant[k] for k in ("bound", "achieved", "peak", "unit", "frac", "traffic")}
     roofline["kernel"] = dominant["kernel"]
-    roofline["peak_source"] = f"{peaks['source']} ({'copy GB/s' if dominant['bound'] == 'hbm' else 'sustained bf16 TFLOP/s'})"
+    roofline["peak_source"] = (f"{env.peaks['source']} "
+                               f"({'copy GB/s' if dominant['bound'] == 'hbm' else 'sustained bf16 TFLOP/s'})")
 
-    # ---- the alternative form of the reconstruction (mode 1: W k formed per tile), outside the timed step
-    per_tile = None
-    if wl.dtype == "bf16" and d == 128:
-        comp.cache.n_ret = budget.n_ret
-        for _ in range(3):
-            comp.decode(qs[0], Wm, out, mode=1)
-        a, b_ = ev(), ev()
-        torch.cuda.synchronize(); a.record()
-        for i in range(10):
-            comp.decode(qs[i % n_q], Wm, out, mode=1)
-        b_.record(); torch.cuda.synchronize()
-        us = a.elapsed_time(b_) * 1e3 / 10
-        step_bytes = U * (2 * n_ret + n_apx) * d * es
-        per_tile = {"us_per_step": us, "gbs": step_bytes / us / 1e3,
-                    "extra_flop_per_step": 2.0 * U * n_apx * d * d}
+    per_tile = keydiff = rope = None
+    if extras:
+        # ---- the alternative form of the reconstruction (mode 1: W k formed per tile), outside the timed step
+        if wl.dtype == "bf16" and d == 128:
+            comp.cache.n_ret = budget.n_ret
+            for _ in range(3):
+                comp.decode(qs[0], Wm, out, mode=1)
+            a, b_ = ev(), ev()
+            torch.cuda.synchronize(); a.record()
+            for i in range(10):
+                comp.decode(qs[i % n_q], Wm, out, mode=1)
+            b_.record(); torch.cuda.synchronize()
+            us = a.elapsed_time(b_) * 1e3 / 10
+            step_bytes = U * (2 * n_ret + n_apx) * d * es
+            extra_flop = 2.0 * U * n_apx * d * d
+            per_tile = {"us_per_step": us, "gbs": step_bytes / us / 1e3, "extra_flop_per_step": extra_flop,
+                        "extra_tflops": extra_flop / (us * 1e-6) / 1e12}
 
-    # ---- the query-agnostic base scorer (key geometry), outside the timed step: two HBM passes over K
-    kd_scores = torch.empty(U, N, dtype=torch.float32, device=dev)
-    for _ in range(2):
-        vec.vector_score_keydiff(shape, Kt, N, kd_scores, comp.ws)
-    a, b_ = ev(), ev()
-    torch.cuda.synchronize(); a.record()
-    for _ in range(5):
-        vec.vector_score_keydiff(shape, Kt, N, kd_scores, comp.ws)
-    b_.record(); torch.cuda.synchronize()
-    kd_ms = a.elapsed_time(b_) / 5
-    kd_bytes = U * (2 * N * d * es + 3 * N * 4)
-    keydiff = {"ms": kd_ms, "gbs": kd_bytes / (kd_ms * 1e-3) / 1e9, "frac_of_measured_copy": kd_bytes / (kd_ms * 1e-3) / 1e9 / hbm,
-               "tokens_per_s": wl.batch * N / (kd_ms * 1e-3)}
-    del kd_scores
-
-    # ---- RoPE decoupling (the stored keys taken as post-RoPE: the residual and the reconstruction
-    #      turn them back by position), outside the timed step; same shapes, same budget
-    rope = None
-    if wl.dtype == "bf16" and d == 128:
-        import dataclasses
-        shape_r = dataclasses.replace(shape, rope_enabled=1, rope_theta=500000.0)
-        comp_r = Compressor(shape_r, budget)
-        comp_r.compress(Qt, Kt, Vt, Wm)
+        # ---- the query-agnostic base scorer (key geometry), outside the timed step: two HBM passes over K
+        kd_scores = torch.empty(U, N, dtype=torch.float32, device=dev)
         for _ in range(2):
-            comp_r.route(Kt, Vt, Wm)
+            vec.vector_score_keydiff(shape, Kt, N, kd_scores, comp.ws)
         a, b_ = ev(), ev()
         torch.cuda.synchronize(); a.record()
         for _ in range(5):
-            comp_r.route(Kt, Vt, Wm)
+            vec.vector_score_keydiff(shape, Kt, N, kd_scores, comp.ws)
         b_.record(); torch.cuda.synchronize()
-        r_ms = a.elapsed_time(b_) / 5
-        for _ in range(3):
-            comp_r.decode(qs[0], Wm, out)
-        a, b_ = ev(), ev()
-        torch.cuda.synchronize(); a.record()
-        for i in range(10):
-            comp_r.decode(qs[i % n_q], Wm, out)
-        b_.record(); torch.cuda.synchronize()
-        us = a.elapsed_time(b_) * 1e3 / 10
-        step_bytes = U * (2 * n_ret + n_apx) * d * es
-        rope = {"theta": 500000.0, "route_ms": r_ms, "route_gbs": (resid_bytes + U * N * 4 * 2) / (r_ms * 1e-3) / 1e9,
-                "decode_us_per_step": us, "decode_gbs": step_bytes / us / 1e3,
-                "sincos_per_decode_step": 2.0 * U * n_apx * (d // 2), "sincos_per_route": 2.0 * U * n_pool * (d // 2)}
-        del comp_r
+        kd_ms = a.elapsed_time(b_) / 5
+        kd_bytes = U * (2 * N * d * es + 3 * N * 4)
+        keydiff = {"ms": kd_ms, "gbs": kd_bytes / (kd_ms * 1e-3) / 1e9,
+                   "frac_of_measured_copy": kd_bytes / (kd_ms * 1e-3) / 1e9 / hbm,
+                   "tokens_per_s": wl.batch * N / (kd_ms * 1e-3)}
+        del kd_scores
 
-    # ---- end to end through host buffers (rank 0 semantics on every rank; reported from rank 0)
+        # ---- RoPE decoupling (the stored keys taken as post-RoPE: the residual and the reconstruction
+        #      turn them back by position), outside the timed step; same shapes, same budget
+        if wl.dtype == "bf16" and d == 128:
+            shape_r = dataclasses.replace(shape, rope_enabled=1, rope_theta=500000.0)
+            comp_r = Compressor(shape_r, budget)
+            comp_r.compress(Qt, Kt, Vt, Wm)
+            for _ in range(2):
+                comp_r.route(Kt, Vt, Wm)
+            a, b_ = ev(), ev()
+            torch.cuda.synchronize(); a.record()
+            for _ in range(5):
+                comp_r.route(Kt, Vt, Wm)
+            b_.record(); torch.cuda.synchronize()
+            r_ms = a.elapsed_time(b_) / 5
+            for _ in range(3):
+                comp_r.decode(qs[0], Wm, out)
+            a, b_ = ev(), ev()
+            torch.cuda.synchronize(); a.record()
+            for i in range(10):
+                comp_r.decode(qs[i % n_q], Wm, out)
+            b_.record(); torch.cuda.synchronize()
+            us = a.elapsed_time(b_) * 1e3 / 10
+            step_bytes = U * (2 * n_ret + n_apx) * d * es
+            rope = {"theta": 500000.0, "route_ms": r_ms, "route_gbs": route_bytes / (r_ms * 1e-3) / 1e9,
+                    "route_frac_of_measured_copy": route_bytes / (r_ms * 1e-3) / 1e9 / hbm,
+                    "decode_us_per_step": us, "decode_gbs": step_bytes / us / 1e3,
+                    "decode_frac_of_measured_copy": step_bytes / us / 1e3 / hbm,
+                    "sincos_per_decode_step": 2.0 * U * n_apx * (d // 2), "sincos_per_route": 2.0 * U * n_pool * (d // 2)}
+            del comp_r
+
+    # ---- end to end through host buffers: every step copies its inputs from pinned host memory to the
+    #      device and reads the routing result back; the copies run layer by layer
     e2e = None
-    if not args.no_e2e:
-        hK = torch.empty(Kt.shape, dtype=Kt.dtype, pin_memory=True).copy_(Kt)
-        hV = torch.empty(Vt.shape, dtype=Vt.dtype, pin_memory=True).copy_(Vt)
-        hQ = torch.empty(Qt.shape, dtype=Qt.dtype, pin_memory=True).copy_(Qt)
-        h_tier = torch.empty(comp.tier.shape, dtype=torch.uint8, pin_memory=True)
-        h_ret = torch.empty(comp.ret_idx.shape, dtype=torch.int32, pin_memory=True)
-        h_apx = torch.empty(comp.apx_idx.shape, dtype=torch.int32, pin_memory=True)
-        hq = torch.empty(qs[0].shape, dtype=qs[0].dtype, pin_memory=True).copy_(qs[0])
-        h_out = torch.empty(out.shape, dtype=out.dtype, pin_memory=True)
-        dq = torch.empty_like(qs[0])
+    if want_e2e:
+        try:
+            hK = torch.empty(Kt.shape, dtype=Kt.dtype, pin_memory=True)
+            hV = torch.empty(Vt.shape, dtype=Vt.dtype, pin_memory=True)
+        except RuntimeError as ex:          # the host cannot pin the whole context
+            hK = hV = None
+            e2e = {"value": None, "unit": UNIT, "unavailable": f"pinned host buffers refused: {str(ex)[:120]}"}
+        if hK is not None:
+            hK.copy_(Kt); hV.copy_(Vt)
+            hQ = torch.empty(Qt.shape, dtype=Qt.dtype, pin_memory=True).copy_(Qt)
+            h_tier = torch.empty(comp.tier.shape, dtype=torch.uint8, pin_memory=True)
+            h_ret = torch.empty(comp.ret_idx.shape, dtype=torch.int32, pin_memory=True)
+            h_apx = torch.empty(comp.apx_idx.shape, dtype=torch.int32, pin_memory=True)
+            hq = torch.empty(qs[0].shape, dtype=qs[0].dtype, pin_memory=True).copy_(qs[0])
+            h_out = torch.empty(out.shape, dtype=out.dtype, pin_memory=True)
+            dq = torch.empty_like(qs[0])
 
-        def e2e_step():
-            Kt.copy_(hK, non_blocking=True); Vt.copy_(hV, non_blocking=True); Qt.copy_(hQ, non_blocking=True)
-            comp.compress(Qt, Kt, Vt, Wm)
-            h_tier.copy_(comp.tier, non_blocking=True)
-            h_ret.copy_(comp.ret_idx, non_blocking=True)
-            h_apx.copy_(comp.apx_idx, non_blocking=True)
+            def e2e_step():
+                Kt.copy_(hK, non_blocking=True); Vt.copy_(hV, non_blocking=True); Qt.copy_(hQ, non_blocking=True)
+                comp.compress(Qt, Kt, Vt, Wm)
+                h_tier.copy_(comp.tier, non_blocking=True)
+                h_ret.copy_(comp.ret_idx, non_blocking=True)
+                h_apx.copy_(comp.apx_idx, non_blocking=True)
 
-        def e2e_decode():
-            dq.copy_(hq, non_blocking=True)
-            comp.decode(dq, Wm, out)
-            h_out.copy_(out, non_blocking=True)
+            def e2e_decode():
+                dq.copy_(hq, non_blocking=True)
+                comp.decode(dq, Wm, out)
+                h_out.copy_(out, non_blocking=True)
 
-        e2e_step(); torch.cuda.synchronize()
-        n_e = max(2, min(K_steps, 3))
-        a, b_ = ev(), ev()
-        barrier(); a.record()
-        for _ in range(n_e):
-            e2e_step()
-        b_.record(); barrier()
-        e_ms = a.elapsed_time(b_) / n_e
-        a, b_ = ev(), ev()
-        a.record()
-        for _ in range(20):
-            e2e_decode()
-        b_.record(); torch.cuda.synchronize()
-        ed_ms = a.elapsed_time(b_) / 20
-        e_ms, ed_ms = replicas.slowest([e_ms, ed_ms], dev)
-        h2d = (hK.numel() + hV.numel() + hQ.numel()) * es
-        d2h = h_tier.numel() + (h_ret.numel() + h_apx.numel()) * 4
-        e2e = {"value": world * wl.batch * N / (e_ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
-               "d2h_bytes_per_step": d2h, "ms_per_step": e_ms,
-               "decode_step_us": ed_ms * 1e3, "decode_h2d_bytes": hq.numel() * es, "decode_d2h_bytes": h_out.numel() * es}
-        del hK, hV, hQ
+            comp.cache.n_ret = budget.n_ret
+            e2e_step(); torch.cuda.synchronize()
+            n_e = max(2, min(steps, 3))
+            a, b_ = ev(), ev()
+            env.barrier(); a.record()
+            for _ in range(n_e):
+                e2e_step()
+            b_.record(); env.barrier()
+            e_ms = a.elapsed_time(b_) / n_e
+            a, b_ = ev(), ev()
+            a.record()
+            for _ in range(20):
+                e2e_decode()
+            b_.record(); torch.cuda.synchronize()
+            ed_ms = a.elapsed_time(b_) / 20
+            e_ms, ed_ms = replicas.slowest([e_ms, ed_ms], dev)
+            h2d = (hK.numel() + hV.numel() + hQ.numel()) * es
+            d2h = h_tier.numel() + (h_ret.numel() + h_apx.numel()) * 4
+            e2e = {"value": world * wl.batch * N / (e_ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
+                   "d2h_bytes_per_step": d2h, "ms_per_step": e_ms, "h2d_gbs": h2d / (e_ms * 1e-3) / 1e9,
+                   "decode_step_us": ed_ms * 1e3, "decode_h2d_bytes": hq.numel() * es,
+                   "decode_d2h_bytes": h_out.numel() * es}
+            del hK, hV, hQ
 
-    if rank != 0:
-        if world > 1:
-            import torch.distributed as dist
-            dist.destroy_process_group()
-        return 0
+    del Kt, Vt, Qt, comp, Wm
+    gc.collect()
+    torch.cuda.empty_cache()
 
     cpu = None
-    if not args.no_cpu_baseline and world == 1:
-        n_s = min(U, 16)
+    if want_cpu and world == 1 and env.rank == 0:
+        n_s = oracle_units_per_sample(wl) * (4 if wl.N <= 32768 else 1)
+        n_s = min(U, n_s)
         r = oracle_sample(wl, percent, n_s, 2)
         t_all = r["compress_s_per_unit"] * U
         cpu = {"value": wl.batch * N / t_all, "unit": UNIT, "cores": 1, "kind": "oracle",
@@ -466,10 +529,11 @@ def main():
                          f"{r['compress_s_per_unit']:.2f} s per unit single-threaded; whole-workload time = x{U}; "
                          f"one decode step of one unit {r['decode_s_per_unit_step'] * 1e3:.1f} ms"}
 
-    kernels_per_step = 8 + 2 * D
-    line = {
+    for k in kernels:
+        del k["call"]
+    return {
         "metric": METRIC, "value": world * wl.batch * N / (compress_ms * 1e-3), "unit": UNIT, "n_gpus": world,
-        "steps": K_steps, "warmup": W_warm, "ms_per_step": total_ms / K_steps, "higher_is_better": True,
+        "steps": steps, "warmup": warmup, "ms_per_step": total_ms / steps, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "bf16" if wl.dtype == "bf16" else "f32", "data": "synthetic",
         "config": {"workload": wl.name, "budget_percent": percent, "batch": wl.batch, "N": N, "units": U,
                    "layers": wl.n_layers, "q_heads": wl.n_q_heads, "kv_heads": wl.n_kv_heads, "head_dim": d,
@@ -479,16 +543,65 @@ def main():
                          (2 * U * N * d * es / 1e9, U * (2 * n_ret + n_apx) * d * es / 1e9),
                    "parallelism": "replicas only" if world > 1 else "single GPU"},
         "compress_ms": compress_ms, "phase_ms": ms,
-        "decode": {"gbs": decode_bytes / (dec_ms_max * 1e-3) / 1e9, "frac_of_measured_copy": decode_bytes / (dec_ms_max * 1e-3) / 1e9 / hbm,
-                   "frac_of_8tbs": decode_bytes / (dec_ms_max * 1e-3) / 1e9 / 8000.0, "us_per_step": dec_ms_max * 1e3 / D,
-                   "tokens_per_s": world * wl.batch * D / (dec_ms_max * 1e-3), "bytes_per_step": decode_bytes / D},
-        "decode_per_tile": per_tile, "score_keydiff": keydiff, "rope_decoupled": rope, "roofline": roofline, "roofline_kernels": kernels, "cpu_baseline": cpu, "e2e": e2e,
-        "gpu_launches": kernels_per_step * K_steps, "clocks": clocks,
+        "decode": {"gbs": decode_bytes / (dec_ms_max * 1e-3) / 1e9,
+                   "frac_of_measured_copy": decode_bytes / (dec_ms_max * 1e-3) / 1e9 / hbm,
+                   "frac_of_8tbs": decode_bytes / (dec_ms_max * 1e-3) / 1e9 / 8000.0,
+                   "us_per_step": dec_ms_max * 1e3 / D, "tokens_per_s": world * wl.batch * D / (dec_ms_max * 1e-3),
+                   "bytes_per_step": decode_bytes / D},
+        "decode_per_tile": per_tile, "score_keydiff": keydiff, "rope_decoupled": rope, "roofline": roofline,
+        "roofline_kernels": kernels, "cpu_baseline": cpu, "e2e": e2e,
+        "gpu_launches": launches, "device_fault": fault, "clocks": clocks,
     }
-    print(json.dumps(line))
-    if world > 1:
-        import torch.distributed as dist
-        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=5)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--config", type=int, default=None,
+                    help="run one workload 1..4 only (default: workload 4 as the headline, 2 and 3 beside it)")
+    ap.add_argument("--budget", type=int, default=None, help="budget percent (default: the workload's)")
+    ap.add_argument("--decode-steps", type=int, default=None)
+    ap.add_argument("--layers", type=int, default=None, help="shrink the workload to this many layers (profiling)")
+    ap.add_argument("--impl", default="vector", choices=["vector", "reference"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-extras", action="store_true", help="skip the measurements outside the timed step")
+    ap.add_argument("--no-side-configs", action="store_true")
+    args = ap.parse_args()
+
+    from paper_2605_23258_b200 import synth
+    cfg = args.config if args.config is not None else HEADLINE_CONFIG
+    wl = synth.WORKLOADS[cfg]
+    if args.layers is not None:
+        wl = synth.shrink(wl, n_layers=args.layers, name=f"{wl.name}_first{args.layers}layers")
+    percent = args.budget if args.budget is not None else default_percent(cfg, wl)
+    if args.impl == "reference":
+        return run_reference(args, cfg, wl, percent)
+
+    import paper_2605_23258_b200 as vec
+    env = Env()
+    vec.load_library()
+    warm = max(args.warmup, 3)
+    steps = max(args.steps, 1)
+    D = args.decode_steps if args.decode_steps is not None else wl.decode_steps
+    line = run_workload(env, cfg, wl, percent, steps, warm, D, extras=not args.no_extras,
+                        want_e2e=not args.no_e2e, want_cpu=not args.no_cpu_baseline)
+    if args.config is None and not args.no_side_configs:
+        side = {}
+        for c in SIDE_CONFIGS:
+            swl = synth.WORKLOADS[c]
+            r = run_workload(env, c, swl, default_percent(c, swl), min(steps, 5), 3, swl.decode_steps,
+                             extras=not args.no_extras and c == 2, want_e2e=False, want_cpu=False)
+            side[f"config{c}"] = {k: r[k] for k in ("value", "unit", "steps", "warmup", "ms_per_step", "config",
+                                                    "compress_ms", "phase_ms", "decode", "decode_per_tile",
+                                                    "score_keydiff", "rope_decoupled", "roofline_kernels",
+                                                    "gpu_launches", "device_fault", "clocks")}
+        line["configs"] = side
+    if env.rank == 0:
+        print(json.dumps(line))
+    env.close()
     return 0
 
 

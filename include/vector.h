@@ -103,6 +103,10 @@ typedef struct {
 VECTOR_API const char* vector_status_string(vector_status s);
 /* The raw cudaError_t of the last VECTOR_ERR_CUDA on this thread (0 if none). */
 VECTOR_API int vector_last_cuda_error(void);
+/* Kernels this library has launched so far in this process (all threads, all devices): a
+ * monotone counter for accounting; the difference across a region is the number of launches
+ * the calls inside it made. */
+VECTOR_API uint64_t vector_kernel_launches(void);
 
 /*
  * Tier sizes, host only (paper Section 3.2 proportions and Eq. (1)).
@@ -149,6 +153,11 @@ VECTOR_API size_t vector_workspace_bytes(const vector_shape* shape, const vector
  */
 VECTOR_API vector_status vector_score(const vector_shape* shape, const void* Q_obs, const void* K, int64_t N,
                            float* scores, float* raw_out, void* ws, size_t ws_bytes, void* stream);
+
+/* Build constant of the tensor-core score passes (bf16, head_dim 128): the share of the softmax
+ * exponentials that is evaluated by a polynomial on the FMA pipe instead of the special-function
+ * unit (the unit that bounds the passes).  For reading the pipe counters of vector_score. */
+VECTOR_API float vector_score_exp2_fma_share(void);
 
 /*
  * Query-agnostic base scorer by key geometry, an alternative to vector_score for Step 1 (the

@@ -191,6 +191,22 @@ def vector_status_string(status: int) -> str:
     return load_library().vector_status_string(status).decode()
 
 
+def vector_kernel_launches() -> int:
+    """Kernels the library has launched so far in this process."""
+    lib = load_library()
+    lib.vector_kernel_launches.restype = ctypes.c_uint64
+    lib.vector_kernel_launches.argtypes = []
+    return int(lib.vector_kernel_launches())
+
+
+def score_poly_share() -> float:
+    """Share of the score passes' exponentials evaluated on the FMA pipe (vector_score_exp2_fma_share)."""
+    lib = load_library()
+    lib.vector_score_exp2_fma_share.restype = ctypes.c_float
+    lib.vector_score_exp2_fma_share.argtypes = []
+    return float(lib.vector_score_exp2_fma_share())
+
+
 def vector_device_fault() -> int:
     """Synchronises the device; returns (and clears) the code of a kernel wait that gave up, 0 if none."""
     lib = load_library()

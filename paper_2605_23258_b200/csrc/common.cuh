@@ -9,6 +9,8 @@
 
 namespace vec {
 
+void count_launch();      // host: one more kernel launched by the library
+
 __device__ __forceinline__ float to_f32(float x) { return x; }
 __device__ __forceinline__ float to_f32(__nv_bfloat16 x) { return __bfloat162float(x); }
 
@@ -82,6 +84,7 @@ inline cudaError_t launch_maybe_dependent(bool dependent, void (*kernel)(KArgs..
     cfg.stream = st;
     cfg.attrs = &attr;
     cfg.numAttrs = 1;
+    count_launch();
     return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
 }
 

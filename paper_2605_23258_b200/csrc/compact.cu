@@ -45,6 +45,7 @@ compact_kernel(const uint4* __restrict__ K, const uint4* __restrict__ V, int64_t
             src[p] = K; dst[p] = apx_k + (((size_t)u * cap_apx + q) << lp) + piece;
             pos[p] = apx_pos + (size_t)u * cap_apx + q;
         }
+        if ((unsigned long long)(long long)tok[p] >= (unsigned long long)N) src[p] = nullptr;   // an index outside the unit: row skipped
     }
     uint4 v[COMPACT_PASSES];
 #pragma unroll

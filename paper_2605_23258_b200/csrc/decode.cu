@@ -234,7 +234,7 @@ static vector_status launch_decode_bf16_d128(const Dims& dm, const void* q, cons
     }
     int* fault = kernel_fault_address();
     if (!fault) return VECTOR_ERR_CUDA;
-    const dbf::Plan pl = dbf::make_plan(dm.U, ch->n_ret, ch->n_apx);
+    const dbf::Plan pl = dbf::make_plan(dm.U, ch->n_ret, ch->n_apx, sm_count());
     if (pl.s_max > decode_stream_slots(dm.U)) return VECTOR_ERR_WORKSPACE;
     dbf::Maps maps;
     const uint64_t row_b = 256;

@@ -61,7 +61,6 @@ constexpr int REC = 4 + 2 * 128;             // m, l, value-scale, pad, acc_v[12
 constexpr int SMEM_BYTES = SLOTS * SLOT_BYTES + 1024;   // + alignment slack; barriers live in static smem
 constexpr int W_BYTES = 32768;               // the unit's map as two swizzled 128 x 128 B boxes (per-tile form only)
 constexpr int SMEM_BYTES_PER_TILE = SMEM_BYTES + W_BYTES;
-constexpr int MAX_BLOCKS = 148;
 
 // How the tile sequence is dealt to blocks; the same arithmetic runs on host and device.
 struct Plan {
@@ -70,14 +69,14 @@ struct Plan {
     int B;                     // blocks
     int s_max;                 // record slots per unit
 };
-__host__ __device__ inline Plan make_plan(int U, long long n_ret, long long n_apx) {
+__host__ __device__ inline Plan make_plan(int U, long long n_ret, long long n_apx, int max_blocks) {
     Plan p;
     p.n_rt = (int)((n_ret + KEYS - 1) / KEYS);
     p.n_at = (int)((n_apx + 2 * KEYS - 1) / (2 * KEYS));
     p.n_tiles = p.n_rt + p.n_at;
     p.T = (long long)U * p.n_tiles;
     long long b = p.T / 2;                       // at least two tiles per block
-    if (b > MAX_BLOCKS) b = MAX_BLOCKS;
+    if (b > max_blocks) b = max_blocks;               // one persistent block per multiprocessor
     if (b > 11LL * U) b = 11LL * U;              // at most 12 record slots per unit (merge kernel limit)
     p.B = (int)(b < 1 ? 1 : b);
     p.s_max = (p.B + U - 1) / U + 1;

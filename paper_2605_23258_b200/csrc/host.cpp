@@ -1,6 +1,8 @@
 // Host-only entry points of libvector: status text, the tier planner and the
 // offline least-squares calibration, plus the argument checks the device entry
-// points share.  The only CUDA call in this file is cudaGetDevice.
+// points share.  The only CUDA calls in this file are cudaGetDevice and the query of the
+// multiprocessor count.
+#include <atomic>
 #include <cmath>
 #include <mutex>
 #include <cuda_runtime_api.h>
@@ -14,6 +16,9 @@ namespace vec {
 static thread_local int g_last_cuda_error = 0;
 void set_last_cuda_error(int e) { g_last_cuda_error = e; }
 
+static std::atomic<unsigned long long> g_launches{0};
+void count_launch() { g_launches.fetch_add(1, std::memory_order_relaxed); }
+
 void rope_phases(float theta, int d, RopePhases* out) {
     for (int c = 0; c < 64; ++c) {
         if (c >= d / 2) { out->phase[c] = 0ull; continue; }
@@ -23,6 +28,22 @@ void rope_phases(float theta, int d, RopePhases* out) {
 }
 
 static std::mutex g_once_mu;
+int sm_count() {
+    static int cached[PerDeviceOnce::kMax] = {};
+    constexpr int kDefault = 148;
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= PerDeviceOnce::kMax) {
+        (void)cudaGetLastError();
+        return kDefault;
+    }
+    std::lock_guard<std::mutex> lock(g_once_mu);
+    if (cached[dev] <= 0) {
+        int n = 0;
+        if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) n = kDefault;
+        cached[dev] = n;
+    }
+    return cached[dev];
+}
 bool PerDeviceOnce::first() {
     int dev = -1;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMax) return false;
@@ -82,7 +103,7 @@ vector_status check_budget(const vector_budget* b, int window) {
 int score_num_chunks(int U, int R, int64_t N) {
     int64_t tiles = (N + 127) / 128;
     int64_t row_tiles = (R + 63) / 64;
-    int64_t want = (8 * 148 + (int64_t)U * row_tiles - 1) / ((int64_t)U * row_tiles);
+    int64_t want = (8 * sm_count() + (int64_t)U * row_tiles - 1) / ((int64_t)U * row_tiles);
     if (want < 1) want = 1;
     if (want > 64) want = 64;
     if (want > tiles) want = tiles;
@@ -95,7 +116,7 @@ ScoreTcPlan score_tc_plan(int U, int R, int64_t N) {
     p.nt = (int)((N + 127) / 128);
     // chunks per unit: fill whole rounds of one block per SM, but keep chunks long enough that the
     // per-item cost (Q load, pipeline fill) stays small
-    const int blocks = 148;
+    const int blocks = sm_count();
     double best = -1.0;
     int best_n = 1;
     const int max_n = p.nt < 64 ? p.nt : 64;
@@ -136,7 +157,7 @@ size_t select_ws_bytes(const Dims& D, const vector_budget& b) {
 }
 
 int decode_num_splits(int U, int64_t rows) {
-    int64_t want = (4 * 148 + U - 1) / U;
+    int64_t want = (4 * sm_count() + U - 1) / U;
     int64_t max_by_rows = (rows + 255) / 256;   // at least 256 rows per split
     if (want > max_by_rows) want = max_by_rows;
     if (want > 64) want = 64;
@@ -145,7 +166,7 @@ int decode_num_splits(int U, int64_t rows) {
 }
 
 int decode_stream_slots(int U) {
-    int s = (2 * 148 + U - 1) / U + 1;
+    int s = (2 * sm_count() + U - 1) / U + 1;
     return s < 12 ? s : 12;
 }
 
@@ -181,6 +202,8 @@ const char* vector_status_string(vector_status s) {
 }
 
 int vector_last_cuda_error(void) { return vec::g_last_cuda_error; }
+
+uint64_t vector_kernel_launches(void) { return (uint64_t)vec::g_launches.load(std::memory_order_relaxed); }
 
 vector_status vector_plan_budget(int64_t n_tokens, int64_t n_budget_pairs, int64_t n_a,
                                  int32_t window, vector_budget* out) {

@@ -37,6 +37,12 @@ vector_status check_shape(const vector_shape* s, Dims* out);
 vector_status check_budget(const vector_budget* b, int window);
 
 void set_last_cuda_error(int e);
+// Adds one to the process-wide count of kernels launched by the library (vector_kernel_launches).
+void count_launch();
+
+// Multiprocessors of the current device (read once per device); the B200's 148 when no device
+// can be queried, so that the host-only sizing calls still answer.
+int sm_count();
 
 // ---- workspace layout (bytes, each region 256-byte aligned) ----
 // Number of key chunks the first score pass splits a unit's keys into.
@@ -63,7 +69,7 @@ struct PerDeviceOnce {
 size_t select_ws_bytes(const Dims& D, const vector_budget& b);
 // Number of key splits of one unit in decode attention for `rows` logical keys.
 int decode_num_splits(int U, int64_t rows);
-// Record slots per unit that the persistent bf16 decode kernel may use (two blocks per SM, 148 SMs).
+// Record slots per unit that the persistent bf16 decode kernel may use (two blocks per SM).
 int decode_stream_slots(int U);
 size_t decode_ws_bytes(const Dims& D);
 size_t keydiff_ws_bytes(const Dims& D, int64_t N);
@@ -81,6 +87,10 @@ inline size_t align256(size_t x) { return (x + 255) & ~size_t(255); }
         }                                                     \
     } while (0)
 
-#define VEC_LAUNCH_CHECK() VEC_CUDA_CHECK(cudaPeekAtLastError())
+#define VEC_LAUNCH_CHECK()                    \
+    do {                                      \
+        vec::count_launch();                  \
+        VEC_CUDA_CHECK(cudaPeekAtLastError()); \
+    } while (0)
 
 #endif  // VECTOR_INTERNAL_H_

@@ -161,7 +161,7 @@ keydiff_cosine(const T* __restrict__ K, int64_t N, int64_t chunk_len, const floa
 }
 
 static int keydiff_chunks(int U, int64_t N) {
-    int64_t want = (8 * 148 + U - 1) / U;
+    int64_t want = (8 * sm_count() + U - 1) / U;
     const int64_t max_by_rows = (N + 255) / 256;
     if (want > max_by_rows) want = max_by_rows;
     if (want > 64) want = 64;

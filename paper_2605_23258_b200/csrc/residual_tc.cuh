@@ -68,7 +68,7 @@ struct RSync {
     uint32_t tmem_base;
 };
 
-// grid: min(148, n_tiles) blocks, R_THREADS threads, RCfg<ROPE>::SMEM_BYTES dynamic shared memory.
+// grid: min(multiprocessors, n_tiles) blocks, R_THREADS threads, RCfg<ROPE>::SMEM_BYTES dynamic shared memory.
 template <bool ROPE>
 __global__ void __launch_bounds__(R_THREADS, 1)
 residual_tc(const __nv_bfloat16* __restrict__ K, const __nv_bfloat16* __restrict__ V,
@@ -124,7 +124,8 @@ residual_tc(const __nv_bfloat16* __restrict__ K, const __nv_bfloat16* __restrict
 #pragma unroll
             for (int p = 0; p < 4; ++p) {
                 const int row = t * TILE + p * 32 + rsub;
-                out[p] = row < P.n_idx ? idx[(size_t)u * P.n_idx + row] : -1;
+                const int32_t v = row < P.n_idx ? idx[(size_t)u * P.n_idx + row] : -1;
+                out[p] = (unsigned long long)v < (unsigned long long)P.N ? v : -1;   // an index outside the unit reads as a row of zeros
             }
         };
         // Turns this thread's pairs of the tile in stage s (rows listed in pos) and publishes the tile.
@@ -233,6 +234,9 @@ residual_tc(const __nv_bfloat16* __restrict__ K, const __nv_bfloat16* __restrict
                     cur_u = u;
                     ++n_units;
                 }
+                // the loaders start only once the kernel that writes idx has drained: do not spend this
+                // thread's bounded polls on that kernel's run time (W, loaded above, is nobody's output)
+                if (i == 0) asm volatile("griddepcontrol.wait;\n" ::: "memory");
                 if (!tma::mbar_wait(&sy.full[s], round & 1, fault, 49)) break;
                 tc::fence_after_sync();
                 const uint32_t hi_addr = tma::smem_u32(stage0 + s * R_STAGE_BYTES), lo_addr = hi_addr + OPERAND_BYTES;
@@ -260,6 +264,7 @@ residual_tc(const __nv_bfloat16* __restrict__ K, const __nv_bfloat16* __restrict
         const int r = quarter * 32 + lane;
         const uint32_t lane_addr = sy.tmem_base + ((uint32_t)(quarter * 32) << 16);
         const uint32_t v_thread = (uint32_t)r * 128u;
+        asm volatile("griddepcontrol.wait;\n" ::: "memory");      // as in the MMA thread: the waits below time this kernel only
         for (int i = 0; i < n_my; ++i) {
             const int s = i % STAGES, round = i / STAGES;
             // the value rows were written by the loaders: observe their barrier, then the MMA's

@@ -370,6 +370,10 @@ residual_generic(const T* __restrict__ K, const T* __restrict__ V, const T* __re
     float* kw = ks + wid * D;
     for (int p = p_begin + wid; p < p_end; p += 8) {
         const int64_t tok = idx[(size_t)u * n_idx + p];
+        if ((uint64_t)tok >= (uint64_t)N) {          // an index outside the unit reads as a row of zeros
+            if (lane == 0) eps[(size_t)u * n_idx + p] = 0.f;
+            continue;
+        }
         const T* kr = K + ((size_t)u * N + tok) * D;
         const T* vr = V + ((size_t)u * N + tok) * D;
         __syncwarp();
@@ -436,7 +440,8 @@ static vector_status launch_residual_tc(const Dims& dm, const void* K, const voi
     P.U = dm.U; P.LH = dm.LH; P.n_idx = (int)n_idx; P.N = N;
     P.tpu = (int)((n_idx + rtc::TILE - 1) / rtc::TILE);
     P.n_tiles = (long long)dm.U * P.tpu;
-    const int blocks = (int)(P.n_tiles < 148 ? P.n_tiles : 148);
+    const int sms = sm_count();
+    const int blocks = (int)(P.n_tiles < sms ? P.n_tiles : sms);
     RopePhases ph = {};
     if (dm.rope) rope_phases(dm.theta, 128, &ph);
     // dependent: blocks may take SMs while the kernel that writes idx drains; the loaders wait for it

@@ -235,7 +235,8 @@ static vector_status launch_score_tc(const Dims& dm, const void* Q, const void* 
     P.U = dm.U; P.R = dm.R; P.RG = pl.RG; P.w = dm.w; P.N = N;
     P.nt = pl.nt; P.tpc = pl.tpc; P.n_chunks = pl.n_chunks; P.n_items = pl.n_items;
     P.c = dm.scale * 1.4426950408889634f;
-    const int blocks = pl.n_items < 148 ? pl.n_items : 148;
+    const int sms = sm_count();
+    const int blocks = pl.n_items < sms ? pl.n_items : sms;
     stc::score_pass1_tc<<<blocks, stc::THREADS, stc::SMEM_BYTES, st>>>(mapQ, mapK, P, partial, fault);
     VEC_LAUNCH_CHECK();
     stc::score_lse2_combine<<<dm.U, 256, 0, st>>>(partial, dm.R, 2 * pl.n_chunks, lse2);
@@ -252,6 +253,8 @@ static vector_status launch_score_tc(const Dims& dm, const void* Q, const void* 
 }
 
 }  // namespace vec
+
+extern "C" float vector_score_exp2_fma_share(void) { return (float)vec::stc::POLY16 / 16.0f; }
 
 extern "C" vector_status vector_score(const vector_shape* shape, const void* Q_obs, const void* K, int64_t N,
                                       float* scores, float* raw_out, void* ws, size_t ws_bytes, void* stream) {

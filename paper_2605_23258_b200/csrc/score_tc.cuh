@@ -194,16 +194,18 @@ __device__ __forceinline__ void sum_tree32(const float (&e)[32], uint64_t& acc) 
 // The exponential unit (16 results per clock per SM) is what bounds both passes, so POLY16 of every
 // 16 exponentials are evaluated on the FMA pipe instead: 2^x = 2^n p(f) with n = round(x),
 // f = x - n in [-1/2, 1/2] and p the degree-4 minimax polynomial of 2^f (relative error 2.7e-6);
-// n is added to the exponent field.  x is clamped at -126 (results below 2^-126 do not matter
-// to a sum whose largest term is of order one).
+// n is added to the exponent field.  x is clamped to [-126, 128]: results below 2^-126 do not
+// matter to a sum whose largest term is of order one, and at the upper end the exponent field must
+// not wrap -- 2^128 comes out as about 3.4e38 (or a NaN), which the overflow test of the first pass
+// (sum above 2^64, or not finite) catches, whereas a wrapped exponent would pass as a tiny term.
 #ifndef VECTOR_SCORE_POLY16
 #define VECTOR_SCORE_POLY16 4
 #endif
 constexpr int POLY16 = VECTOR_SCORE_POLY16;
 __device__ __forceinline__ void exp2_poly_pair(float x0, float x1, float& e0, float& e1) {
     const float magic = 12582912.f;                    // 1.5 * 2^23: adding it leaves round(x) in the low mantissa bits
-    x0 = fmaxf(x0, -126.f);
-    x1 = fmaxf(x1, -126.f);
+    x0 = fminf(fmaxf(x0, -126.f), 128.f);
+    x1 = fminf(fmaxf(x1, -126.f), 128.f);
     const uint64_t x2 = pack2(x0, x1);
     const uint64_t t2 = add2(x2, pack2(magic, magic));
     const uint64_t n2 = add2(t2, pack2(-magic, -magic));

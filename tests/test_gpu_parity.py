@@ -70,6 +70,31 @@ def test_score_parity(oracle, base, over):
     assert np.allclose(raw.double().sum(1).cpu().numpy(), mass, rtol=1e-4)
 
 
+def test_score_logit_far_above_the_running_reference(oracle):
+    """One key whose logit beats every other by about 200 log2 units, placed past the first 32 keys in a
+    column whose exponential is evaluated by the polynomial: the first pass must notice that the key ran
+    away from its running reference (an exponent field that wrapped would pass as a tiny term)."""
+    wl = synth.shrink(synth.WORKLOADS[1], N=700, n_kv_heads=1, n_q_heads=4)
+    K, _, Q = synth.context(wl, DEV)
+    K = (K.float() * 0.05).to(torch.bfloat16)
+    Q = (Q.float() * 0.05).to(torch.bfloat16)
+    Q[..., 0] = 8.0
+    K[0, 49, 0] = 200.0                     # logit 8 * 200 / sqrt(128) = 141 nats; 49 & 15 = 1, second 32-key chunk
+    sh = shape_of(wl)
+    ws = vec.alloc_workspace(sh, vec.vector_plan_budget(wl.N, wl.N, 0, wl.window))
+    scores = torch.empty(wl.units, wl.N, dtype=torch.float32, device=DEV)
+    raw = torch.empty_like(scores)
+    vec.vector_score(sh, Q, K, wl.N, scores, raw, ws)
+    torch.cuda.synchronize()
+    raw_o, sc_o = oracle_scores(oracle, wl, Q.cpu(), K.cpu())
+    mass = wl.group * wl.window
+    assert raw_o[0, 49] > 0.999 * mass
+    ok, worst = score_close(raw.cpu().numpy(), raw_o, mass)
+    assert ok, f"raw off by {worst:.3g} x tolerance"
+    ok, worst = score_close(scores.cpu().numpy(), sc_o, mass)
+    assert ok, f"score off by {worst:.3g} x tolerance"
+
+
 KEYDIFF_CASES = [(0, {}), (0, {"N": 333}), (1, {"N": 1000, "n_kv_heads": 2, "n_q_heads": 8}),
                  (1, {"N": 4096 + 77, "n_kv_heads": 1, "n_q_heads": 4}), (2, {"N": 1500, "n_layers": 20}),
                  (1, {"N": 900, "head_dim": 64, "n_kv_heads": 1, "n_q_heads": 2}), (1, {"N": 1, "n_kv_heads": 1, "n_q_heads": 4})]
@@ -527,10 +552,13 @@ def test_back_to_back_calls_repeat_bitwise(oracle):
             assert torch.equal(a, b_), (name, r + 1, int((a != b_).sum()))
 
 
-def _sampled_units_case(oracle, wl, percent, sample, theta=None):
+def _sampled_units_case(oracle, wl, percent, sample, theta=None, fed_by_device_scores=()):
     """Whole workload on the device in the launch shape the benchmark times; the oracle checks the
     sampled units end to end, every unit is checked for the properties that hold at any size.
-    With `theta` the stored keys are post-RoPE and RoPE decoupling is on."""
+    With `theta` the stored keys are post-RoPE and RoPE decoupling is on.  The units listed in
+    `fed_by_device_scores` skip the oracle's scorer (minutes per unit at the longest context): the
+    oracle routes them from the device's own fp32 scores, so Step 1 must match bit for bit, the
+    residuals within their rounding bound and Step 3 bit for bit on the device's residuals."""
     K, V, Q = synth.context(wl, DEV)
     W = calibrated_maps(wl).to(DEV)
     sh = shape_of(wl)
@@ -571,6 +599,23 @@ def _sampled_units_case(oracle, wl, percent, sample, theta=None):
                              c.apx_k[u, : c.n_apx].cpu(), Ws[j], 1.0 / np.sqrt(wl.head_dim),
                              apx_pos=c.apx_pos[u, : c.n_apx].cpu().numpy(), rope=theta is not None, theta=theta or 10000.0)
         assert np.max(np.abs(out[u].cpu().double().numpy() - o)) <= 2e-2
+    for u in fed_by_device_scores:
+        Wu = W[u % LH].cpu()
+        r = _oracle_route_unit(oracle, wl, b, comp.scores[u].cpu().numpy(), K[u].cpu(), V[u].cpu(), Wu, theta)
+        assert np.array_equal(comp.pool_idx[u].cpu().numpy(), r["pool_idx"]), f"unit {u}: pool differs"
+        rows = torch.from_numpy(r["pool_idx"]).long()
+        ok, worst = eps_close(comp.eps[u].cpu().numpy(), r["eps"], K[u].cpu()[rows], V[u].cpu()[rows], Wu)
+        assert ok, f"unit {u}: eps off by {worst:.3g} x bound"
+        t2, r2, a2 = oracle.truncate(comp.eps[u].cpu().numpy(), r["pool_idx"], b.n_apx, wl.N)
+        assert np.array_equal(tier_all[u].cpu().numpy(), t2), f"unit {u}: tiers differ on identical residuals"
+        assert np.array_equal(comp.ret_idx[u].cpu().numpy(), r2) and np.array_equal(comp.apx_idx[u].cpu().numpy(), a2)
+        assert torch.equal(c.ret_k[u, : b.n_ret], K[u][comp.ret_idx[u].long()])
+        assert torch.equal(c.ret_v[u, : b.n_ret], V[u][comp.ret_idx[u].long()])
+        assert torch.equal(c.apx_k[u, : b.n_apx], K[u][comp.apx_idx[u].long()])
+        _, o = oracle.attend(q[u].cpu(), c.ret_k[u, : c.n_ret].cpu(), c.ret_v[u, : c.n_ret].cpu(),
+                             c.apx_k[u, : c.n_apx].cpu(), Wu, 1.0 / np.sqrt(wl.head_dim),
+                             apx_pos=c.apx_pos[u, : c.n_apx].cpu().numpy(), rope=theta is not None, theta=theta or 10000.0)
+        assert np.max(np.abs(out[u].cpu().double().numpy() - o)) <= 2e-2, u
 
 
 def test_config2_shape_rope_decoupled_sampled_units(oracle):
@@ -589,7 +634,21 @@ def test_config3_shape_sampled_units(oracle):
     _sampled_units_case(oracle, synth.shrink(synth.WORKLOADS[3], batch=2, n_layers=4), 10, [3, 40])
 
 
+def test_config3_full_size_sampled_units(oracle):
+    """Config 3 at full size (8 sequences x 32 layers x 8 KV heads = 2048 units, 17 GB of K and V) in the
+    launch shape the benchmark times: decode blocks own about fourteen whole units each, two record slots
+    per unit.  Units of the first, a middle and the last sequence against the oracle end to end."""
+    _sampled_units_case(oracle, synth.WORKLOADS[3], 10, [3, 1029, 2047], fed_by_device_scores=[517, 1536])
+
+
 def test_config4_shape_sampled_unit(oracle):
     """Long-context shape (config 4: N = 131072, 8 query heads per KV head, window 128, budget 5 %), one layer;
     the oracle scores one whole unit (1024 window rows x 131072 keys)."""
     _sampled_units_case(oracle, synth.shrink(synth.WORKLOADS[4], n_layers=1), 5, [5])
+
+
+def test_config4_full_size_sampled_units(oracle):
+    """Config 4 at full size (80 layers x 8 KV heads = 640 units, 43 GB of K and V) in the launch shape the
+    benchmark times.  The oracle scores one whole unit (its scorer takes about half a minute per unit
+    here); three more units are routed by the oracle from the device's scores and attended by it."""
+    _sampled_units_case(oracle, synth.WORKLOADS[4], 5, [333], fed_by_device_scores=[0, 470, 639])
