@@ -182,7 +182,9 @@ def _selection_inputs(U, N, seed, ties):
                                            # more candidates after the first digit than the list holds, with
                                            # and without the bit masks (N above 32768), and nothing but ties
                                            (20000, 7000, "narrow"), (70000, 20000, "narrow"), (32768, 11000, "equal"),
-                                           (40000, 100, "equal")])
+                                           (40000, 100, "equal"),
+                                           # longer than the bit masks kept in shared memory can cover
+                                           (400000, 50000, True), (400000, 150001, "narrow"), (4097, 33, True)])
 def test_pool_select_bit_exact(oracle, N, n_pool, ties):
     U = 3
     s = _selection_inputs(U, N, N + n_pool, ties)
@@ -221,7 +223,8 @@ def test_residual_parity(oracle, base, over, n_idx):
 @pytest.mark.parametrize("N,n_pool,n_apx,ties", [(1024, 384, 256, False), (1024, 384, 256, True),
                                                  (4000, 1501, 0, True), (4000, 1500, 1500, True),
                                                  (131072, 9829, 6552, False), (50, 20, 2, True),
-                                                 (32768, 11468, 6552, "narrow"), (131072, 45000, 30000, "narrow")])
+                                                 (32768, 11468, 6552, "narrow"), (131072, 45000, 30000, "narrow"),
+                                                 (16384, 2457, 1638, False), (500000, 450000, 200000, True)])
 def test_truncate_bit_exact(oracle, N, n_pool, n_apx, ties):
     U = 3
     g = torch.Generator().manual_seed(N + n_apx)
