@@ -13,6 +13,7 @@
 
 #include "common.cuh"
 #include "decode_bf16.cuh"
+#include "decode_pertile_tc.cuh"
 #include "internal.h"
 
 namespace vec {
@@ -230,6 +231,8 @@ static vector_status launch_decode_bf16_d128(const Dims& dm, const void* q, cons
         if (e == cudaSuccess)
             e = cudaFuncSetAttribute(dbf::decode_stream_bf16_d128<true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                      dbf::SMEM_BYTES_PER_TILE);
+        if (e == cudaSuccess)
+            e = cudaFuncSetAttribute(dpt::decode_stream_pertile_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, dpt::SMEM_BYTES);
         if (e != cudaSuccess) { once.undo(); VEC_CUDA_CHECK(e); }
     }
     int* fault = kernel_fault_address();
@@ -255,10 +258,16 @@ static vector_status launch_decode_bf16_d128(const Dims& dm, const void* q, cons
     const float c2 = dm.scale * 1.4426950408889634f;
     RopePhases ph = {};
     if (dm.rope) rope_phases(dm.theta, 128, &ph);
-    if (mode == 1)
-        dbf::decode_stream_bf16_d128<true, false><<<pl.B, dbf::THREADS, dbf::SMEM_BYTES_PER_TILE, st>>>(
-            (const T*)q, maps, pl, (int)ch->n_ret, (int)ch->n_apx, dm.g, dm.LH, c2, partial, fault, nullptr, 0, ph);
-    else if (dm.rope)
+    if (mode == 1) {
+        // reconstruction tile by tile on the tensor cores: its own streaming kernel, two consumer warps
+        dpt::Maps pm;
+        pm.ret_k = maps.ret_k; pm.ret_v = maps.ret_v; pm.w = maps.w; pm.apx_k = maps.apx_k;
+        if (ch->n_apx > 0 && !tma::encode_bf16_3d(&pm.apx_k, ch->apx_k, 128, (uint64_t)ch->n_apx, (uint64_t)dm.U, row_b,
+                                                  (uint64_t)ch->cap_apx * row_b, 64, 128))
+            return VECTOR_ERR_CUDA;
+        dpt::decode_stream_pertile_tc<<<pl.B, dpt::THREADS, dpt::SMEM_BYTES, st>>>(
+            (const T*)q, pm, pl, (int)ch->n_ret, (int)ch->n_apx, dm.g, dm.LH, c2, partial, fault);
+    } else if (dm.rope)
         dbf::decode_stream_bf16_d128<false, true><<<pl.B, dbf::ROPE_THREADS, dbf::SMEM_BYTES, st>>>(
             (const T*)q, maps, pl, (int)ch->n_ret, (int)ch->n_apx, dm.g, dm.LH, c2, partial, fault, ch->apx_pos,
             (long long)ch->cap_apx, ph);
@@ -269,13 +278,14 @@ static vector_status launch_decode_bf16_d128(const Dims& dm, const void* q, cons
     // programmatic dependent launch: the merge blocks start while the streaming kernel drains
     const float* rec = partial;
     const int apply_w = mode == 1 ? 0 : 1;
+    const int cw = mode == 1 ? dpt::CONSUMERS : dbf::CONSUMER_WARPS;      // records a block leaves per unit
     const T* Wp = (const T*)W;
     if (out_dtype == VECTOR_F32)
         VEC_CUDA_CHECK(launch_maybe_dependent(true, dbf::decode_merge_bf16_d128<float>, dim3(dm.U), dim3(128 * dm.g), 0, st, rec,
-                                              Wp, dm.LH, dm.g, pl, apply_w, (float*)out));
+                                              Wp, dm.LH, dm.g, pl, apply_w, cw, (float*)out));
     else
         VEC_CUDA_CHECK(launch_maybe_dependent(true, dbf::decode_merge_bf16_d128<T>, dim3(dm.U), dim3(128 * dm.g), 0, st, rec, Wp,
-                                              dm.LH, dm.g, pl, apply_w, (T*)out));
+                                              dm.LH, dm.g, pl, apply_w, cw, (T*)out));
     return VECTOR_OK;
 }
 

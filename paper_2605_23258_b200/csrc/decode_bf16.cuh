@@ -626,7 +626,7 @@ decode_stream_bf16_d128(const __nv_bfloat16* __restrict__ q, const __grid_consta
 template <typename TO>
 __global__ void __launch_bounds__(1024)
 decode_merge_bf16_d128(const float* __restrict__ partial, const __nv_bfloat16* __restrict__ W, int LH, int g,
-                       Plan pl, int apply_w, TO* __restrict__ out) {
+                       Plan pl, int apply_w, int cw, TO* __restrict__ out) {
     __shared__ uint32_t Ws[128 * 65];          // W rows as bf16 pairs, row stride 65 words (conflict-free)
     __shared__ __align__(8) float aks[8][128];
     __shared__ float fv[8][48], fk[8][48];     // per head, per record: factor for the value part / the key part
@@ -643,8 +643,8 @@ decode_merge_bf16_d128(const float* __restrict__ partial, const __nv_bfloat16* _
     // everything above reads only W, which the streaming kernel does not write; its records from here on
     asm volatile("griddepcontrol.wait;\n" ::: "memory");
     const int first = block_of_tile((long long)u * pl.n_tiles, pl);
-    const int n_rec = (block_of_tile((long long)(u + 1) * pl.n_tiles - 1, pl) - first + 1) * CONSUMER_WARPS;   // <= 36
-    const float* base = partial + (size_t)u * pl.s_max * CONSUMER_WARPS * g * REC;
+    const int n_rec = (block_of_tile((long long)(u + 1) * pl.n_tiles - 1, pl) - first + 1) * cw;   // <= 36; cw records per block
+    const float* base = partial + (size_t)u * pl.s_max * cw * g * REC;
     // The first twelve records' sums are requested before the headers are looked at, so that the
     // two loads share one memory latency (a unit has at most a dozen records unless it is very long).
     float rv[12], rk[12];
