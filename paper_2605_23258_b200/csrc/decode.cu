@@ -223,14 +223,11 @@ static vector_status launch_decode_bf16_d128(const Dims& dm, const void* q, cons
     using T = __nv_bfloat16;
     static PerDeviceOnce once;
     if (once.first()) {
-        cudaError_t e = cudaFuncSetAttribute(dbf::decode_stream_bf16_d128<false, false>,
+        cudaError_t e = cudaFuncSetAttribute(dbf::decode_stream_bf16_d128<false>,
                                              cudaFuncAttributeMaxDynamicSharedMemorySize, dbf::SMEM_BYTES);
         if (e == cudaSuccess)
-            e = cudaFuncSetAttribute(dbf::decode_stream_bf16_d128<false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+            e = cudaFuncSetAttribute(dbf::decode_stream_bf16_d128<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                      dbf::SMEM_BYTES);
-        if (e == cudaSuccess)
-            e = cudaFuncSetAttribute(dbf::decode_stream_bf16_d128<true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                     dbf::SMEM_BYTES_PER_TILE);
         if (e == cudaSuccess)
             e = cudaFuncSetAttribute(dpt::decode_stream_pertile_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, dpt::SMEM_BYTES);
         if (e != cudaSuccess) { once.undo(); VEC_CUDA_CHECK(e); }
@@ -251,7 +248,6 @@ static vector_status launch_decode_bf16_d128(const Dims& dm, const void* q, cons
     if (ch->n_apx > 0)
         ok = ok && tma::encode_bf16_3d(&maps.apx_k, ch->apx_k, 128, (uint64_t)ch->n_apx, (uint64_t)dm.U, row_b,
                                        (uint64_t)ch->cap_apx * row_b, 64, 64);
-    ok = ok && tma::encode_bf16_3d(&maps.w, W, 128, 128, (uint64_t)dm.LH, row_b, 128 * row_b, 64, 128);
     if (!ok) return VECTOR_ERR_CUDA;
     if (ch->n_ret == 0) { maps.ret_k = maps.apx_k; maps.ret_v = maps.apx_k; }   // never dereferenced: no such tiles
     if (ch->n_apx == 0) maps.apx_k = maps.ret_k;
@@ -261,18 +257,19 @@ static vector_status launch_decode_bf16_d128(const Dims& dm, const void* q, cons
     if (mode == 1) {
         // reconstruction tile by tile on the tensor cores: its own streaming kernel, two consumer warps
         dpt::Maps pm;
-        pm.ret_k = maps.ret_k; pm.ret_v = maps.ret_v; pm.w = maps.w; pm.apx_k = maps.apx_k;
+        pm.ret_k = maps.ret_k; pm.ret_v = maps.ret_v; pm.apx_k = maps.apx_k;
+        if (!tma::encode_bf16_3d(&pm.w, W, 128, 128, (uint64_t)dm.LH, row_b, 128 * row_b, 64, 128)) return VECTOR_ERR_CUDA;
         if (ch->n_apx > 0 && !tma::encode_bf16_3d(&pm.apx_k, ch->apx_k, 128, (uint64_t)ch->n_apx, (uint64_t)dm.U, row_b,
                                                   (uint64_t)ch->cap_apx * row_b, 64, 128))
             return VECTOR_ERR_CUDA;
         dpt::decode_stream_pertile_tc<<<pl.B, dpt::THREADS, dpt::SMEM_BYTES, st>>>(
             (const T*)q, pm, pl, (int)ch->n_ret, (int)ch->n_apx, dm.g, dm.LH, c2, partial, fault);
     } else if (dm.rope)
-        dbf::decode_stream_bf16_d128<false, true><<<pl.B, dbf::ROPE_THREADS, dbf::SMEM_BYTES, st>>>(
+        dbf::decode_stream_bf16_d128<true><<<pl.B, dbf::ROPE_THREADS, dbf::SMEM_BYTES, st>>>(
             (const T*)q, maps, pl, (int)ch->n_ret, (int)ch->n_apx, dm.g, dm.LH, c2, partial, fault, ch->apx_pos,
             (long long)ch->cap_apx, ph);
     else
-        dbf::decode_stream_bf16_d128<false, false><<<pl.B, dbf::THREADS, dbf::SMEM_BYTES, st>>>(
+        dbf::decode_stream_bf16_d128<false><<<pl.B, dbf::THREADS, dbf::SMEM_BYTES, st>>>(
             (const T*)q, maps, pl, (int)ch->n_ret, (int)ch->n_apx, dm.g, dm.LH, c2, partial, fault, nullptr, 0, ph);
     VEC_LAUNCH_CHECK();
     // programmatic dependent launch: the merge blocks start while the streaming kernel drains

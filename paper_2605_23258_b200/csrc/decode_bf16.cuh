@@ -19,10 +19,6 @@
 //   O += P V  (retained tile)  or  A += P K  (key-only tile: the p-weighted key
 //             sum that the merge step multiplies by W); P enters as bf16 hi in
 //             MMA rows 0-7 and bf16 lo in rows 8-15, one MMA for both parts
-// Per-tile reconstruction (PER_TILE, the alternative form o = sum_R p v + sum_A p (W k)): for a
-// key-only step the warp first forms V^T = W K^T for its 64 keys on the tensor cores (W of the unit in
-// shared memory, 512 MMAs), then accumulates O^T += V^T P^T with V^T and P split into bf16 hi + lo; the
-// merge step then adds that part without applying W.
 // RoPE decoupling (ROPE): the value of a key-only token is W applied to the key turned back by its
 // original position.  The logits use the stored keys; before the P K product the warp rotates its 64
 // keys in shared memory, channel c with c + 64 by the angle -pos * theta^(-2c/128).  The angle is
@@ -59,8 +55,6 @@ constexpr int ROPE_TEAM_THREADS = 32 * (1 + ROPE_HELPERS);
 static_assert(CONSUMER_WARPS + 1 == 4 && ROPE_HELPERS == 4, "register hand-over is per warpgroup: owners + producer, then helpers");
 constexpr int REC = 4 + 2 * 128;             // m, l, value-scale, pad, acc_v[128], acc_k[128]
 constexpr int SMEM_BYTES = SLOTS * SLOT_BYTES + 1024;   // + alignment slack; barriers live in static smem
-constexpr int W_BYTES = 32768;               // the unit's map as two swizzled 128 x 128 B boxes (per-tile form only)
-constexpr int SMEM_BYTES_PER_TILE = SMEM_BYTES + W_BYTES;
 
 // How the tile sequence is dealt to blocks; the same arithmetic runs on host and device.
 struct Plan {
@@ -203,12 +197,11 @@ static_assert(SLOTS % CONSUMER_WARPS == 0, "a slot must always be consumed by th
 
 struct Maps {
     CUtensorMap ret_k, ret_v, apx_k;     // rank 3: (128 dims, pool rows, U units), box 64 x 64 x 1, 128B swizzle
-    CUtensorMap w;                       // rank 3: (128 in, 128 out, L*Hkv maps), box 64 x 128 x 1 (per-tile form only)
 };
 
 // grid (plan.B), THREADS threads, SMEM_BYTES dynamic shared memory.
 // partial: [U][s_max][CONSUMER_WARPS][g][REC]; slot of (unit u, block b) = b - block_of_tile(first tile of u).
-template <bool PER_TILE, bool ROPE>
+template <bool ROPE>
 __global__ void __launch_bounds__(ROPE ? ROPE_THREADS : THREADS, 1)
 decode_stream_bf16_d128(const __nv_bfloat16* __restrict__ q, const __grid_constant__ Maps maps, Plan pl, int n_ret,
                         int n_apx, int g, int LH, float scale_log2e, float* __restrict__ partial,
@@ -220,7 +213,6 @@ decode_stream_bf16_d128(const __nv_bfloat16* __restrict__ q, const __grid_consta
     __shared__ volatile int team_ok[CONSUMER_WARPS];     // RoPE: the owner's go / no-go for the tile at hand
     __shared__ __align__(8) uint64_t full_bar[SLOTS];
     __shared__ __align__(8) uint64_t empty_bar[SLOTS];
-    __shared__ __align__(8) uint64_t w_bar;
     // 128B-swizzled TMA boxes want 1024-byte aligned destinations
     unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     const int b = blockIdx.x;
@@ -238,7 +230,6 @@ decode_stream_bf16_d128(const __nv_bfloat16* __restrict__ q, const __grid_consta
     if (tid == 0) {
 #pragma unroll
         for (int s = 0; s < SLOTS; ++s) { tma::mbar_init(&full_bar[s], 1); tma::mbar_init(&empty_bar[s], 1); }
-        tma::mbar_init(&w_bar, 1);
         tma::mbar_fence_init();
     }
     __syncthreads();
@@ -317,9 +308,8 @@ decode_stream_bf16_d128(const __nv_bfloat16* __restrict__ q, const __grid_consta
     const uint32_t pv_row = (uint32_t)(r8 + (mat & 1) * 8) * 128u;       // PV: matrices = (chunk lo|hi) x (keys 0-7|8-15)
     const uint32_t pv_x = (uint32_t)(((mat >> 1) ^ r8) << 4);
 
-    const uint32_t wbase = tma::smem_u32(smem + SLOTS * SLOT_BYTES);     // the unit's W (per-tile form only)
     uint32_t qa[8][2];
-    float acc[16][4];                  // [dim tile][c0,c1: P_hi rows | c2,c3: P_lo rows]; per-tile form: acc[0..7] = O^T
+    float acc[16][4];                  // [dim tile][c0,c1: P_hi rows | c2,c3: P_lo rows]
     float m = -INFINITY, l = 0.f, stash_scale = 1.f;
     bool stashed = false;
 
@@ -353,21 +343,11 @@ decode_stream_bf16_d128(const __nv_bfloat16* __restrict__ q, const __grid_consta
         if (gid < g) {
             float* rec = record_of(unit);
             if (tig == 0) *reinterpret_cast<float4*>(rec) = make_float4(m * 0.69314718055994531f, lt, stashed ? stash_scale : 1.f, 0.f);
-            if (stashed) { if (!PER_TILE) store_acc(rec + 4 + 128); }  // value part was written at the pool switch
+            if (stashed) store_acc(rec + 4 + 128);      // value part was written at the pool switch
             else {
                 store_acc(rec + 4);
 #pragma unroll
                 for (int n = 0; n < 16; ++n) *reinterpret_cast<float2*>(rec + 4 + 128 + n * 8 + 2 * tig) = make_float2(0.f, 0.f);
-            }
-        }
-        if (PER_TILE && stashed) {
-            // acc[mt] holds O^T: dims mt*16 + gid (+8) x heads 2 tig, 2 tig + 1; it goes where the key sum would
-            float* rec0 = record_of(unit) - (size_t)gid * REC + 4 + 128;       // head 0 of this warp's record group
-#pragma unroll
-            for (int mt = 0; mt < 8; ++mt) {
-                const int dim = mt * 16 + gid;
-                if (2 * tig < g) { rec0[(size_t)(2 * tig) * REC + dim] = acc[mt][0]; rec0[(size_t)(2 * tig) * REC + dim + 8] = acc[mt][2]; }
-                if (2 * tig + 1 < g) { rec0[(size_t)(2 * tig + 1) * REC + dim] = acc[mt][1]; rec0[(size_t)(2 * tig + 1) * REC + dim + 8] = acc[mt][3]; }
             }
         }
         zero_acc();
@@ -422,12 +402,7 @@ decode_stream_bf16_d128(const __nv_bfloat16* __restrict__ q, const __grid_consta
         m = m_new;
         stash_scale *= alpha;
         if (__any_sync(0xffffffffu, alpha != 1.f)) {
-            if (PER_TILE && stashed) {
-                // O^T: this thread's columns are heads 2 tig and 2 tig + 1, whose factors live in the quads of those rows
-                const float al0 = __shfl_sync(0xffffffffu, alpha, 8 * tig), al1 = __shfl_sync(0xffffffffu, alpha, 8 * tig + 4);
-#pragma unroll
-                for (int n = 0; n < 8; ++n) { acc[n][0] *= al0; acc[n][1] *= al1; acc[n][2] *= al0; acc[n][3] *= al1; }
-            } else {
+            {
 #pragma unroll
                 for (int n = 0; n < 16; ++n) { acc[n][0] *= alpha; acc[n][1] *= alpha; acc[n][2] *= alpha; acc[n][3] *= alpha; }
             }
@@ -436,80 +411,6 @@ decode_stream_bf16_d128(const __nv_bfloat16* __restrict__ q, const __grid_consta
     };
     // The second part adds p x (the 64 rows at vbase: values, or the keys themselves for a key-only tile).
     auto accumulate64 = [&](uint32_t vbase, bool retained, float (&sc)[8][2]) {
-        if (PER_TILE && !retained) {
-            // ---- P^T as B operands (k = keys, n = heads), bf16 hi and lo, per 16-key k-step
-            uint32_t pb_hi[4][2], pb_lo[4][2];
-#pragma unroll
-            for (int kk = 0; kk < 4; ++kk) {
-#pragma unroll
-                for (int h = 0; h < 2; ++h) {
-                    const float p0 = sc[2 * kk + h][0], p1 = sc[2 * kk + h][1];
-                    const float h0 = __bfloat162float(__float2bfloat16_rn(p0)), h1 = __bfloat162float(__float2bfloat16_rn(p1));
-                    pb_hi[kk][h] = pack_bf16(h0, h1);
-                    pb_lo[kk][h] = pack_bf16(p0 - h0, p1 - h1);
-                }
-            }
-            const uint32_t w_row = (uint32_t)((lane & 7) + ((lane >> 3) & 1) * 8);      // A operand rows inside a 16-row tile
-            const uint32_t w_hi = (uint32_t)(lane >> 4);                              // second 16-byte chunk of the k-step
-#pragma unroll 1
-            for (int mg = 0; mg < 4; ++mg) {           // 32 output dims at a time
-                float vt[2][8][4];                     // V^T[dim][key] for two 16-dim row tiles x eight 8-key column tiles
-#pragma unroll
-                for (int i = 0; i < 2; ++i)
-#pragma unroll
-                    for (int n = 0; n < 8; ++n) { vt[i][n][0] = vt[i][n][1] = vt[i][n][2] = vt[i][n][3] = 0.f; }
-#pragma unroll
-                for (int ks = 0; ks < 8; ++ks) {
-                    uint32_t wa[2][4];
-#pragma unroll
-                    for (int i = 0; i < 2; ++i) {
-                        const uint32_t row = (uint32_t)((2 * mg + i) * 16) + w_row, chunk = 2 * ks + w_hi;
-                        ldsm_x4(wbase + (chunk >> 3) * 16384 + row * 128 + (((chunk & 7) ^ (row & 7)) << 4), wa[i][0], wa[i][1],
-                                wa[i][2], wa[i][3]);
-                    }
-#pragma unroll
-                    for (int j = 0; j < 4; ++j) {
-                        uint32_t b0, b1, b2, b3;
-                        ldsm_x4(vbase + (ks >> 2) * BOX_BYTES + j * 16 * 128 + qk_row + ((((2 * ks) & 7) << 4) ^ qk_x), b0, b1, b2, b3);
-#pragma unroll
-                        for (int i = 0; i < 2; ++i) {
-                            mma_16(vt[i][2 * j], wa[i][0], wa[i][1], wa[i][2], wa[i][3], b0, b1);
-                            mma_16(vt[i][2 * j + 1], wa[i][0], wa[i][1], wa[i][2], wa[i][3], b2, b3);
-                        }
-                    }
-                }
-                // ---- O^T[dims][heads] += V^T P^T, V^T as A operand (accumulator layout = A layout), hi + lo
-                float ot[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
-#pragma unroll
-                for (int i = 0; i < 2; ++i) {
-#pragma unroll
-                    for (int kk = 0; kk < 4; ++kk) {
-                        uint32_t ah[4], al[4];
-#pragma unroll
-                        for (int r = 0; r < 4; ++r) {       // a0, a1: key tile 2kk rows gid, gid+8; a2, a3: key tile 2kk+1
-                            const float x0 = vt[i][2 * kk + (r >> 1)][(r & 1) * 2], x1 = vt[i][2 * kk + (r >> 1)][(r & 1) * 2 + 1];
-                            const float h0 = __bfloat162float(__float2bfloat16_rn(x0)), h1 = __bfloat162float(__float2bfloat16_rn(x1));
-                            ah[r] = pack_bf16(h0, h1);
-                            al[r] = pack_bf16(x0 - h0, x1 - h1);
-                        }
-                        mma_16(ot[i], ah[0], ah[1], ah[2], ah[3], pb_hi[kk][0], pb_hi[kk][1]);
-                        mma_16(ot[i], al[0], al[1], al[2], al[3], pb_hi[kk][0], pb_hi[kk][1]);
-                        mma_16(ot[i], ah[0], ah[1], ah[2], ah[3], pb_lo[kk][0], pb_lo[kk][1]);
-                    }
-                }
-                // add into the running O^T; the loop over mg stays rolled, so the register index is made static
-#pragma unroll
-                for (int ms = 0; ms < 4; ++ms) {
-                    if (ms == mg) {
-#pragma unroll
-                        for (int i = 0; i < 2; ++i)
-#pragma unroll
-                            for (int r = 0; r < 4; ++r) acc[2 * ms + i][r] += ot[i][r];
-                    }
-                }
-            }
-            return;
-        }
         // ---- accumulate P x (V rows | K rows): four k-steps of 16 keys x 16 column tiles of 8 dims
 #pragma unroll
         for (int kk = 0; kk < 4; ++kk) {
@@ -573,18 +474,7 @@ decode_stream_bf16_d128(const __nv_bfloat16* __restrict__ q, const __grid_consta
     // Walk the units the block touches; this warp owns the block's tiles i with i % CONSUMER_WARPS == wq.
     int i = wq;                                        // index into the block's tile sequence
     bool ok = true;                                    // false once a wait gave up: keep walking, touch nothing
-    uint32_t units_done = 0;
-    for (int u = u0; u <= u_last; ++u, ++units_done) {
-        if (PER_TILE) {
-            // all three warps have left the previous unit: its W may be replaced
-            asm volatile("bar.sync 1, %0;\n" ::"n"(32 * CONSUMER_WARPS) : "memory");
-            if (wq == 0 && lane == 0) {
-                tma::mbar_expect_tx(&w_bar, W_BYTES);
-                tma::load_3d(smem + SLOTS * SLOT_BYTES, &maps.w, 0, 0, u % LH, &w_bar);
-                tma::load_3d(smem + SLOTS * SLOT_BYTES + W_BYTES / 2, &maps.w, 64, 0, u % LH, &w_bar);
-            }
-            if (ok) ok = tma::mbar_wait_warp(&w_bar, units_done & 1, fault, 4);
-        }
+    for (int u = u0; u <= u_last; ++u) {
         const long long unit_end = (long long)(u + 1) * pl.n_tiles - gt_lo;     // first sequence index past the unit
         bool loaded = false;
         for (; i < n_my && i < unit_end; i += CONSUMER_WARPS) {

@@ -4,23 +4,24 @@
 // of the generation-time attention (paper Section 3.2, Step 3: the value of an approximated token
 // is rebuilt as W k).  For every tile of 128 key-only keys the reconstructed values are
 // materialised as  V^T = W K_tile^T  (128 dims x 128 keys x 128) by tcgen05.mma with the accumulator
-// in tensor memory -- W and K are bf16 data, so the products are exact -- and weighted by the softmax
-// probabilities in fp32.
+// in tensor memory -- W and K are bf16 data, so the products are exact -- brought back to shared
+// memory as a bf16 pair hi + lo (sixteen mantissa bits) over the keys they came from, and then
+// weighted exactly like stored values.
 //
 // The mixed cache is streamed once, as in the factored kernel: 32 KB tiles (64 retained keys + their
 // 64 values, or 128 key-only keys) dealt in equal contiguous ranges to one persistent block per
 // multiprocessor.  Roles inside a block (256 threads):
 //   warps 0-1  consumers: tile i belongs to warp i % 2.  Scores S = Q K^T with warp-level MMAs (the g
-//              query heads padded to the MMA rows), online softmax per warp.  A retained tile also adds
-//              P V in the warp; for a key-only tile the warp only publishes its probabilities P (fp32)
-//              and the factor alpha by which its running maximum moved
+//              query heads padded to the MMA rows), online softmax, O += P V with P as bf16 hi + lo.
+//              For a key-only tile V is the reconstructed tile: the warp says when it has read the
+//              keys for the last time, waits for the conversion, and adds P V_hi + P_hi V_lo
 //   warp  2    producer: TMA loads of the tiles into four 32 KB slots
 //   warp  3    MMA issuer, owner of tensor memory; TMA-loads the unit's W when the range enters a unit
-//   warps 4-7  reconstruction: thread = output dim (its TMEM lane).  Per key-only tile: reads its row
-//              of V^T from tensor memory, O^T[dim][head] = alpha O^T + sum_key V^T[dim][key] P[key][head]
-//              in fp32 registers, one accumulator set per consumer warp (its softmax reference)
-// Per unit every consumer warp leaves a partial record (m, l, sum p v) and the reconstruction warps
-// add that warp's sum p (W k) to it; the merge kernel combines the records without applying W.
+//   warps 4-7  conversion: thread = output dim (its TMEM lane).  Per key-only tile: reads its row of
+//              V^T from tensor memory, splits it into bf16 hi and lo, and writes hi over the tile's keys
+//              (the slot is a [128 dims][128 keys] tile from then on) and lo into the consumer's side buffer
+// Per unit every consumer warp leaves one partial record (m, l, sum p v + sum p (W k)); the merge
+// kernel combines the records without applying W.
 // All hand-offs are mbarriers; every wait is bounded and records a fault code.
 #ifndef VECTOR_DECODE_PERTILE_TC_CUH_
 #define VECTOR_DECODE_PERTILE_TC_CUH_
@@ -43,8 +44,8 @@ constexpr int SLOTS = 4;                     // a multiple of CONSUMERS: a slot 
 constexpr int SLOT_BYTES = 32768;
 constexpr int HALF_BYTES = 16384;
 constexpr int W_BYTES = 32768;
-constexpr int P_BYTES = 128 * 8 * 4;         // probabilities of one key-only tile: [128 keys][8 heads] fp32
-constexpr int SMEM_BYTES = SLOTS * SLOT_BYTES + W_BYTES + CONSUMERS * 2 * P_BYTES + 1024;
+constexpr int LO_BYTES = 32768;              // low halves of one reconstructed tile: [128 dims][128 keys] bf16
+constexpr int SMEM_BYTES = SLOTS * SLOT_BYTES + W_BYTES + CONSUMERS * LO_BYTES + 1024;
 constexpr int NB = 3;                        // V^T accumulators in tensor memory (128 columns each)
 constexpr int TMEM_COLS = 512;
 constexpr int THREADS = 256;
@@ -60,10 +61,11 @@ struct Maps {
 struct Sync {
     uint64_t full[SLOTS], empty[SLOTS];
     uint64_t vhat_full[NB], vhat_empty[NB];
-    uint64_t p_full[CONSUMERS][2], p_empty[CONSUMERS][2];
+    uint64_t keys_read[SLOTS];           // the consumer has formed its scores: the slot's keys may be overwritten
+    uint64_t vt_ready[SLOTS];            // the slot holds V^T hi, the consumer's side buffer V^T lo
+    uint64_t lo_free[CONSUMERS];         // the consumer has finished with its side buffer
     uint64_t w_full, w_empty;
     uint32_t tmem_base;
-    float alpha[CONSUMERS][2][8];
 };
 
 // grid (plan.B), THREADS threads, SMEM_BYTES dynamic shared memory.
@@ -75,7 +77,7 @@ decode_stream_pertile_tc(const __nv_bfloat16* __restrict__ q, const __grid_const
     __shared__ Sync sy;
     unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     unsigned char* Ws = smem + SLOTS * SLOT_BYTES;
-    float* Pbuf = reinterpret_cast<float*>(smem + SLOTS * SLOT_BYTES + W_BYTES);      // [consumer][2][128][8]
+    unsigned char* Lo = smem + SLOTS * SLOT_BYTES + W_BYTES;                            // [consumer][128 dims][128 keys] bf16
     const int b = blockIdx.x;
     const int tid = threadIdx.x, lane = tid & 31, wq = tid >> 5;
     const long long gt_lo = dbf::tile_begin(b, pl), gt_hi = dbf::tile_begin(b + 1, pl);
@@ -91,9 +93,9 @@ decode_stream_pertile_tc(const __nv_bfloat16* __restrict__ q, const __grid_const
 #pragma unroll
         for (int k = 0; k < NB; ++k) { tma::mbar_init(&sy.vhat_full[k], 1); tma::mbar_init(&sy.vhat_empty[k], RECON_WARPS); }
 #pragma unroll
-        for (int w = 0; w < CONSUMERS; ++w)
+        for (int s = 0; s < SLOTS; ++s) { tma::mbar_init(&sy.keys_read[s], 1); tma::mbar_init(&sy.vt_ready[s], RECON_WARPS); }
 #pragma unroll
-            for (int k = 0; k < 2; ++k) { tma::mbar_init(&sy.p_full[w][k], 1); tma::mbar_init(&sy.p_empty[w][k], RECON_WARPS); }
+        for (int w = 0; w < CONSUMERS; ++w) tma::mbar_init(&sy.lo_free[w], 1);
         tma::mbar_init(&sy.w_full, 1);
         tma::mbar_init(&sy.w_empty, 1);
         tma::mbar_fence_init();
@@ -106,9 +108,8 @@ decode_stream_pertile_tc(const __nv_bfloat16* __restrict__ q, const __grid_const
     __syncthreads();
     tc::fence_after_sync();
 
-    // Slot release: a retained tile is released by its consumer warp, a key-only tile by the
-    // reconstruction warps' lane-0 thread of warp 4 once the MMA that read it has completed and the
-    // consumer has published its probabilities (so has finished reading the keys): one arrival either way.
+    // A slot is released by the consumer warp that owns it, for a key-only tile after it has weighted
+    // the reconstructed values that took the keys' place.
     if (wq == 2) {
         // ------------------------------------------------------------------ producer
         if (lane == 0 && n_my > 0) {
@@ -176,56 +177,40 @@ decode_stream_pertile_tc(const __nv_bfloat16* __restrict__ q, const __grid_const
             }
         }
     } else if (wq >= 4) {
-        // ------------------------------------------------------------------ reconstruction warps
-        const int quarter = wq & 3, c = quarter * 32 + lane;          // this thread's output dim = its TMEM lane
+        // ------------------------------------------------------------------ conversion warps
+        const int quarter = wq & 3, c = quarter * 32 + lane;          // this thread's output dim = its TMEM lane = its row of V^T
         const uint32_t lane_addr = sy.tmem_base + ((uint32_t)(quarter * 32) << 16);
-        float acc[CONSUMERS][8];
-        bool used[CONSUMERS];
-#pragma unroll
-        for (int w = 0; w < CONSUMERS; ++w) {
-            used[w] = false;
-#pragma unroll
-            for (int a = 0; a < 8; ++a) acc[w][a] = 0.f;
-        }
-        uint32_t j = 0, pcount[CONSUMERS] = {0u, 0u};
+        const uint32_t row_off = (uint32_t)c * 128u;                   // rows of 128 bytes, 16-byte chunk index XOR (row & 7)
+        uint32_t j = 0, kcount[SLOTS] = {0u, 0u, 0u, 0u}, lcount[CONSUMERS] = {0u, 0u};
         bool ok = n_my > 0;
-        int u = u0, t = n_my > 0 ? (int)(gt_lo - (long long)u0 * pl.n_tiles) : 0;
+        int t = n_my > 0 ? (int)(gt_lo - (long long)u0 * pl.n_tiles) : 0;
         for (int i = 0; i < n_my && ok; ++i) {
             if (t >= pl.n_rt) {
                 const int w = i % CONSUMERS, s = i % SLOTS;
-                const uint32_t vb = j % NB, use = j / NB, pb = pcount[w] & 1, puse = pcount[w] >> 1;
-                if (!tma::mbar_wait_warp(&sy.p_full[w][pb], puse & 1, fault, 71)) { ok = false; break; }
+                const uint32_t vb = j % NB, use = j / NB;
+                // the MMA has read the keys and left V^T; the consumer has formed its scores; its side buffer is free
                 if (!tma::mbar_wait_warp(&sy.vhat_full[vb], use & 1, fault, 72)) { ok = false; break; }
+                if (!tma::mbar_wait_warp(&sy.keys_read[s], kcount[s] & 1, fault, 71)) { ok = false; break; }
+                if (lcount[w] > 0 && !tma::mbar_wait_warp(&sy.lo_free[w], (lcount[w] - 1) & 1, fault, 73)) { ok = false; break; }
                 tc::fence_after_sync();
-                const float* P = Pbuf + (size_t)(w * 2 + pb) * (128 * 8);
-                float al[8];
-#pragma unroll
-                for (int a = 0; a < 8; ++a) al[a] = sy.alpha[w][pb][a];
-                float o[8];
-#pragma unroll
-                for (int a = 0; a < 8; ++a) o[a] = 0.f;
-                // 16 keys at a time in a loop that stays rolled: the four roles of this block run four different
-                // instruction streams, and an unrolled 128-key body alone would not fit the instruction cache
+                const uint32_t hi_base = tma::smem_u32(smem + s * SLOT_BYTES) + row_off;
+                const uint32_t lo_base = tma::smem_u32(Lo + w * LO_BYTES) + row_off;
                 const uint32_t taddr = lane_addr + vb * 128;
-                auto weigh16 = [&](const uint32_t (&v16)[16], int key0) {
-                    // all sixteen rows of P are requested before the first product: a warp issues in order, and a
-                    // load placed behind the products of the key before it would show its full latency every time
-                    float4 pr[16];
+                // 16 keys = two 16-byte chunks of this row at a time, in a loop that stays rolled
+                auto split16 = [&](const uint32_t (&v16)[16], int chunk0) {
+                    uint32_t hi[8], lo[8];
 #pragma unroll
-                    for (int k = 0; k < 16; ++k) pr[k] = *reinterpret_cast<const float4*>(P + (key0 + k) * 8);      // the same address in every lane
-#pragma unroll
-                    for (int k = 0; k < 16; ++k) {
-                        const float v = __uint_as_float(v16[k]);
-                        o[0] = fmaf(v, pr[k].x, o[0]); o[1] = fmaf(v, pr[k].y, o[1]); o[2] = fmaf(v, pr[k].z, o[2]); o[3] = fmaf(v, pr[k].w, o[3]);
+                    for (int e = 0; e < 8; ++e) {
+                        const float x0 = __uint_as_float(v16[2 * e]), x1 = __uint_as_float(v16[2 * e + 1]);
+                        hi[e] = dbf::pack_bf16(x0, x1);
+                        lo[e] = dbf::pack_bf16(x0 - __uint_as_float(hi[e] << 16), x1 - __uint_as_float(hi[e] & 0xffff0000u));
                     }
-                    if (g > 4) {
 #pragma unroll
-                        for (int k = 0; k < 16; ++k) pr[k] = *reinterpret_cast<const float4*>(P + (key0 + k) * 8 + 4);
-#pragma unroll
-                        for (int k = 0; k < 16; ++k) {
-                            const float v = __uint_as_float(v16[k]);
-                            o[4] = fmaf(v, pr[k].x, o[4]); o[5] = fmaf(v, pr[k].y, o[5]); o[6] = fmaf(v, pr[k].z, o[6]); o[7] = fmaf(v, pr[k].w, o[7]);
-                        }
+                    for (int h = 0; h < 2; ++h) {
+                        const int chunk = chunk0 + h;                  // keys 8 chunk .. 8 chunk + 7: box chunk / 8, chunk % 8 inside the row
+                        const uint32_t off = (uint32_t)(chunk >> 3) * HALF_BYTES + (uint32_t)(((chunk & 7) ^ (c & 7)) << 4);
+                        asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};\n" ::"r"(hi_base + off), "r"(hi[4 * h]), "r"(hi[4 * h + 1]), "r"(hi[4 * h + 2]), "r"(hi[4 * h + 3]) : "memory");
+                        asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};\n" ::"r"(lo_base + off), "r"(lo[4 * h]), "r"(lo[4 * h + 1]), "r"(lo[4 * h + 2]), "r"(lo[4 * h + 3]) : "memory");
                     }
                 };
                 uint32_t ra[16], rb[16];
@@ -234,49 +219,24 @@ decode_stream_pertile_tc(const __nv_bfloat16* __restrict__ q, const __grid_const
                 for (int c2 = 0; c2 < 8; c2 += 2) {
                     tc::tmem_ld_wait16(ra);
                     tc::tmem_ld16(taddr + (c2 + 1) * 16, rb);
-                    weigh16(ra, c2 * 16);
+                    split16(ra, 2 * c2);
                     tc::tmem_ld_wait16(rb);
                     if (c2 + 2 < 8) tc::tmem_ld16(taddr + (c2 + 2) * 16, ra);
-                    weigh16(rb, (c2 + 1) * 16);
+                    split16(rb, 2 * c2 + 2);
                 }
-                // the accumulator, the probabilities and the slot are free again
+                // the slot is refilled by a bulk copy once released: order these stores ahead of it
+                asm volatile("fence.proxy.async.shared::cta;\n" ::: "memory");
                 tc::fence_before_sync();
                 __syncwarp();
                 if (lane == 0) {
                     tma::mbar_arrive(&sy.vhat_empty[vb]);
-                    tma::mbar_arrive(&sy.p_empty[w][pb]);
-                    if (wq == 4) tma::mbar_arrive(&sy.empty[s]);
-                }
-#pragma unroll
-                for (int ww = 0; ww < CONSUMERS; ++ww) {
-                    if (ww == w) {
-#pragma unroll
-                        for (int a = 0; a < 8; ++a) acc[ww][a] = fmaf(acc[ww][a], al[a], o[a]);
-                        used[ww] = true;
-                    }
+                    tma::mbar_arrive(&sy.vt_ready[s]);
                 }
                 ++j;
-                ++pcount[w];
+                ++kcount[s];
+                ++lcount[w];
             }
-            const bool unit_ends = t + 1 == pl.n_tiles || i + 1 == n_my;
-            if (unit_ends) {
-                // this block's share of the unit is complete: sum p (W k) of each consumer warp into its record
-                int slot = b - dbf::block_of_tile((long long)u * pl.n_tiles, pl);
-                if (slot < 0 || slot >= pl.s_max) { atomicCAS(fault, 0, 75); slot = 0; }
-#pragma unroll
-                for (int w = 0; w < CONSUMERS; ++w) {
-                    if (used[w]) {
-                        float* rec = partial + ((((size_t)u * pl.s_max + slot) * CONSUMERS + w) * g) * REC + 4 + 128;
-#pragma unroll
-                        for (int a = 0; a < 8; ++a)
-                            if (a < g) rec[(size_t)a * REC + c] = acc[w][a];
-                    }
-                    used[w] = false;
-#pragma unroll
-                    for (int a = 0; a < 8; ++a) acc[w][a] = 0.f;
-                }
-            }
-            if (++t == pl.n_tiles) { t = 0; ++u; }
+            if (++t == pl.n_tiles) t = 0;
         }
     } else if (n_my > 0) {
         // ------------------------------------------------------------------ consumers (warps 0 and 1)
@@ -289,9 +249,8 @@ decode_stream_pertile_tc(const __nv_bfloat16* __restrict__ q, const __grid_const
         const uint32_t pv_x = (uint32_t)(((mat >> 1) ^ r8) << 4);
         uint32_t qa[8][2];
         float acc[16][4];                  // sum p v: [dim tile][c0,c1: P_hi rows | c2,c3: P_lo rows]
-        float m = -INFINITY, l = 0.f, stash_scale = 1.f;
-        bool stashed = false;
-        uint32_t pcount = 0;
+        float m = -INFINITY, l = 0.f;
+        uint32_t vcount[SLOTS / CONSUMERS] = {0u, 0u};      // key-only tiles this warp has had in each of its two slots
 
         auto record_of = [&](int unit) -> float* {
             int slot = b - dbf::block_of_tile((long long)unit * pl.n_tiles, pl);
@@ -331,21 +290,62 @@ decode_stream_pertile_tc(const __nv_bfloat16* __restrict__ q, const __grid_const
                 }
             }
         };
+        // P (this thread: head gid, keys 8 n + 2 tig, + 1 of 64) times the 64 rows at vbase (two boxes `box`
+        // bytes apart: rows = keys of stored values, `trans`; or rows = dims of a reconstructed tile, keys
+        // along the row).  P enters as bf16 hi in MMA rows 0-7 and, with `with_lo`, its bf16 remainder in rows 8-15.
+        auto weigh64_values = [&](uint32_t vbase, const float (&sc)[8][2]) {
+#pragma unroll
+            for (int kk = 0; kk < 4; ++kk) {
+                const float p00 = sc[2 * kk][0], p01 = sc[2 * kk][1], p10 = sc[2 * kk + 1][0], p11 = sc[2 * kk + 1][1];
+                const float h00 = __bfloat162float(__float2bfloat16_rn(p00)), h01 = __bfloat162float(__float2bfloat16_rn(p01));
+                const float h10 = __bfloat162float(__float2bfloat16_rn(p10)), h11 = __bfloat162float(__float2bfloat16_rn(p11));
+                const uint32_t a0 = dbf::pack_bf16(h00, h01), a2 = dbf::pack_bf16(h10, h11);
+                const uint32_t a1 = dbf::pack_bf16(p00 - h00, p01 - h01), a3 = dbf::pack_bf16(p10 - h10, p11 - h11);
+#pragma unroll
+                for (int np = 0; np < 8; ++np) {
+                    uint32_t b0, b1, b2, b3;
+                    dbf::ldsm_x4_t(vbase + (np >> 2) * 8192 + kk * 16 * 128 + pv_row + ((((2 * np) & 7) << 4) ^ pv_x), b0, b1, b2, b3);
+                    dbf::mma_16(acc[2 * np], a0, a1, a2, a3, b0, b1);
+                    dbf::mma_16(acc[2 * np + 1], a0, a1, a2, a3, b2, b3);
+                }
+            }
+        };
+        // The same for 64 keys of a reconstructed tile: V^T hi at hibase, V^T lo at lobase, both [128 dims][keys]
+        // in boxes of 128 rows; `kc0` = first 16-byte chunk of these keys inside the row (0 or 8 -> box 0 or 1).
+        auto weigh64_rebuilt = [&](uint32_t hibase, uint32_t lobase, const float (&sc)[8][2]) {
+#pragma unroll
+            for (int kk = 0; kk < 4; ++kk) {
+                const float p00 = sc[2 * kk][0], p01 = sc[2 * kk][1], p10 = sc[2 * kk + 1][0], p11 = sc[2 * kk + 1][1];
+                const float h00 = __bfloat162float(__float2bfloat16_rn(p00)), h01 = __bfloat162float(__float2bfloat16_rn(p01));
+                const float h10 = __bfloat162float(__float2bfloat16_rn(p10)), h11 = __bfloat162float(__float2bfloat16_rn(p11));
+                const uint32_t a0 = dbf::pack_bf16(h00, h01), a2 = dbf::pack_bf16(h10, h11);
+                const uint32_t a1 = dbf::pack_bf16(p00 - h00, p01 - h01), a3 = dbf::pack_bf16(p10 - h10, p11 - h11);
+#pragma unroll
+                for (int jj = 0; jj < 8; ++jj) {        // 16 dims per ldmatrix: rows 16 jj .. of V^T, keys 16 kk .. along the row
+                    uint32_t b0, b1, b2, b3;
+                    const uint32_t off = jj * 16 * 128 + qk_row + ((((2 * kk) & 7) << 4) ^ qk_x);
+                    dbf::ldsm_x4(hibase + off, b0, b1, b2, b3);
+                    dbf::mma_16(acc[2 * jj], a0, a1, a2, a3, b0, b1);
+                    dbf::mma_16(acc[2 * jj + 1], a0, a1, a2, a3, b2, b3);
+                    dbf::ldsm_x4(lobase + off, b0, b1, b2, b3);
+                    dbf::mma_16(acc[2 * jj], a0, 0u, a2, 0u, b0, b1);          // P_hi V_lo: the product of the two remainders is dropped
+                    dbf::mma_16(acc[2 * jj + 1], a0, 0u, a2, 0u, b2, b3);
+                }
+            }
+        };
         auto flush = [&](int unit) {
             float lt = l;
             lt += __shfl_xor_sync(0xffffffffu, lt, 1);
             lt += __shfl_xor_sync(0xffffffffu, lt, 2);
             if (gid < g) {
                 float* rec = record_of(unit);
-                if (tig == 0) *reinterpret_cast<float4*>(rec) = make_float4(m * 0.69314718055994531f, lt, stashed ? stash_scale : 1.f, 0.f);
-                if (!stashed) {         // no key-only tile: sum p v goes out now, and nothing follows it
-                    store_acc(rec + 4);
+                if (tig == 0) *reinterpret_cast<float4*>(rec) = make_float4(m * 0.69314718055994531f, lt, 1.f, 0.f);
+                store_acc(rec + 4);
 #pragma unroll
-                    for (int n = 0; n < 16; ++n) *reinterpret_cast<float2*>(rec + 4 + 128 + n * 8 + 2 * tig) = make_float2(0.f, 0.f);
-                }
+                for (int n = 0; n < 16; ++n) *reinterpret_cast<float2*>(rec + 4 + 128 + n * 8 + 2 * tig) = make_float2(0.f, 0.f);
             }
             zero_acc();
-            m = -INFINITY; l = 0.f; stash_scale = 1.f; stashed = false;
+            m = -INFINITY; l = 0.f;
         };
 
         zero_acc();
@@ -393,37 +393,19 @@ decode_stream_pertile_tc(const __nv_bfloat16* __restrict__ q, const __grid_const
 #pragma unroll
                         for (int n = 0; n < 16; ++n) { acc[n][0] *= alpha; acc[n][1] *= alpha; acc[n][2] *= alpha; acc[n][3] *= alpha; }
                     }
-                    const uint32_t vbase = base + HALF_BYTES;
-#pragma unroll
-                    for (int kk = 0; kk < 4; ++kk) {
-                        // P as bf16 hi (MMA rows 0-7) + lo (rows 8-15)
-                        const float p00 = sc[2 * kk][0], p01 = sc[2 * kk][1], p10 = sc[2 * kk + 1][0], p11 = sc[2 * kk + 1][1];
-                        const float h00 = __bfloat162float(__float2bfloat16_rn(p00)), h01 = __bfloat162float(__float2bfloat16_rn(p01));
-                        const float h10 = __bfloat162float(__float2bfloat16_rn(p10)), h11 = __bfloat162float(__float2bfloat16_rn(p11));
-                        const uint32_t a0 = dbf::pack_bf16(h00, h01), a2 = dbf::pack_bf16(h10, h11);
-                        const uint32_t a1 = dbf::pack_bf16(p00 - h00, p01 - h01), a3 = dbf::pack_bf16(p10 - h10, p11 - h11);
-#pragma unroll
-                        for (int np = 0; np < 8; ++np) {
-                            uint32_t b0, b1, b2, b3;
-                            dbf::ldsm_x4_t(vbase + (np >> 2) * 8192 + kk * 16 * 128 + pv_row + ((((2 * np) & 7) << 4) ^ pv_x), b0, b1, b2, b3);
-                            dbf::mma_16(acc[2 * np], a0, a1, a2, a3, b0, b1);
-                            dbf::mma_16(acc[2 * np + 1], a0, a1, a2, a3, b2, b3);
-                        }
-                    }
+                    weigh64_values(base + HALF_BYTES, sc);
                     __syncwarp();
                     if (lane == 0) tma::mbar_arrive(&sy.empty[s]);
                 } else {
                     // ---- key-only tile: 128 keys, each half of the head dimension in a box of 128 rows
                     const int r0 = (t - pl.n_rt) * 2 * KEYS;
                     const int nrows = min(2 * KEYS, n_apx - r0);
-                    if (!stashed) {            // first key-only keys of this unit for this warp: park sum p v
-                        if (gid < g) store_acc(record_of(u) + 4);
-                        stashed = true;
-                        stash_scale = 1.f;
-                    }
                     float sa[8][2], sb[8][2];
                     qk64(base, (uint32_t)HALF_BYTES, sa);
                     qk64(base + 64 * 128, (uint32_t)HALF_BYTES, sb);
+                    // every lane is past its last read of the keys: the conversion warps may put V^T in their place
+                    __syncwarp();
+                    if (lane == 0) tma::mbar_arrive(&sy.keys_read[s]);
                     float mx = -INFINITY;
 #pragma unroll
                     for (int n = 0; n < 8; ++n) {
@@ -438,28 +420,30 @@ decode_stream_pertile_tc(const __nv_bfloat16* __restrict__ q, const __grid_const
                     mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
                     const float m_new = fmaxf(m, mx);
                     const float alpha = exp2f(m - m_new);
-                    const uint32_t pb = pcount & 1, puse = pcount >> 1;
-                    ok = puse == 0 || tma::mbar_wait_warp(&sy.p_empty[wq][pb], (puse - 1) & 1, fault, 68);
-                    if (ok) {
-                        float* P = Pbuf + (size_t)(wq * 2 + pb) * (128 * 8);
-                        float ls = 0.f;
+                    float ls = 0.f;
 #pragma unroll
-                        for (int n = 0; n < 8; ++n) {
-                            const int kc = n * 8 + 2 * tig;
-                            const float p0 = exp2f(sa[n][0] - m_new), p1 = exp2f(sa[n][1] - m_new);
-                            const float p2 = exp2f(sb[n][0] - m_new), p3 = exp2f(sb[n][1] - m_new);
-                            ls += (p0 + p1) + (p2 + p3);
-                            P[kc * 8 + gid] = p0; P[(kc + 1) * 8 + gid] = p1;
-                            P[(64 + kc) * 8 + gid] = p2; P[(64 + kc + 1) * 8 + gid] = p3;
-                        }
-                        if (tig == 0) sy.alpha[wq][pb][gid] = alpha;
-                        l = l * alpha + ls;
-                        m = m_new;
-                        stash_scale *= alpha;
-                        __syncwarp();
-                        if (lane == 0) tma::mbar_arrive(&sy.p_full[wq][pb]);       // release: the stores above are ordered before it
-                        ++pcount;
+                    for (int n = 0; n < 8; ++n) {
+                        sa[n][0] = exp2f(sa[n][0] - m_new); sa[n][1] = exp2f(sa[n][1] - m_new);
+                        sb[n][0] = exp2f(sb[n][0] - m_new); sb[n][1] = exp2f(sb[n][1] - m_new);
+                        ls += (sa[n][0] + sa[n][1]) + (sb[n][0] + sb[n][1]);
                     }
+                    l = l * alpha + ls;
+                    m = m_new;
+                    if (__any_sync(0xffffffffu, alpha != 1.f)) {
+#pragma unroll
+                        for (int n = 0; n < 16; ++n) { acc[n][0] *= alpha; acc[n][1] *= alpha; acc[n][2] *= alpha; acc[n][3] *= alpha; }
+                    }
+                    // the reconstructed values: hi where the keys were, lo in this warp's side buffer
+                    const int sl = (i / CONSUMERS) % (SLOTS / CONSUMERS);
+                    ok = tma::mbar_wait_warp(&sy.vt_ready[s], vcount[sl] & 1, fault, 68);
+                    ++vcount[sl];
+                    if (ok) {
+                        const uint32_t lob = tma::smem_u32(Lo + wq * LO_BYTES);
+                        weigh64_rebuilt(base, lob, sa);
+                        weigh64_rebuilt(base + HALF_BYTES, lob + HALF_BYTES, sb);
+                    }
+                    __syncwarp();
+                    if (lane == 0) { tma::mbar_arrive(&sy.lo_free[wq]); tma::mbar_arrive(&sy.empty[s]); }
                 }
             }
             flush(u);
