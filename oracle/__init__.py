@@ -246,6 +246,56 @@ def attend(q, ret_k, ret_v, apx_k, W, scale: float, apx_pos=None, rope: bool = F
     return o1, o2
 
 
+# ---- one map per layer (Section 5.1 calibrates the map layer-wise): the same steps on the keys and
+# values concatenated over the layer's KV heads.  Tensors come head-major, [Hkv][N][d].
+def concat_heads(X) -> np.ndarray:
+    """[Hkv][N][d] -> [N][Hkv d]: a token's vector over the whole layer."""
+    X = _f64(X)
+    Hkv, N, d = X.shape
+    return np.ascontiguousarray(X.transpose(1, 0, 2).reshape(N, Hkv * d))
+
+
+def calibrate_layer(K, V, lam: float) -> np.ndarray:
+    """K, V [Hkv][n][d] -> W [Hkv d][Hkv d] minimising sum ||W k - v||^2 + lam ||W||_F^2 over whole-layer vectors."""
+    return calibrate(concat_heads(K), concat_heads(V), lam)
+
+
+def layer_score(scores_per_head) -> np.ndarray:
+    """The routing decision holds for a token of the layer: its score is the sum of its per-head base scores."""
+    return np.asarray(scores_per_head, dtype=np.float64).sum(axis=0)
+
+
+def residual_layer(K, V, W, idx) -> np.ndarray:
+    """eps_i = || v_i - W k_i ||^2 over the whole-layer vectors; K, V [Hkv][N][d], W [Hkv d][Hkv d]."""
+    return residual(concat_heads(K), concat_heads(V), W, idx)
+
+
+def route_layer(layer_score_f32, K, V, W, n_pool: int, n_apx: int):
+    """Steps 1-3 per layer: one tier per token for all heads.  Same dict as route()."""
+    return route(layer_score_f32, concat_heads(K), concat_heads(V), W, n_pool, n_apx)
+
+
+def attend_layer(q, ret_k, ret_v, apx_k, W, scale: float):
+    """q [Hq][d]; ret_k, ret_v [Hkv][n_ret][d]; apx_k [Hkv][n_apx][d]; W [Hkv d][Hkv d]
+    -> (o_per_token [Hq][d], o_factored [Hq][d]) float64."""
+    q, W = _f64(q), _f64(W)
+    Hq, d = q.shape
+    Hkv = int(np.asarray(ret_k).shape[0]) if np.asarray(ret_k).ndim == 3 else int(np.asarray(apx_k).shape[0])
+    def cat(X, n_hint=None):
+        X = _f64(X)
+        if X.ndim != 3:
+            X = X.reshape(Hkv, -1, d)
+        return concat_heads(X) if X.shape[1] > 0 else np.zeros((0, Hkv * d))
+    rk, rv, ak = cat(ret_k), cat(ret_v), cat(apx_k)
+    o1 = np.empty((Hq, d), dtype=np.float64)
+    o2 = np.empty((Hq, d), dtype=np.float64)
+    rc = lib().oracle_attend_layer(_p(q), ctypes.c_int32(Hq), ctypes.c_int32(Hkv), ctypes.c_int32(d),
+                                   _p(rk), _p(rv), ctypes.c_int64(rk.shape[0]), _p(ak), ctypes.c_int64(ak.shape[0]),
+                                   _p(W), ctypes.c_double(scale), _p(o1), _p(o2))
+    _check(rc, "attend_layer")
+    return o1, o2
+
+
 def rope_inverse(k, pos: int, theta: float = 10000.0) -> np.ndarray:
     k = _f64(k)
     out = np.empty_like(k)

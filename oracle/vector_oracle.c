@@ -453,6 +453,76 @@ int oracle_attend(const double* q, int32_t g, int32_t d,
 
 
 /*
+ * The same attention with ONE map per layer (Section 5.1 "Implementation Details" calibrates the
+ * map layer-wise; the Remark of Section 3.1 writes K and V as whole-layer projections): a token's
+ * key and value are the concatenations over the layer's Hkv KV heads, k_i, v_i in R^{Hkv d}, and an
+ * approximated token's value is W k_i with W of shape [Hkv d][Hkv d].  The tier of a token holds
+ * for all heads of the layer.  Query head a belongs to KV head h = a / (Hq / Hkv); its logits use
+ * slice h of the keys, its output slice h of the (stored or reconstructed) values:
+ *   per-token:  o_a = sum_R p_i v_i[h] + sum_A p_i (W k_i)[h]
+ *   factored:   o_a = sum_R p_i v_i[h] + W[h rows] (sum_A p_i k_i)
+ * q: [Hq][d]; ret_k, ret_v: [n_ret][Hkv d]; apx_k: [n_apx][Hkv d]; outputs (either nullable): [Hq][d].
+ */
+int oracle_attend_layer(const double* q, int32_t Hq, int32_t Hkv, int32_t d,
+                        const double* ret_k, const double* ret_v, int64_t n_ret,
+                        const double* apx_k, int64_t n_apx, const double* W, double scale,
+                        double* out_token, double* out_factored) {
+    if (!q || !W || Hq <= 0 || Hkv <= 0 || Hq % Hkv != 0 || d <= 0 || n_ret < 0 || n_apx < 0 || n_ret + n_apx <= 0)
+        return ORACLE_ERR_ARG;
+    const int64_t n = n_ret + n_apx;
+    const int64_t D = (int64_t)Hkv * d;
+    const int g = Hq / Hkv;
+    double* p = (double*)malloc((size_t)n * sizeof(double));
+    double* acc = (double*)malloc((size_t)D * sizeof(double));
+    if (!p || !acc) { free(p); free(acc); return ORACLE_ERR_ARG; }
+    for (int a = 0; a < Hq; ++a) {
+        const int h = a / g;
+        const double* qa = q + (size_t)a * d;
+        double m = -INFINITY;
+        for (int64_t i = 0; i < n; ++i) {
+            const double* k = ((i < n_ret) ? ret_k + i * D : apx_k + (i - n_ret) * D) + (size_t)h * d;
+            double dot = 0.0;
+            for (int c = 0; c < d; ++c) dot += qa[c] * k[c];
+            p[i] = scale * dot;
+            if (p[i] > m) m = p[i];
+        }
+        double z = 0.0;
+        for (int64_t i = 0; i < n; ++i) { p[i] = exp(p[i] - m); z += p[i]; }
+        for (int64_t i = 0; i < n; ++i) p[i] /= z;
+        if (out_token) {
+            double* o = out_token + (size_t)a * d;
+            for (int c = 0; c < d; ++c) o[c] = 0.0;
+            for (int64_t i = 0; i < n_ret; ++i)
+                for (int c = 0; c < d; ++c) o[c] += p[i] * ret_v[i * D + (size_t)h * d + c];
+            for (int64_t i = 0; i < n_apx; ++i) {
+                const double* k = apx_k + i * D;
+                for (int c = 0; c < d; ++c) {
+                    double r = 0.0;                 /* row h d + c of W against the whole concatenated key */
+                    for (int64_t c2 = 0; c2 < D; ++c2) r += W[((size_t)h * d + c) * D + c2] * k[c2];
+                    o[c] += p[n_ret + i] * r;
+                }
+            }
+        }
+        if (out_factored) {
+            double* o = out_factored + (size_t)a * d;
+            for (int c = 0; c < d; ++c) o[c] = 0.0;
+            for (int64_t c2 = 0; c2 < D; ++c2) acc[c2] = 0.0;
+            for (int64_t i = 0; i < n_ret; ++i)
+                for (int c = 0; c < d; ++c) o[c] += p[i] * ret_v[i * D + (size_t)h * d + c];
+            for (int64_t i = 0; i < n_apx; ++i)
+                for (int64_t c2 = 0; c2 < D; ++c2) acc[c2] += p[n_ret + i] * apx_k[i * D + c2];
+            for (int c = 0; c < d; ++c) {
+                double r = 0.0;
+                for (int64_t c2 = 0; c2 < D; ++c2) r += W[((size_t)h * d + c) * D + c2] * acc[c2];
+                o[c] += r;
+            }
+        }
+    }
+    free(p); free(acc);
+    return ORACLE_OK;
+}
+
+/*
  * Diagnostics of one routed unit (Section 4: the distortion measure E, R^2_approx and the
  * threshold of Proposition 1).  importance: [N] non-negative weights w_i (normalised here to sum 1);
  * tier: [N] 0 evicted / 1 approximated / 2 retained; K, V: [N][d]; W: [d][d] (y = W x).

@@ -509,3 +509,93 @@ def test_diagnostics_pins(oracle):
     assert r3["E"] == pytest.approx(0.3) and r3["sum_approximated_w"] == 0.0 and r3["r2_approx"] == 1.0
     r4 = oracle.diagnostics(w, np.array([2, 1, 1, 2], dtype=np.uint8), K, V2, Wm)
     assert r4["w_star"] == 0.0 and r4["threshold"] == pytest.approx(1.0) and r4["w_bar"] == pytest.approx(0.25)
+
+
+# ---- one map per layer (Section 5.1: the map is calibrated layer-wise; Section 3.1 Remark: K and V as
+#      whole-layer projections): keys and values concatenated over the layer's KV heads
+def _layer_case(rng, Hkv=3, d=8, N=40, g=2):
+    K = rng.standard_normal((Hkv, N, d))
+    V = rng.standard_normal((Hkv, N, d))
+    W = rng.standard_normal((Hkv * d, Hkv * d)) / np.sqrt(Hkv * d)
+    q = rng.standard_normal((Hkv * g, d))
+    return K, V, W, q
+
+
+def test_layer_map_block_diagonal_reduces_to_the_per_head_maps(oracle):
+    """With no cross-head blocks the whole-layer residual is the sum of the per-head residuals and the
+    whole-layer attention is the per-head attention over the shared token sets."""
+    rng = np.random.default_rng(11)
+    Hkv, d, N, g = 3, 8, 40, 2
+    K, V, _, q = _layer_case(rng, Hkv, d, N, g)
+    blocks = rng.standard_normal((Hkv, d, d)) / np.sqrt(d)
+    W = np.zeros((Hkv * d, Hkv * d))
+    for h in range(Hkv):
+        W[h * d:(h + 1) * d, h * d:(h + 1) * d] = blocks[h]
+    idx = np.array([0, 3, 4, 17, 39], dtype=np.int32)
+    want = sum(oracle.residual(K[h], V[h], blocks[h], idx) for h in range(Hkv))
+    assert np.allclose(oracle.residual_layer(K, V, W, idx), want, rtol=1e-12)
+    ret, apx = np.arange(0, 15), np.arange(20, 40)
+    o_tok, o_fac = oracle.attend_layer(q, K[:, ret], V[:, ret], K[:, apx], W, 0.3)
+    for h in range(Hkv):
+        per_tok, _ = oracle.attend(q[h * g:(h + 1) * g], K[h, ret], V[h, ret], K[h, apx], blocks[h], 0.3)
+        assert np.allclose(o_tok[h * g:(h + 1) * g], per_tok, rtol=1e-11, atol=1e-13)
+    assert np.allclose(o_tok, o_fac, rtol=1e-11, atol=1e-13)
+
+
+def test_layer_map_against_numpy_with_cross_head_blocks(oracle):
+    """Residual and attention re-derived with einsum / a library softmax; a map whose cross-head blocks were
+    dropped, or that was applied transposed, gives something else."""
+    rng = np.random.default_rng(12)
+    Hkv, d, N, g = 2, 8, 30, 3
+    K, V, W, q = _layer_case(rng, Hkv, d, N, g)
+    Kc = K.transpose(1, 0, 2).reshape(N, Hkv * d)
+    Vc = V.transpose(1, 0, 2).reshape(N, Hkv * d)
+    idx = np.arange(N, dtype=np.int32)
+    want = ((Vc - np.einsum("oc,nc->no", W, Kc)) ** 2).sum(1)
+    got = oracle.residual_layer(K, V, W, idx)
+    assert np.allclose(got, want, rtol=1e-12)
+    assert not np.allclose(got, ((Vc - np.einsum("co,nc->no", W, Kc)) ** 2).sum(1), rtol=1e-3)      # transposed map
+    ret, apx = np.arange(0, 12), np.arange(12, 30)
+    o_tok, o_fac = oracle.attend_layer(q, K[:, ret], V[:, ret], K[:, apx], W, 0.25)
+    Vhat = np.einsum("oc,nc->no", W, Kc[apx]).reshape(len(apx), Hkv, d)       # reconstructed values, whole layer
+    for a in range(Hkv * g):
+        h = a // g
+        keys = np.concatenate([K[h, ret], K[h, apx]])
+        p = softmax(0.25 * keys @ q[a])
+        want_o = p[:len(ret)] @ V[h, ret] + p[len(ret):] @ Vhat[:, h]
+        assert np.allclose(o_tok[a], want_o, rtol=1e-11, atol=1e-13) and np.allclose(o_fac[a], want_o, rtol=1e-11, atol=1e-13)
+    Wd = W.copy(); Wd[:d, d:] = 0.0; Wd[d:, :d] = 0.0
+    assert not np.allclose(oracle.attend_layer(q, K[:, ret], V[:, ret], K[:, apx], Wd, 0.25)[0], o_tok, rtol=1e-3)
+
+
+def test_layer_map_exact_recovery_across_heads(oracle):
+    """V = W_true K with a dense whole-layer map and no noise: calibration finds the map (cross-head blocks
+    included), every residual is zero, routing order is by index, and attention over any retain / approximate
+    split equals plain attention over the pool."""
+    rng = np.random.default_rng(13)
+    Hkv, d, g, n = 2, 8, 2, 600
+    Wt = rng.standard_normal((Hkv * d, Hkv * d)) / np.sqrt(Hkv * d)
+    Kc = rng.standard_normal((n, Hkv * d))
+    Vc = Kc @ Wt.T
+    K = Kc.reshape(n, Hkv, d).transpose(1, 0, 2)
+    V = Vc.reshape(n, Hkv, d).transpose(1, 0, 2)
+    W = oracle.calibrate_layer(K, V, 1e-9)
+    assert W.shape == (Hkv * d, Hkv * d) and np.max(np.abs(W - Wt)) < 1e-7
+    N = 50
+    assert np.max(oracle.residual_layer(K[:, :N], V[:, :N], Wt, np.arange(N, dtype=np.int32))) < 1e-24
+    sc = rng.random(N).astype(np.float32)
+    r = oracle.route_layer(sc, K[:, :N], V[:, :N], Wt, 30, 20)
+    assert np.array_equal(r["pool_idx"], np.sort(np.argsort(-sc, kind="stable")[:30]))
+    assert sorted(np.concatenate([r["ret_idx"], r["apx_idx"]]).tolist()) == r["pool_idx"].tolist()
+    q = rng.standard_normal((Hkv * g, d))
+    pool = r["pool_idx"]
+    full, _ = oracle.attend_layer(q, K[:, pool], V[:, pool], K[:, :0], Wt, 0.35)
+    for n_ret in (0, 7, 30):
+        o_tok, o_fac = oracle.attend_layer(q, K[:, pool[:n_ret]], V[:, pool[:n_ret]], K[:, pool[n_ret:]], Wt, 0.35)
+        # the order of keys inside a softmax does not matter: retained first, approximated after
+        assert np.allclose(o_tok, full, rtol=1e-10, atol=1e-12) and np.allclose(o_fac, full, rtol=1e-10, atol=1e-12)
+
+
+def test_layer_score_is_the_sum_over_heads(oracle):
+    s = np.array([[0.5, 0.25, np.inf], [0.125, 1.0, np.inf]])
+    assert np.array_equal(oracle.layer_score(s), np.array([0.625, 1.25, np.inf]))
