@@ -255,6 +255,53 @@ VECTOR_API vector_status vector_diagnostics(const vector_shape* shape, const vec
                                  const float* eps, const void* V, float* out /* [U][8] */, void* stream);
 
 /*
+ * ---- One map per layer --------------------------------------------------------------------------
+ * The paper calibrates its map layer-wise (Section 5.1, "Implementation Details"; the Remark of
+ * Section 3.1 writes K and V as whole-layer projections): a token's key and value are then the
+ * concatenations over the layer's Hkv KV heads, W_layer has shape [Hkv d][Hkv d] (row-major,
+ * y = W x, one per layer: device [L][Hkv d][Hkv d] of shape->dtype), and because the reconstruction
+ * of one head's value reads every head's key of the token, a token's tier holds for the whole layer:
+ * scores, tier maps and index lists are per (sequence, layer), [B][L][...], while K, V, the cache
+ * pools, q and out keep the per-head layouts of the calls above (the Hkv pools of a layer list the
+ * same tokens).  Calibrate with vector_calibrate on host rows of Hkv d elements (d_k = d_v = Hkv d).
+ * RoPE decoupling is not implemented for this variant (VECTOR_ERR_UNSUPPORTED).
+ */
+/* Bytes of device workspace that suffice for vector_route_layer and vector_decode_attn_layer. */
+VECTOR_API size_t vector_layer_workspace_bytes(const vector_shape* shape, const vector_budget* budget);
+
+/* Layer score of a token = the sum over the layer's KV heads of its per-head base scores (window
+ * tokens stay +inf).  scores: device fp32 [B][L][Hkv][N]; layer_scores: device fp32 [B][L][N]. */
+VECTOR_API vector_status vector_layer_scores(const vector_shape* shape, const float* scores, int64_t N,
+                                             float* layer_scores, void* stream);
+
+/* Step 2 with the layer's map: eps[ul][p] = sum_h || v_{i,h} - (W_layer k_i)[h] ||^2, i = idx[ul][p],
+ * k_i the token's keys of all heads.  idx: device [B L][n_idx]; eps: device fp32 [B L][n_idx]. */
+VECTOR_API vector_status vector_residual_layer(const vector_shape* shape, const void* K, const void* V,
+                                               const void* W_layer, int64_t N, const int32_t* idx, int64_t n_idx,
+                                               float* eps, void* stream);
+
+/* Steps 1-3 per (sequence, layer) (Section 3.2 with the layer-wise map of Section 5.1).
+ * layer_scores: device fp32 [B L][N]; tier: device [B L][N]; ret_idx: device [B L][n_ret]; apx_idx:
+ * device [B L][n_apx]; eps_out, pool_idx_out (nullable): device [B L][n_pool]. */
+VECTOR_API vector_status vector_route_layer(const vector_shape* shape, const vector_budget* budget,
+                                            const float* layer_scores, const void* K, const void* V,
+                                            const void* W_layer, uint8_t* tier, int32_t* ret_idx, int32_t* apx_idx,
+                                            float* eps_out, int32_t* pool_idx_out, void* ws, size_t ws_bytes,
+                                            void* stream);
+
+/* vector_compact with one pair of index lists per (sequence, layer), shared by the layer's heads. */
+VECTOR_API vector_status vector_compact_layer(const vector_shape* shape, const vector_budget* budget,
+                                              const void* K, const void* V, const int32_t* ret_idx,
+                                              const int32_t* apx_idx, const vector_cache* cache, void* stream);
+
+/* Generation-time attention with the layer's map, factored form: per query head a of KV head h,
+ *   o_a = sum_R p_i v_{i,h} + sum_h' W_layer[h][h'] (sum_A p_i k_{i,h'}),  p = softmax over head h's keys
+ * (W_layer[h][h'] = the d x d block of output head h, input head h').  Arguments as vector_decode_attn. */
+VECTOR_API vector_status vector_decode_attn_layer(const vector_shape* shape, const void* q, const vector_cache* cache,
+                                                  const void* W_layer, void* out, int32_t out_dtype, void* ws,
+                                                  size_t ws_bytes, void* stream);
+
+/*
  * Allocation-free variant of vector_decode_attn (the paper has no counterpart:
  * this entry point exists for the integration, not for the method).
  *

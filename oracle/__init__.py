@@ -280,11 +280,9 @@ def attend_layer(q, ret_k, ret_v, apx_k, W, scale: float):
     -> (o_per_token [Hq][d], o_factored [Hq][d]) float64."""
     q, W = _f64(q), _f64(W)
     Hq, d = q.shape
-    Hkv = int(np.asarray(ret_k).shape[0]) if np.asarray(ret_k).ndim == 3 else int(np.asarray(apx_k).shape[0])
-    def cat(X, n_hint=None):
-        X = _f64(X)
-        if X.ndim != 3:
-            X = X.reshape(Hkv, -1, d)
+    Hkv = W.shape[0] // d
+    def cat(X):
+        X = _f64(X).reshape(Hkv, -1, d)
         return concat_heads(X) if X.shape[1] > 0 else np.zeros((0, Hkv * d))
     rk, rv, ak = cat(ret_k), cat(ret_v), cat(apx_k)
     o1 = np.empty((Hq, d), dtype=np.float64)

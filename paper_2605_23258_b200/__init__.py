@@ -11,5 +11,7 @@ from .binding import (  # noqa: F401
     vector_status_string, vector_plan_budget, vector_calibrate, vector_workspace_bytes,
     vector_score, vector_score_keydiff, vector_pool_select, vector_residual, vector_truncate, vector_route,
     vector_compact, vector_diagnostics, DIAG_FIELDS, vector_decode_attn, alloc_cache, alloc_workspace,
+    vector_layer_workspace_bytes, vector_layer_scores, vector_residual_layer, vector_route_layer, vector_compact_layer,
+    vector_decode_attn_layer,
     vector_device_fault, vector_kernel_launches, vector_decode_attn_static, vector_decode_scratch_bytes, VECTOR_STATIC_SCRATCH_BYTES,
 )

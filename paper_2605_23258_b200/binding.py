@@ -151,6 +151,16 @@ def load_library() -> ctypes.CDLL:
     lib.vector_decode_scratch_bytes.argtypes = [SP]
     lib.vector_decode_attn_static.argtypes = [SP, P, CP, P, P, I32, I32, P]
     lib.vector_decode_attn_static.restype = ctypes.c_int
+    lib.vector_layer_workspace_bytes.restype = SZ
+    lib.vector_layer_workspace_bytes.argtypes = [SP, BP]
+    lib.vector_layer_scores.argtypes = [SP, P, I64, P, P]
+    lib.vector_residual_layer.argtypes = [SP, P, P, P, I64, P, I64, P, P]
+    lib.vector_route_layer.argtypes = [SP, BP, P, P, P, P, P, P, P, P, P, P, SZ, P]
+    lib.vector_compact_layer.argtypes = [SP, BP, P, P, P, P, CP, P]
+    lib.vector_decode_attn_layer.argtypes = [SP, P, CP, P, P, I32, P, SZ, P]
+    for name in ("vector_layer_scores", "vector_residual_layer", "vector_route_layer", "vector_compact_layer",
+                 "vector_decode_attn_layer"):
+        getattr(lib, name).restype = ctypes.c_int
     for name in ("vector_plan_budget", "vector_calibrate", "vector_score", "vector_pool_select",
                  "vector_residual", "vector_truncate", "vector_route", "vector_compact", "vector_decode_attn"):
         getattr(lib, name).restype = ctypes.c_int
@@ -343,6 +353,59 @@ def vector_decode_attn(shape: Shape, q, cache: Cache, W, out, mode: int = 0, ws=
                                            ctypes.byref(c), _dev(W, shape.torch_dtype, "W"), _dev(out, None, "out"),
                                            out_dt, mode, wp, wn, _stream(stream))
     _check(rc, "vector_decode_attn")
+
+
+# ---- one map per layer: scores, tiers and index lists per (sequence, layer); pools per head
+def vector_layer_workspace_bytes(shape: Shape, budget: Budget) -> int:
+    return int(load_library().vector_layer_workspace_bytes(ctypes.byref(shape._c()), ctypes.byref(budget._c())))
+
+
+def vector_layer_scores(shape: Shape, scores, N: int, layer_scores, stream=None):
+    rc = load_library().vector_layer_scores(ctypes.byref(shape._c()), _dev(scores, torch.float32, "scores"), N,
+                                            _dev(layer_scores, torch.float32, "layer_scores"), _stream(stream))
+    _check(rc, "vector_layer_scores")
+
+
+def vector_residual_layer(shape: Shape, K, V, W_layer, N: int, idx, n_idx: int, eps, stream=None):
+    rc = load_library().vector_residual_layer(ctypes.byref(shape._c()), _dev(K, shape.torch_dtype, "K"),
+                                              _dev(V, shape.torch_dtype, "V"), _dev(W_layer, shape.torch_dtype, "W_layer"),
+                                              N, _dev(idx, torch.int32, "idx"), n_idx, _dev(eps, torch.float32, "eps"),
+                                              _stream(stream))
+    _check(rc, "vector_residual_layer")
+
+
+def vector_route_layer(shape: Shape, budget: Budget, layer_scores, K, V, W_layer, tier, ret_idx, apx_idx,
+                       eps_out=None, pool_idx_out=None, ws=None, stream=None):
+    wp, wn = _ws(ws)
+    rc = load_library().vector_route_layer(ctypes.byref(shape._c()), ctypes.byref(budget._c()),
+                                           _dev(layer_scores, torch.float32, "layer_scores"),
+                                           _dev(K, shape.torch_dtype, "K"), _dev(V, shape.torch_dtype, "V"),
+                                           _dev(W_layer, shape.torch_dtype, "W_layer"), _dev(tier, torch.uint8, "tier"),
+                                           _dev(ret_idx, torch.int32, "ret_idx"), _dev(apx_idx, torch.int32, "apx_idx"),
+                                           _dev(eps_out, torch.float32, "eps_out"),
+                                           _dev(pool_idx_out, torch.int32, "pool_idx_out"), wp, wn, _stream(stream))
+    _check(rc, "vector_route_layer")
+
+
+def vector_compact_layer(shape: Shape, budget: Budget, K, V, ret_idx, apx_idx, cache: Cache, stream=None):
+    c = cache._c()
+    rc = load_library().vector_compact_layer(ctypes.byref(shape._c()), ctypes.byref(budget._c()),
+                                             _dev(K, shape.torch_dtype, "K"), _dev(V, shape.torch_dtype, "V"),
+                                             _dev(ret_idx, torch.int32, "ret_idx"), _dev(apx_idx, torch.int32, "apx_idx"),
+                                             ctypes.byref(c), _stream(stream))
+    _check(rc, "vector_compact_layer")
+
+
+def vector_decode_attn_layer(shape: Shape, q, cache: Cache, W_layer, out, ws=None, stream=None):
+    wp, wn = _ws(ws)
+    c = cache._c()
+    if out.dtype not in (torch.float32, torch.bfloat16):
+        raise ValueError("out must be fp32 or bf16")
+    out_dt = VECTOR_BF16 if out.dtype == torch.bfloat16 else VECTOR_F32
+    rc = load_library().vector_decode_attn_layer(ctypes.byref(shape._c()), _dev(q, shape.torch_dtype, "q"),
+                                                 ctypes.byref(c), _dev(W_layer, shape.torch_dtype, "W_layer"),
+                                                 _dev(out, None, "out"), out_dt, wp, wn, _stream(stream))
+    _check(rc, "vector_decode_attn_layer")
 
 
 VECTOR_STATIC_SCRATCH_BYTES = 16 << 20

@@ -10,7 +10,7 @@ CSRC = os.path.join(HERE, "csrc")
 INCLUDE = os.path.join(os.path.dirname(HERE), "include")
 LIB = os.path.join(HERE, "libvector.so")
 
-SOURCES = ["host.cpp", "score.cu", "keydiff.cu", "route.cu", "compact.cu", "decode.cu", "diagnostics.cu"]
+SOURCES = ["host.cpp", "score.cu", "keydiff.cu", "route.cu", "compact.cu", "decode.cu", "decode_layer.cu", "diagnostics.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xptxas=-v",
               "-Xcompiler", "-fPIC,-O3,-fvisibility=hidden", "-I", INCLUDE, "-I", CSRC]

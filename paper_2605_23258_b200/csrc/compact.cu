@@ -13,14 +13,17 @@ constexpr int COMPACT_PASSES = 4;
 // Logical row r of a unit: [0, n_ret) K -> ret_k ; [n_ret, 2 n_ret) V -> ret_v ;
 // [2 n_ret, 2 n_ret + n_apx) K -> apx_k.  A row is `pieces` = 2^lp pieces of 16 bytes; a block owns
 // COMPACT_PASSES * (COMPACT_THREADS >> lp) consecutive rows of one unit.  grid: U * chunks blocks.
+// idx_div = 1: one pair of index lists per unit; idx_div = Hkv: one pair per (sequence, layer), shared
+// by the layer's KV heads (routing with one map per layer).
 __global__ void __launch_bounds__(COMPACT_THREADS)
 compact_kernel(const uint4* __restrict__ K, const uint4* __restrict__ V, int64_t N, int lp,
                const int32_t* __restrict__ ret_idx, const int32_t* __restrict__ apx_idx, int n_ret, int n_apx,
                uint4* __restrict__ ret_k, uint4* __restrict__ ret_v, uint4* __restrict__ apx_k,
                int32_t* __restrict__ ret_pos, int32_t* __restrict__ apx_pos, int64_t cap_ret, int64_t cap_apx,
-               int chunks) {
+               int chunks, int idx_div) {
     const int rows = 2 * n_ret + n_apx, pieces = 1 << lp;
     const int u = blockIdx.x / chunks, chunk = blockIdx.x - u * chunks;
+    const int ui = u / idx_div;                      // owner of the index lists: the unit, or its (sequence, layer)
     const int piece = threadIdx.x & (pieces - 1), rsub = threadIdx.x >> lp, per_pass = COMPACT_THREADS >> lp;
     const uint4* src[COMPACT_PASSES];
     uint4* dst[COMPACT_PASSES];
@@ -32,16 +35,16 @@ compact_kernel(const uint4* __restrict__ K, const uint4* __restrict__ V, int64_t
         src[p] = nullptr; dst[p] = nullptr; pos[p] = nullptr; tok[p] = 0;
         if (r >= rows) continue;
         if (r < n_ret) {
-            tok[p] = ret_idx[(size_t)u * n_ret + r];
+            tok[p] = ret_idx[(size_t)ui * n_ret + r];
             src[p] = K; dst[p] = ret_k + (((size_t)u * cap_ret + r) << lp) + piece;
             pos[p] = ret_pos + (size_t)u * cap_ret + r;
         } else if (r < 2 * n_ret) {
             const int q = r - n_ret;
-            tok[p] = ret_idx[(size_t)u * n_ret + q];
+            tok[p] = ret_idx[(size_t)ui * n_ret + q];
             src[p] = V; dst[p] = ret_v + (((size_t)u * cap_ret + q) << lp) + piece;
         } else {
             const int q = r - 2 * n_ret;
-            tok[p] = apx_idx[(size_t)u * n_apx + q];
+            tok[p] = apx_idx[(size_t)ui * n_apx + q];
             src[p] = K; dst[p] = apx_k + (((size_t)u * cap_apx + q) << lp) + piece;
             pos[p] = apx_pos + (size_t)u * cap_apx + q;
         }
@@ -63,9 +66,9 @@ compact_kernel(const uint4* __restrict__ K, const uint4* __restrict__ V, int64_t
 
 using namespace vec;
 
-extern "C" vector_status vector_compact(const vector_shape* shape, const vector_budget* budget, const void* K,
-                                        const void* V, const int32_t* ret_idx, const int32_t* apx_idx,
-                                        const vector_cache* cache, void* stream) {
+static vector_status compact_launch(const vector_shape* shape, const vector_budget* budget, const void* K,
+                                    const void* V, const int32_t* ret_idx, const int32_t* apx_idx,
+                                    const vector_cache* cache, void* stream, bool per_layer) {
     Dims dm;
     vector_status rc = check_shape(shape, &dm);
     if (rc != VECTOR_OK) return rc;
@@ -88,7 +91,19 @@ extern "C" vector_status vector_compact(const vector_shape* shape, const vector_
     compact_kernel<<<(unsigned)blocks, COMPACT_THREADS, 0, (cudaStream_t)stream>>>(
         (const uint4*)K, (const uint4*)V, budget->n_tokens, lp, ret_idx, apx_idx, (int)budget->n_ret,
         (int)budget->n_apx, (uint4*)cache->ret_k, (uint4*)cache->ret_v, (uint4*)cache->apx_k, cache->ret_pos,
-        cache->apx_pos, cache->cap_ret, cache->cap_apx, (int)chunks);
+        cache->apx_pos, cache->cap_ret, cache->cap_apx, (int)chunks, per_layer ? shape->n_kv_heads : 1);
     VEC_LAUNCH_CHECK();
     return VECTOR_OK;
+}
+
+extern "C" vector_status vector_compact(const vector_shape* shape, const vector_budget* budget, const void* K,
+                                        const void* V, const int32_t* ret_idx, const int32_t* apx_idx,
+                                        const vector_cache* cache, void* stream) {
+    return compact_launch(shape, budget, K, V, ret_idx, apx_idx, cache, stream, false);
+}
+
+extern "C" vector_status vector_compact_layer(const vector_shape* shape, const vector_budget* budget, const void* K,
+                                              const void* V, const int32_t* ret_idx, const int32_t* apx_idx,
+                                              const vector_cache* cache, void* stream) {
+    return compact_launch(shape, budget, K, V, ret_idx, apx_idx, cache, stream, true);
 }

@@ -7,6 +7,7 @@
 // indices in ascending order.  One thread block per unit.
 #include "common.cuh"
 #include "internal.h"
+#include "residual_layer_tc.cuh"
 #include "residual_tc.cuh"
 #include "select.cuh"
 
@@ -239,6 +240,95 @@ static vector_status launch_truncate(const Dims& dm, const vector_budget* budget
     return VECTOR_OK;
 }
 
+// ---- one map per layer: a token's tier holds for all KV heads of its layer -----------------------
+// Layer score of a token = the sum of its per-head base scores (window tokens stay +inf), summed in
+// head order.  grid (ceil(N / 256), B L), 256 threads.
+__global__ void __launch_bounds__(256)
+layer_scores_kernel(const float* __restrict__ scores, int64_t N, int Hkv, float* __restrict__ layer_scores) {
+    const int ul = blockIdx.y;
+    const int64_t i = (int64_t)blockIdx.x * 256 + threadIdx.x;
+    if (i >= N) return;
+    float s = 0.f;
+    for (int h = 0; h < Hkv; ++h) s += scores[((size_t)ul * Hkv + h) * N + i];
+    layer_scores[(size_t)ul * N + i] = s;
+}
+
+// Step 2 with one map per layer on CUDA cores (any dtype and head size): a warp per listed token,
+// the token's keys of all heads in shared memory, lane = output channels lane, lane + 32, ...
+// grid (ceil(n_idx / 8), B L), 256 threads, dynamic shared memory 8 * Hkv * D floats.
+template <typename T, int D>
+__global__ void __launch_bounds__(256)
+residual_layer_generic(const T* __restrict__ K, const T* __restrict__ V, const T* __restrict__ W, int64_t N, int L,
+                       int Hkv, const int32_t* __restrict__ idx, int n_idx, float* __restrict__ eps) {
+    extern __shared__ float ksm[];
+    const int ul = blockIdx.y, lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
+    const int DL = Hkv * D;
+    const int p = blockIdx.x * 8 + wid;
+    if (p >= n_idx) return;
+    const int64_t tok = idx[(size_t)ul * n_idx + p];
+    if ((uint64_t)tok >= (uint64_t)N) {              // an index outside the unit reads as rows of zeros
+        if (lane == 0) eps[(size_t)ul * n_idx + p] = 0.f;
+        return;
+    }
+    float* kw = ksm + (size_t)wid * DL;
+    for (int c = lane; c < DL; c += 32) kw[c] = to_f32(K[(((size_t)ul * Hkv + c / D) * N + tok) * D + c % D]);
+    __syncwarp();
+    const T* Wl = W + (size_t)(ul % L) * DL * DL;
+    float e = 0.f;
+    for (int co = lane; co < DL; co += 32) {
+        const T* row = Wl + (size_t)co * DL;
+        float pred = 0.f;
+        for (int ci = 0; ci < DL; ++ci) pred = fmaf(to_f32(row[ci]), kw[ci], pred);
+        const float r = to_f32(V[(((size_t)ul * Hkv + co / D) * N + tok) * D + co % D]) - pred;
+        e = fmaf(r, r, e);
+    }
+    e = warp_sum(e);
+    if (lane == 0) eps[(size_t)ul * n_idx + p] = e;
+}
+
+static vector_status residual_layer_dispatch(const Dims& dm, int Hkv, int L, const void* K, const void* V, const void* W,
+                                             int64_t N, const int32_t* idx, int64_t n_idx, float* eps, cudaStream_t st,
+                                             bool dependent) {
+    if (n_idx == 0) return VECTOR_OK;
+    const int UL = dm.U / Hkv;
+    if (dm.dtype == VECTOR_BF16 && dm.d == 128) {
+        static PerDeviceOnce once;
+        if (once.first()) {
+            const cudaError_t e = cudaFuncSetAttribute(rlt::residual_layer_tc, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                                       rlt::SMEM_BYTES);
+            if (e != cudaSuccess) { once.undo(); VEC_CUDA_CHECK(e); }
+        }
+        int* fault = kernel_fault_address();
+        if (!fault) return VECTOR_ERR_CUDA;
+        const uint64_t DL = (uint64_t)Hkv * 128;
+        CUtensorMap mapW;
+        if (!tma::encode_bf16_3d(&mapW, W, DL, DL, (uint64_t)L, DL * 2, DL * DL * 2, 64, 128)) return VECTOR_ERR_CUDA;
+        rlt::Params P;
+        P.UL = UL; P.L = L; P.Hkv = Hkv; P.n_idx = (int)n_idx; P.N = N;
+        P.tpu = (int)((n_idx + rlt::TILE - 1) / rlt::TILE);
+        P.n_tiles = (long long)UL * P.tpu;
+        const int sms = sm_count();
+        const int blocks = (int)(P.n_tiles < sms ? P.n_tiles : sms);
+        VEC_CUDA_CHECK(launch_maybe_dependent(dependent, rlt::residual_layer_tc, dim3(blocks), dim3(rlt::THREADS), rlt::SMEM_BYTES,
+                                              st, (const __nv_bfloat16*)K, (const __nv_bfloat16*)V, mapW, idx, P, eps, fault));
+        return VECTOR_OK;
+    }
+    const dim3 grid((unsigned)((n_idx + 7) / 8), UL);
+    const size_t smem = (size_t)8 * Hkv * dm.d * sizeof(float);
+#define VEC_RL(T, D)                                                                                                   \
+    do {                                                                                                               \
+        VEC_CUDA_CHECK(cudaFuncSetAttribute(residual_layer_generic<T, D>, cudaFuncAttributeMaxDynamicSharedMemorySize, \
+                                            (int)smem));                                                               \
+        residual_layer_generic<T, D><<<grid, 256, smem, st>>>((const T*)K, (const T*)V, (const T*)W, N, L, Hkv, idx,   \
+                                                              (int)n_idx, eps);                                        \
+    } while (0)
+    if (dm.dtype == VECTOR_F32) { if (dm.d == 64) VEC_RL(float, 64); else VEC_RL(float, 128); }
+    else { if (dm.d == 64) VEC_RL(__nv_bfloat16, 64); else VEC_RL(__nv_bfloat16, 128); }
+#undef VEC_RL
+    VEC_LAUNCH_CHECK();
+    return VECTOR_OK;
+}
+
 }  // namespace vec
 
 using namespace vec;
@@ -298,4 +388,58 @@ extern "C" vector_status vector_route(const vector_shape* shape, const vector_bu
     rc = residual_dispatch(dm, K, V, W, budget->n_tokens, pool, budget->n_pool, eps, st, true);
     if (rc != VECTOR_OK) return rc;
     return launch_truncate(dm, budget, eps, pool, tier, ret_idx, apx_idx, st, true);
+}
+
+extern "C" vector_status vector_layer_scores(const vector_shape* shape, const float* scores, int64_t N,
+                                             float* layer_scores, void* stream) {
+    Dims dm;
+    vector_status rc = check_shape(shape, &dm);
+    if (rc != VECTOR_OK) return rc;
+    if (!scores || !layer_scores) return VECTOR_ERR_NULL;
+    if (N <= 0 || N > (int64_t(1) << 30)) return VECTOR_ERR_SHAPE;
+    const int Hkv = shape->n_kv_heads;
+    const dim3 grid((unsigned)((N + 255) / 256), dm.U / Hkv);
+    layer_scores_kernel<<<grid, 256, 0, (cudaStream_t)stream>>>(scores, N, Hkv, layer_scores);
+    VEC_LAUNCH_CHECK();
+    return VECTOR_OK;
+}
+
+extern "C" vector_status vector_residual_layer(const vector_shape* shape, const void* K, const void* V, const void* W_layer,
+                                               int64_t N, const int32_t* idx, int64_t n_idx, float* eps, void* stream) {
+    Dims dm;
+    vector_status rc = check_shape(shape, &dm);
+    if (rc != VECTOR_OK) return rc;
+    if (!K || !V || !W_layer || !idx || !eps) return VECTOR_ERR_NULL;
+    if (N <= 0 || N > (int64_t(1) << 30) || n_idx < 0 || n_idx > N) return VECTOR_ERR_SHAPE;
+    if (dm.rope) return VECTOR_ERR_UNSUPPORTED;
+    return residual_layer_dispatch(dm, shape->n_kv_heads, shape->n_layers, K, V, W_layer, N, idx, n_idx, eps,
+                                   (cudaStream_t)stream, false);
+}
+
+extern "C" vector_status vector_route_layer(const vector_shape* shape, const vector_budget* budget, const float* layer_scores,
+                                            const void* K, const void* V, const void* W_layer, uint8_t* tier,
+                                            int32_t* ret_idx, int32_t* apx_idx, float* eps_out, int32_t* pool_idx_out,
+                                            void* ws, size_t ws_bytes, void* stream) {
+    Dims dm;
+    vector_status rc = check_shape(shape, &dm);
+    if (rc != VECTOR_OK) return rc;
+    if ((rc = check_budget(budget, dm.w)) != VECTOR_OK) return rc;
+    if (!layer_scores || !K || !V || !W_layer || !tier) return VECTOR_ERR_NULL;
+    if ((budget->n_ret > 0 && !ret_idx) || (budget->n_apx > 0 && !apx_idx)) return VECTOR_ERR_NULL;
+    if (dm.rope) return VECTOR_ERR_UNSUPPORTED;
+    const int Hkv = shape->n_kv_heads;
+    Dims dl = dm;                       // the selections run per (sequence, layer)
+    dl.U = dm.U / Hkv;
+    const size_t need = align256((size_t)dl.U * (size_t)budget->n_pool * sizeof(int32_t)) +
+                        align256((size_t)dl.U * (size_t)budget->n_pool * sizeof(float));
+    if (!ws || ((uintptr_t)ws & 255) || ws_bytes < need) return VECTOR_ERR_WORKSPACE;
+    char* p = (char*)ws;
+    int32_t* pool = pool_idx_out ? pool_idx_out : (int32_t*)p;
+    p += align256((size_t)dl.U * (size_t)budget->n_pool * sizeof(int32_t));
+    float* eps = eps_out ? eps_out : (float*)p;
+    cudaStream_t st = (cudaStream_t)stream;
+    if ((rc = launch_pool_select(dl, budget, layer_scores, pool, st)) != VECTOR_OK) return rc;
+    rc = residual_layer_dispatch(dm, Hkv, shape->n_layers, K, V, W_layer, budget->n_tokens, pool, budget->n_pool, eps, st, true);
+    if (rc != VECTOR_OK) return rc;
+    return launch_truncate(dl, budget, eps, pool, tier, ret_idx, apx_idx, st, true);
 }

@@ -182,6 +182,45 @@ def context(wl: Workload, device, units=None):
     return K, V, Q
 
 
+# ---- one map per layer: values depend on the keys of all heads of the layer ------------------------
+def layer_params(wl: Workload, l: int, device):
+    """-> sigma_K [Hkv][d], sigma_Q [Hkv][d], W_true [Hkv d][Hkv d] (fp32) for one layer: the channel scales of
+    its heads and a dense whole-layer map (cross-head blocks included)."""
+    per_head = [head_params(wl, l, h, device) for h in range(wl.n_kv_heads)]
+    D = wl.n_kv_heads * wl.head_dim
+    gen = _gen(device, wl.wid, _STREAM["head"], l, 10**6)
+    w_true = torch.randn(D, D, generator=gen, device=device, dtype=torch.float32) / math.sqrt(D)
+    return torch.stack([p[0] for p in per_head]), torch.stack([p[1] for p in per_head]), w_true
+
+
+def _layer_kv(wl: Workload, gen, n: int, sigma_k, w_true, l: int, device):
+    Hkv, d = wl.n_kv_heads, wl.head_dim
+    k = torch.randn(n, Hkv, d, generator=gen, device=device, dtype=torch.float32) * sigma_k[None]
+    if wl.noise == "two_level":
+        pick = torch.rand(n, generator=gen, device=device) < 0.5
+        s = torch.where(pick, torch.tensor(0.05, device=device), torch.tensor(1.0, device=device))
+    else:
+        s = _loguniform((n,), 0.02, 2.0, gen, device)
+    s = s * _layer_factor(wl, l)
+    z = torch.randn(n, Hkv * d, generator=gen, device=device, dtype=torch.float32)
+    v = k.reshape(n, Hkv * d) @ w_true.T + s[:, None] * z
+    k = k.permute(1, 0, 2).contiguous().to(wl.torch_dtype)                       # [Hkv][n][d]
+    v = v.reshape(n, Hkv, d).permute(1, 0, 2).contiguous().to(wl.torch_dtype)
+    return k, v
+
+
+def layer_kv(wl: Workload, b: int, l: int, device, params=None):
+    """Context K, V [Hkv][N][d] of one (sequence, layer): V = W_true K + noise over whole-layer vectors."""
+    sigma_k, _, w_true = params if params is not None else layer_params(wl, l, device)
+    return _layer_kv(wl, _gen(device, wl.wid, _STREAM["ctx"], l, 10**6, b), wl.N, sigma_k, w_true, l, device)
+
+
+def layer_calib_kv(wl: Workload, l: int, device, params=None):
+    """Calibration draw K, V [Hkv][n_calib][d] for one layer: separate seed, same law."""
+    sigma_k, _, w_true = params if params is not None else layer_params(wl, l, device)
+    return _layer_kv(wl, _gen(device, wl.wid, _STREAM["calib"], l, 10**6), wl.n_calib, sigma_k, w_true, l, device)
+
+
 def all_head_params(wl: Workload, device):
     """Stacked sigma_K [LH][d], sigma_Q [LH][d], W_true [LH][d][d]."""
     sk, sq, wt = [], [], []
