@@ -409,8 +409,10 @@ def run_workload(env, cfg, wl, percent, steps, warmup, D, extras=True, want_e2e=
             us = a.elapsed_time(b_) * 1e3 / 10
             step_bytes = U * (2 * n_ret + n_apx) * d * es
             extra_flop = 2.0 * U * n_apx * d * d
+            fac_us = ms["decode"] * 1e3 / D
             per_tile = {"us_per_step": us, "gbs": step_bytes / us / 1e3, "extra_flop_per_step": extra_flop,
-                        "extra_tflops": extra_flop / (us * 1e-6) / 1e12}
+                        "ratio_to_factored_step": us / fac_us,
+                        "extra_tflops_over_added_time": extra_flop / (max(us - fac_us, 1e-3) * 1e-6) / 1e12}
 
         # ---- the query-agnostic base scorer (key geometry), outside the timed step: two HBM passes over K
         kd_scores = torch.empty(U, N, dtype=torch.float32, device=dev)
@@ -457,6 +459,45 @@ def run_workload(env, cfg, wl, percent, steps, warmup, D, extras=True, want_e2e=
                     "decode_frac_of_measured_copy": step_bytes / us / 1e3 / hbm,
                     "sincos_per_decode_step": 2.0 * U * n_apx * (d // 2), "sincos_per_route": 2.0 * U * n_pool * (d // 2)}
             del comp_r
+
+    # ---- one map per layer (the paper's layer-wise calibration): routing per (sequence, layer) with the
+    #      K = Hkv d residual contraction, and decode attention with the cross-head blocks; outside the timed
+    #      step, a random map (the time does not depend on its values; parity is the tests' business)
+    layer_map = None
+    if extras and wl.dtype == "bf16" and d == 128 and cfg == 2:
+        Hkv, UL = wl.n_kv_heads, U // wl.n_kv_heads
+        DL = Hkv * d
+        Wl = (torch.randn(wl.n_layers, DL, DL, device=dev) * (1.0 / DL ** 0.5)).to(wl.torch_dtype)
+        lws = torch.empty(vec.vector_layer_workspace_bytes(shape, budget), dtype=torch.uint8, device=dev)
+        lsc = torch.empty(UL, N, dtype=torch.float32, device=dev)
+        l_tier = torch.empty(UL, N, dtype=torch.uint8, device=dev)
+        l_ret = torch.empty(UL, n_ret, dtype=torch.int32, device=dev)
+        l_apx = torch.empty(UL, n_apx, dtype=torch.int32, device=dev)
+        comp.score(Qt, Kt)
+        comp.cache.n_ret = budget.n_ret
+
+        def timed(f, n):
+            for _ in range(2):
+                f()
+            a, b_ = ev(), ev()
+            torch.cuda.synchronize(); a.record()
+            for _ in range(n):
+                f()
+            b_.record(); torch.cuda.synchronize()
+            return a.elapsed_time(b_) / n
+
+        ls_ms = timed(lambda: vec.vector_layer_scores(shape, comp.scores, N, lsc), 5)
+        rl_ms = timed(lambda: vec.vector_route_layer(shape, budget, lsc, Kt, Vt, Wl, l_tier, l_ret, l_apx, None, None, lws), 5)
+        cl_ms = timed(lambda: vec.vector_compact_layer(shape, budget, Kt, Vt, l_ret, l_apx, comp.cache), 5)
+        dl_ms = timed(lambda: vec.vector_decode_attn_layer(shape, qs[0], comp.cache, Wl, out, lws), 3)
+        rl_flop = 2.0 * UL * n_pool * DL * DL
+        layer_map = {"layer_scores_ms": ls_ms, "route_layer_ms": rl_ms, "route_layer_tflops": rl_flop / (rl_ms * 1e-3) / 1e12,
+                     "route_layer_frac_of_sustained_bf16": rl_flop / (rl_ms * 1e-3) / 1e12 / tf,
+                     "compact_layer_ms": cl_ms, "decode_layer_us_per_step": dl_ms * 1e3,
+                     "decode_layer_gbs": U * (2 * n_ret + n_apx) * d * es / (dl_ms * 1e-3) / 1e9,
+                     "note": "first device version: tcgen05 residual at the L2 rate, CUDA-core decode"}
+        del Wl, lws, lsc, l_tier, l_ret, l_apx
+        comp.compact(Kt, Vt)              # the per-head cache back in place for what follows
 
     # ---- end to end through host buffers: every step copies its inputs from pinned host memory to the
     #      device and reads the routing result back; the copies run layer by layer
@@ -548,7 +589,7 @@ def run_workload(env, cfg, wl, percent, steps, warmup, D, extras=True, want_e2e=
                    "frac_of_8tbs": decode_bytes / (dec_ms_max * 1e-3) / 1e9 / 8000.0,
                    "us_per_step": dec_ms_max * 1e3 / D, "tokens_per_s": world * wl.batch * D / (dec_ms_max * 1e-3),
                    "bytes_per_step": decode_bytes / D},
-        "decode_per_tile": per_tile, "score_keydiff": keydiff, "rope_decoupled": rope, "roofline": roofline,
+        "decode_per_tile": per_tile, "score_keydiff": keydiff, "rope_decoupled": rope, "layer_map": layer_map, "roofline": roofline,
         "roofline_kernels": kernels, "cpu_baseline": cpu, "e2e": e2e,
         "gpu_launches": launches, "device_fault": fault, "clocks": clocks,
     }
@@ -596,7 +637,7 @@ def main():
                              extras=not args.no_extras and c == 2, want_e2e=False, want_cpu=False)
             side[f"config{c}"] = {k: r[k] for k in ("value", "unit", "steps", "warmup", "ms_per_step", "config",
                                                     "compress_ms", "phase_ms", "decode", "decode_per_tile",
-                                                    "score_keydiff", "rope_decoupled", "roofline_kernels",
+                                                    "score_keydiff", "rope_decoupled", "layer_map", "roofline_kernels",
                                                     "gpu_launches", "device_fault", "clocks")}
         line["configs"] = side
     if env.rank == 0:

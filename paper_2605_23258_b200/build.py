@@ -32,7 +32,9 @@ def _stale() -> bool:
 
 
 def build(force: bool = False, verbose: bool = False) -> str:
-    """Compile every translation unit to an object and link the shared library."""
+    """Compile every translation unit to an object and link the shared library.  Extra nvcc flags can be
+    given in the environment variable VECTOR_NVCC_FLAGS (e.g. -DVECTOR_SCORE_POLY16=6 for the sweep of the
+    share of softmax exponentials evaluated on the FMA pipe)."""
     if not force and not _stale():
         return LIB
     objdir = os.path.join(HERE, "_build")
@@ -41,7 +43,7 @@ def build(force: bool = False, verbose: bool = False) -> str:
     procs = []
     for src in SOURCES:
         obj = os.path.join(objdir, src + ".o")
-        cmd = [nvcc, *NVCC_FLAGS, "-c", os.path.join(CSRC, src), "-o", obj]
+        cmd = [nvcc, *NVCC_FLAGS, *os.environ.get("VECTOR_NVCC_FLAGS", "").split(), "-c", os.path.join(CSRC, src), "-o", obj]
         procs.append((src, obj, subprocess.Popen(cmd, stdout=subprocess.PIPE, stderr=subprocess.STDOUT, text=True)))
     objs = []
     for src, obj, p in procs:
