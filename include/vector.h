@@ -28,7 +28,9 @@
  *    row-major, one d x d map per (layer, KV head): index l * n_kv_heads + h.
  *  - Supported: head_dim 64 or 128; dtype fp32 or bf16; n_q_heads % n_kv_heads == 0,
  *    g <= 8; window * g <= 1024; pool_kernel odd, 1..15; at most 65535 units per call;
- *    every device pointer 16-byte aligned.
+ *    every device pointer 16-byte aligned.  The tensor-core kernels (tcgen05 score passes and residual,
+ *    TMA-fed decode) serve bf16 with head_dim 128; fp32 and head_dim 64 run on CUDA-core kernels of the
+ *    same interface, written for parity rather than speed.
  */
 #ifndef VECTOR_H_
 #define VECTOR_H_
@@ -55,7 +57,7 @@ typedef enum {
     VECTOR_ERR_WORKSPACE = -5,   /* workspace NULL, misaligned or too small         */
     VECTOR_ERR_SINGULAR = -6,    /* Gram matrix not positive definite               */
     VECTOR_ERR_CUDA = -7,        /* a CUDA runtime call failed (see last_cuda_error) */
-    VECTOR_ERR_TIMEOUT = -8,     /* reserved for host-side waits                    */
+    VECTOR_ERR_TIMEOUT = -8,     /* a bounded wait inside a kernel gave up (vector_sync_check) */
     VECTOR_ERR_UNSUPPORTED = -9  /* valid request this build does not implement     */
 } vector_status;
 
@@ -137,6 +139,13 @@ VECTOR_API vector_status vector_calibrate(const void* K, const void* V, int64_t 
  * clearing it.  Results of the call that recorded a fault are invalid.
  */
 VECTOR_API int vector_device_fault(void);
+
+/*
+ * The same check as a status and on one stream: waits until the work queued on `stream` has finished,
+ * then returns VECTOR_OK, VECTOR_ERR_TIMEOUT if a bounded wait inside a kernel gave up since the last
+ * check (the record is cleared; outputs written since then are invalid), or VECTOR_ERR_CUDA.
+ */
+VECTOR_API vector_status vector_sync_check(void* stream);
 
 /* Bytes of device workspace that suffice for every device call with this shape and budget. */
 VECTOR_API size_t vector_workspace_bytes(const vector_shape* shape, const vector_budget* budget);
@@ -253,6 +262,18 @@ VECTOR_API vector_status vector_decode_attn(const vector_shape* shape, const voi
 VECTOR_API vector_status vector_diagnostics(const vector_shape* shape, const vector_budget* budget,
                                  const float* importance, const uint8_t* tier, const int32_t* pool_idx,
                                  const float* eps, const void* V, float* out /* [U][8] */, void* stream);
+
+/*
+ * K -> V predictability of a map over a whole context (the R^2_global of the paper's Section 3.1,
+ * "Empirical Evidence", and its cross-model table): per unit, over ALL N tokens,
+ *   R^2 = 1 - sum_i ||v_i - W k_i||^2 / sum_i ||v_i - mean(v)||^2.
+ * K, V: device [U][N][d]; W: device [L][Hkv][d][d]; out: device fp32 [U][4] = { R^2, SS_res, SS_tot, N }
+ * (R^2 = 1 when both sums are 0, -inf when only SS_tot is).  The residuals come from the kernel of
+ * vector_residual, the sums are carried in fp64.  ws: at least vector_r2_global_workspace_bytes().
+ */
+VECTOR_API size_t vector_r2_global_workspace_bytes(const vector_shape* shape, int64_t N);
+VECTOR_API vector_status vector_r2_global(const vector_shape* shape, const void* K, const void* V, const void* W,
+                                          int64_t N, float* out /* [U][4] */, void* ws, size_t ws_bytes, void* stream);
 
 /*
  * ---- One map per layer --------------------------------------------------------------------------

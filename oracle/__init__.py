@@ -214,6 +214,25 @@ def diagnostics(importance, tier, K, V, W) -> dict:
     return dict(zip(DIAG_FIELDS, out.tolist()))
 
 
+def r2_global(K, V, W) -> dict:
+    """K -> V predictability of a fixed map over a whole context (Section 3.1, "Empirical Evidence"):
+    R^2 = 1 - sum_i ||v_i - W k_i||^2 / sum_i ||v_i - mean(v)||^2 over ALL tokens, the residual of each token
+    taken by the residual step itself (identity index list)."""
+    K, V, W = _f64(K), _f64(V), _f64(W)
+    N = K.shape[0]
+    eps = residual(K, V, W, np.arange(N, dtype=np.int32))
+    ss_res = float(np.sum(eps))
+    mean = np.zeros(V.shape[1])
+    for i in range(N):
+        mean += V[i]
+    mean /= N
+    ss_tot = 0.0
+    for i in range(N):
+        ss_tot += float(np.sum((V[i] - mean) ** 2))
+    r2 = 1.0 - ss_res / ss_tot if ss_tot > 0.0 else (1.0 if ss_res == 0.0 else -np.inf)
+    return dict(r2=r2, ss_res=ss_res, ss_tot=ss_tot, n=N)
+
+
 def gather_rows(src, idx):
     """-> (rows [n_idx][d] float64, pos int32)."""
     src, idx = _f64(src), _i32(idx)

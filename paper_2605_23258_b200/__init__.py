@@ -13,5 +13,6 @@ from .binding import (  # noqa: F401
     vector_compact, vector_diagnostics, DIAG_FIELDS, vector_decode_attn, alloc_cache, alloc_workspace,
     vector_layer_workspace_bytes, vector_layer_scores, vector_residual_layer, vector_route_layer, vector_compact_layer,
     vector_decode_attn_layer,
+    vector_r2_global, vector_r2_global_workspace_bytes, R2_FIELDS, vector_sync_check,
     vector_device_fault, vector_kernel_launches, vector_decode_attn_static, vector_decode_scratch_bytes, VECTOR_STATIC_SCRATCH_BYTES,
 )

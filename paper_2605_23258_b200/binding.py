@@ -158,6 +158,12 @@ def load_library() -> ctypes.CDLL:
     lib.vector_route_layer.argtypes = [SP, BP, P, P, P, P, P, P, P, P, P, P, SZ, P]
     lib.vector_compact_layer.argtypes = [SP, BP, P, P, P, P, CP, P]
     lib.vector_decode_attn_layer.argtypes = [SP, P, CP, P, P, I32, P, SZ, P]
+    lib.vector_r2_global_workspace_bytes.restype = SZ
+    lib.vector_r2_global_workspace_bytes.argtypes = [SP, I64]
+    lib.vector_r2_global.argtypes = [SP, P, P, P, I64, P, P, SZ, P]
+    lib.vector_r2_global.restype = ctypes.c_int
+    lib.vector_sync_check.argtypes = [P]
+    lib.vector_sync_check.restype = ctypes.c_int
     for name in ("vector_layer_scores", "vector_residual_layer", "vector_route_layer", "vector_compact_layer",
                  "vector_decode_attn_layer"):
         getattr(lib, name).restype = ctypes.c_int
@@ -332,6 +338,27 @@ def vector_diagnostics(shape: Shape, budget: Budget, importance, tier, pool_idx,
                                            _dev(pool_idx, torch.int32, "pool_idx"), _dev(eps, torch.float32, "eps"),
                                            _dev(V, shape.torch_dtype, "V"), _dev(out, torch.float32, "out"), _stream(stream))
     _check(rc, "vector_diagnostics")
+
+
+R2_FIELDS = ("r2", "ss_res", "ss_tot", "n")
+
+
+def vector_r2_global_workspace_bytes(shape: Shape, N: int) -> int:
+    return int(load_library().vector_r2_global_workspace_bytes(ctypes.byref(shape._c()), N))
+
+
+def vector_r2_global(shape: Shape, K, V, W, N: int, out, ws, stream=None):
+    """out [U][4] fp32: the R2_FIELDS of every unit over all N tokens."""
+    wp, wn = _ws(ws)
+    rc = load_library().vector_r2_global(ctypes.byref(shape._c()), _dev(K, shape.torch_dtype, "K"),
+                                         _dev(V, shape.torch_dtype, "V"), _dev(W, shape.torch_dtype, "W"),
+                                         N, _dev(out, torch.float32, "out"), wp, wn, _stream(stream))
+    _check(rc, "vector_r2_global")
+
+
+def vector_sync_check(stream=None):
+    """Waits for the stream; raises VectorError(VECTOR_ERR_TIMEOUT) if a bounded wait inside a kernel gave up."""
+    _check(load_library().vector_sync_check(_stream(stream)), "vector_sync_check")
 
 
 def vector_compact(shape: Shape, budget: Budget, K, V, ret_idx, apx_idx, cache: Cache, stream=None):

@@ -92,6 +92,67 @@ diagnostics_kernel(const float* __restrict__ importance, const uint8_t* __restri
     }
 }
 
+// ---- R^2 of the map over a whole context (the statistic of the paper's predictability table) ----
+__global__ void iota_rows_kernel(int32_t* __restrict__ idx, int64_t N) {
+    const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i < N) idx[(size_t)blockIdx.y * N + i] = (int32_t)i;
+}
+
+constexpr int R2_ROWS = 2048;   // tokens per block of the reduction
+
+// grid (ceil(N / R2_ROWS), U), DG_THREADS threads.  acc[u][D + 2] (fp64, zeroed by the caller) receives the
+// per-channel sums of v, then sum ||v||^2 and sum eps.  Thread t owns channel t % D of rows t / D, t / D + rpp, ...
+template <typename T, int D>
+__global__ void __launch_bounds__(DG_THREADS)
+r2_partial_kernel(const T* __restrict__ V, const float* __restrict__ eps, int64_t N, double* __restrict__ acc) {
+    __shared__ double shd[DG_THREADS / 32];
+    __shared__ double chan[DG_THREADS];
+    const int u = blockIdx.y;
+    const int64_t r0 = (int64_t)blockIdx.x * R2_ROWS, r1 = min(N, r0 + (int64_t)R2_ROWS);
+    constexpr int RPP = DG_THREADS / D;            // rows per pass
+    const int c = threadIdx.x % D, rr = threadIdx.x / D;
+    const T* Vu = V + (size_t)u * N * D;
+    double s = 0.0, s2 = 0.0;
+    for (int64_t r = r0 + rr; r < r1; r += RPP) {
+        const double x = (double)to_f32(Vu[(size_t)r * D + c]);
+        s += x;
+        s2 = fma(x, x, s2);
+    }
+    double e = 0.0;
+    for (int64_t r = r0 + threadIdx.x; r < r1; r += DG_THREADS) e += (double)eps[(size_t)u * N + r];
+    chan[threadIdx.x] = s;
+    s2 = block_sum(s2, shd);
+    e = block_sum(e, shd);
+    double* a = acc + (size_t)u * (D + 2);
+    if (threadIdx.x < D) {
+        double t = 0.0;
+#pragma unroll
+        for (int k = 0; k < RPP; ++k) t += chan[threadIdx.x + k * D];
+        atomicAdd(a + threadIdx.x, t);
+    }
+    if (threadIdx.x == 0) { atomicAdd(a + D, s2); atomicAdd(a + D + 1, e); }
+}
+
+// out[u][4] = { R^2, SS_res, SS_tot, N }
+__global__ void r2_finish_kernel(const double* __restrict__ acc, int D, int64_t N, int U, float* __restrict__ out) {
+    const int u = blockIdx.x * blockDim.x + threadIdx.x;
+    if (u >= U) return;
+    const double* a = acc + (size_t)u * (D + 2);
+    double m2 = 0.0;
+    for (int c = 0; c < D; ++c) m2 += a[c] * a[c];
+    const double ss_tot = a[D] - m2 / (double)N, ss_res = a[D + 1];
+    float* o = out + (size_t)u * 4;
+    o[0] = (float)(ss_tot > 0.0 ? 1.0 - ss_res / ss_tot : (ss_res > 0.0 ? -INFINITY : 1.0));
+    o[1] = (float)ss_res;
+    o[2] = (float)ss_tot;
+    o[3] = (float)N;
+}
+
+static size_t r2_ws_bytes(const Dims& dm, int64_t N) {
+    return align256((size_t)dm.U * (size_t)N * sizeof(int32_t)) + align256((size_t)dm.U * (size_t)N * sizeof(float)) +
+           align256((size_t)dm.U * (size_t)(dm.d + 2) * sizeof(double));
+}
+
 }  // namespace vec
 
 extern "C" vector_status vector_diagnostics(const vector_shape* shape, const vector_budget* budget,
@@ -112,4 +173,53 @@ extern "C" vector_status vector_diagnostics(const vector_shape* shape, const vec
 #undef VEC_DIAG
     VEC_LAUNCH_CHECK();
     return VECTOR_OK;
+}
+
+extern "C" size_t vector_r2_global_workspace_bytes(const vector_shape* shape, int64_t N) {
+    using namespace vec;
+    Dims dm;
+    if (check_shape(shape, &dm) != VECTOR_OK || N <= 0) return 0;
+    return r2_ws_bytes(dm, N);
+}
+
+extern "C" vector_status vector_r2_global(const vector_shape* shape, const void* K, const void* V, const void* W,
+                                          int64_t N, float* out, void* ws, size_t ws_bytes, void* stream) {
+    using namespace vec;
+    Dims dm;
+    vector_status rc = check_shape(shape, &dm);
+    if (rc != VECTOR_OK) return rc;
+    if (!K || !V || !W || !out) return VECTOR_ERR_NULL;
+    if (N <= 0 || N > (int64_t(1) << 30)) return VECTOR_ERR_SHAPE;
+    if (!ws || ((uintptr_t)ws & 255) || ws_bytes < r2_ws_bytes(dm, N)) return VECTOR_ERR_WORKSPACE;
+    cudaStream_t st = (cudaStream_t)stream;
+    char* p = (char*)ws;
+    int32_t* idx = (int32_t*)p;  p += align256((size_t)dm.U * (size_t)N * sizeof(int32_t));
+    float* eps = (float*)p;      p += align256((size_t)dm.U * (size_t)N * sizeof(float));
+    double* acc = (double*)p;
+    if (cudaMemsetAsync(acc, 0, (size_t)dm.U * (size_t)(dm.d + 2) * sizeof(double), st) != cudaSuccess) return VECTOR_ERR_CUDA;
+    iota_rows_kernel<<<dim3((unsigned)((N + 255) / 256), dm.U), 256, 0, st>>>(idx, N);
+    VEC_LAUNCH_CHECK();
+    if ((rc = vector_residual(shape, K, V, W, N, idx, N, eps, stream)) != VECTOR_OK) return rc;
+    const dim3 grid((unsigned)((N + R2_ROWS - 1) / R2_ROWS), dm.U);
+#define VEC_R2(T, D) r2_partial_kernel<T, D><<<grid, DG_THREADS, 0, st>>>((const T*)V, eps, N, acc)
+    if (dm.dtype == VECTOR_F32) { if (dm.d == 64) VEC_R2(float, 64); else VEC_R2(float, 128); }
+    else { if (dm.d == 64) VEC_R2(__nv_bfloat16, 64); else VEC_R2(__nv_bfloat16, 128); }
+#undef VEC_R2
+    VEC_LAUNCH_CHECK();
+    r2_finish_kernel<<<(dm.U + 127) / 128, 128, 0, st>>>(acc, dm.d, N, dm.U, out);
+    VEC_LAUNCH_CHECK();
+    return VECTOR_OK;
+}
+
+extern "C" vector_status vector_sync_check(void* stream) {
+    int* addr = vec::kernel_fault_address();
+    if (!addr) return VECTOR_ERR_CUDA;
+    cudaStream_t st = (cudaStream_t)stream;
+    int v = 0;
+    if (cudaMemcpyAsync(&v, addr, sizeof(int), cudaMemcpyDeviceToHost, st) != cudaSuccess) return VECTOR_ERR_CUDA;
+    if (cudaStreamSynchronize(st) != cudaSuccess) return VECTOR_ERR_CUDA;
+    if (v == 0) return VECTOR_OK;
+    if (cudaMemsetAsync(addr, 0, sizeof(int), st) != cudaSuccess || cudaStreamSynchronize(st) != cudaSuccess)
+        return VECTOR_ERR_CUDA;
+    return VECTOR_ERR_TIMEOUT;
 }

@@ -162,6 +162,27 @@ def test_diagnostics_parity(oracle):
         assert 0.0 <= got["E"] <= 1.0 and got["mu_a"] < 0.5          # the approximated tokens are the reconstructable ones
 
 
+@pytest.mark.parametrize("dtype,d,N", [("bf16", 128, 3000), ("fp32", 64, 1111), ("bf16", 128, 2048)])
+def test_r2_global_parity(oracle, dtype, d, N):
+    """R^2 of the calibrated map over every token of the context, per unit, and the stream check after it."""
+    wl = synth.shrink(synth.WORKLOADS[1], N=N, n_kv_heads=2, n_q_heads=8, n_calib=2048, head_dim=d, dtype=dtype)
+    K, V, _q = synth.context(wl, DEV)
+    W = calibrated_maps(wl).to(DEV)
+    sh = shape_of(wl)
+    ws = torch.empty(vec.vector_r2_global_workspace_bytes(sh, wl.N), dtype=torch.uint8, device=DEV)
+    out = torch.full((wl.units, 4), float("nan"), dtype=torch.float32, device=DEV)
+    vec.vector_r2_global(sh, K, V, W, wl.N, out, ws)
+    vec.vector_sync_check()                               # no bounded wait gave up
+    for u in range(wl.units):
+        want = oracle.r2_global(K[u].cpu(), V[u].cpu(), W[u].cpu())
+        got = dict(zip(vec.R2_FIELDS, out[u].cpu().double().tolist()))
+        for name in vec.R2_FIELDS:                        # fp64 sums; the fp32 residuals' rounding is what is left
+            assert got[name] == pytest.approx(want[name], rel=1e-4), (u, name, got[name], want[name])
+        assert got["r2"] < 1.0
+    with pytest.raises(vec.VectorError):                  # too small a workspace is refused before any launch
+        vec.vector_r2_global(sh, K, V, W, wl.N, out, ws[:256])
+
+
 def _selection_inputs(U, N, seed, ties):
     g = torch.Generator().manual_seed(seed)
     s = torch.rand(U, N, generator=g)

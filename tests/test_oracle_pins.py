@@ -150,6 +150,30 @@ def test_calibrate_r2_of_generator(oracle):
     assert 1 - sse / sst == pytest.approx(sig / (sig + 16 * 1.0), abs=0.01)
 
 
+def test_r2_global_against_library_and_closed_forms(oracle):
+    from sklearn.metrics import r2_score
+    rng = np.random.default_rng(31)
+    K, V, Wt = _kv(rng, 700, 16, 16, 0.7)
+    V = V + 3.0                                         # a mean the total sum of squares must remove
+    W = rng.standard_normal((16, 16)) * 0.3
+    r = oracle.r2_global(K, V, W)
+    # the library's variance-weighted multi-output R^2 is the same ratio of sums
+    assert r["r2"] == pytest.approx(r2_score(V, K @ W.T, multioutput="variance_weighted"), abs=1e-12)
+    assert r["n"] == 700
+    # exact map: 1; zero map: 1 - sum||v||^2 / SS_tot, below zero once the mean is not
+    assert oracle.r2_global(K, K @ W.T, W)["r2"] == pytest.approx(1.0, abs=1e-12)
+    z = oracle.r2_global(K, V, np.zeros((16, 16)))
+    assert z["ss_res"] == pytest.approx(np.sum(V * V)) and z["r2"] < 0
+    # a transposed map is a different, worse predictor
+    assert oracle.r2_global(K, K @ W.T, W.T)["r2"] < 0.9
+    # on its own calibration samples the least-squares fit without intercept explains what the generator puts in
+    Kc, Vc, Wc = _kv(rng, 20000, 16, 16, 1.0)
+    sig = np.sum(np.var(Kc @ Wc.T, axis=0))
+    assert oracle.r2_global(Kc, Vc, oracle.calibrate(Kc, Vc, 1e-4))["r2"] == pytest.approx(sig / (sig + 16.0), abs=0.01)
+    # constant values: nothing to explain
+    assert oracle.r2_global(K, np.ones((700, 16)), np.zeros((16, 16)))["r2"] == -np.inf
+
+
 # -------------------------------------------------------------------------- score
 def _brute_raw(Q, K, scale):
     """Full causal attention over all N positions with a library softmax; only
