@@ -15,14 +15,50 @@ namespace vec {
 
 using sel::Layout;
 
-// Blocks of 32 warps (two resident per multiprocessor) for long inputs, of 8 warps (eight resident)
+// Blocks of 32 warps (one resident per multiprocessor, masks and list in up to 200 KB) for inputs beyond a
+// quarter of a million elements, of 16 warps (two resident) for medium ones and of 8 warps (four resident)
 // for short ones, where what a block costs is its fixed sequence of barriers rather than its passes.
-constexpr int SEL_SHORT = 4096;
-constexpr size_t SEL_SMEM_LONG = 100 * 1024, SEL_SMEM_SHORT = 18 * 1024;
+constexpr int SEL_SHORT = 8192, SEL_MANY = 32768, SEL_LONG = 262144;
+constexpr size_t SEL_SMEM_LONG = 200 * 1024, SEL_SMEM_MID = 92 * 1024, SEL_SMEM_SHORT = 36 * 1024;
+#define VEC_SEL_BOUNDS(NW) __launch_bounds__(32 * NW, NW == 32 ? 1 : NW == 16 ? 2 : 4)
+
+// The general selection (select_emit) as functions of their own: the kernels run the lean path inline and
+// come here only when it gives up, so its registers are not theirs to carry.
+template <int NW>
+__device__ __noinline__ void pool_select_general(const float* __restrict__ s, int n, int n_pool, int32_t* __restrict__ out,
+                                                 sel::Scratch& S, const Layout& L, uint32_t* dyn) {
+    sel::select_emit<false, NW, true>(s, n, n_pool, true, S, L, dyn, [&](int i, bool chosen, int pos) { if (chosen) out[pos] = i; });
+}
+
+struct PoolOut {
+    int32_t* out;
+    __device__ __forceinline__ int32_t* list() const { return out; }
+};
+
+struct TruncateOut {
+    const int32_t* pool;
+    uint8_t* tr;
+    int32_t* ro;
+    int32_t* ao;
+    int64_t N;
+    __device__ __forceinline__ int fetch(int p) const { return pool[p]; }
+    __device__ __forceinline__ void put(int, int token, bool is_apx, int pos) const {
+        if ((uint64_t)(int64_t)token >= (uint64_t)N) return;          // a pool entry outside the unit is dropped
+        if (is_apx) { ao[pos] = token; tr[token] = 1; }
+        else        { ro[pos] = token; tr[token] = 2; }
+    }
+    __device__ __forceinline__ void operator()(int p, bool is_apx, int pos) const { put(p, pool[p], is_apx, pos); }
+};
+
+template <int NW>
+__device__ __noinline__ void truncate_general(const float* __restrict__ e, int n_pool, int n_apx, const TruncateOut& emit,
+                                              sel::Scratch& S, const Layout& L, uint32_t* dyn) {
+    sel::select_emit<true, NW, false>(e, n_pool, n_apx, n_apx > 0, S, L, dyn, emit);
+}
 
 // Step 1.  grid (U), 32 NW threads, L.bytes() of dynamic shared memory.
 template <int NW>
-__global__ void __launch_bounds__(32 * NW, NW == 32 ? 2 : 8)
+__global__ void VEC_SEL_BOUNDS(NW)
 pool_select_kernel(const float* __restrict__ scores, int64_t N, int n_pool, int32_t* __restrict__ pool_idx, const Layout L) {
     __shared__ sel::Scratch S;
     extern __shared__ __align__(16) uint32_t sel_dyn[];
@@ -33,13 +69,14 @@ pool_select_kernel(const float* __restrict__ scores, int64_t N, int n_pool, int3
     const float* s = scores + (size_t)u * N;
     int32_t* out = pool_idx + (size_t)u * n_pool;
     if (n_pool <= 0) return;
-    sel::select_emit<false, NW, true>(s, n, n_pool, true, S, L, sel_dyn, [&](int i, bool chosen, int pos) { if (chosen) out[pos] = i; });
+    if (L.keyed && sel::select_lean<false, NW, true>(s, n, n_pool, S, L, sel_dyn, PoolOut{out})) return;
+    pool_select_general<NW>(s, n, n_pool, out, S, L, sel_dyn);
 }
 
 // Step 3.  grid (U), 32 NW threads, L.bytes() of dynamic shared memory (the residuals' images are
-// staged there when they fit).
+// staged there when the lean path cannot run and they fit).
 template <int NW>
-__global__ void __launch_bounds__(32 * NW, NW == 32 ? 2 : 8)
+__global__ void VEC_SEL_BOUNDS(NW)
 truncate_kernel(const float* __restrict__ eps, const int32_t* __restrict__ pool_idx, int64_t N, int n_pool,
                 int n_apx, uint8_t* __restrict__ tier, int32_t* __restrict__ ret_idx,
                 int32_t* __restrict__ apx_idx, const Layout L) {
@@ -47,11 +84,7 @@ truncate_kernel(const float* __restrict__ eps, const int32_t* __restrict__ pool_
     extern __shared__ __align__(16) uint32_t sel_dyn[];
     const int u = blockIdx.x;
     const float* e = eps + (size_t)u * n_pool;
-    const int32_t* pool = pool_idx + (size_t)u * n_pool;
     uint8_t* tr = tier + (size_t)u * N;
-    const int n_ret = n_pool - n_apx;
-    int32_t* ro = ret_idx + (size_t)u * n_ret;
-    int32_t* ao = apx_idx + (size_t)u * n_apx;
     if ((N & 15) == 0) {
         for (int64_t i = threadIdx.x; i < N / 16; i += 32 * NW) reinterpret_cast<uint4*>(tr)[i] = make_uint4(0, 0, 0, 0);
     } else {
@@ -61,12 +94,10 @@ truncate_kernel(const float* __restrict__ eps, const int32_t* __restrict__ pool_
     // kernels before this one (a no-op unless launched as a programmatic dependent)
     asm volatile("griddepcontrol.wait;\n" ::: "memory");
     __syncthreads();
-    sel::select_emit<true, NW, false>(e, n_pool, n_apx, n_apx > 0, S, L, sel_dyn, [&](int p, bool is_apx, int pos) {
-        const int32_t token = pool[p];
-        if ((uint64_t)(int64_t)token >= (uint64_t)N) return;          // a pool entry outside the unit is dropped
-        if (is_apx) { ao[pos] = token; tr[token] = 1; }
-        else        { ro[pos] = token; tr[token] = 2; }
-    });
+    const int n_ret = n_pool - n_apx;
+    const TruncateOut emit = {pool_idx + (size_t)u * n_pool, tr, ret_idx + (size_t)u * n_ret, apx_idx + (size_t)u * n_apx, N};
+    if (L.keyed && n_apx > 0 && sel::select_lean<true, NW, false>(e, n_pool, n_apx, S, L, sel_dyn, emit)) return;
+    truncate_general<NW>(e, n_pool, n_apx, emit, S, L, sel_dyn);
 }
 
 // Step 2 on CUDA cores.  grid (ceil(n_idx / 64), U), 256 threads; W^T staged in
@@ -196,11 +227,28 @@ static vector_status select_kernels_setup() {
     static PerDeviceOnce once;
     if (!once.first()) return VECTOR_OK;
     cudaError_t e = cudaFuncSetAttribute(pool_select_kernel<32>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SEL_SMEM_LONG);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(pool_select_kernel<16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SEL_SMEM_MID);
     if (e == cudaSuccess) e = cudaFuncSetAttribute(pool_select_kernel<8>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SEL_SMEM_SHORT);
     if (e == cudaSuccess) e = cudaFuncSetAttribute(truncate_kernel<32>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SEL_SMEM_LONG);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(truncate_kernel<16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SEL_SMEM_MID);
     if (e == cudaSuccess) e = cudaFuncSetAttribute(truncate_kernel<8>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SEL_SMEM_SHORT);
     if (e != cudaSuccess) { once.undo(); VEC_CUDA_CHECK(e); }
     return VECTOR_OK;
+}
+
+// Block size, shared-memory budget and smallest useful list of U selections over n elements each.  Short
+// inputs take the small blocks; so do medium ones when there are units enough to fill the small blocks'
+// slots twice over (the phases after the two passes are latency, which more resident blocks hide).
+struct SelPlan { int nw; Layout L; };
+static SelPlan plan_selection(int64_t n, int U) {
+    SelPlan p;
+    const bool small = n < SEL_SHORT || (n < SEL_MANY && U >= 2 * 4 * sm_count());
+    const size_t budget = small ? SEL_SMEM_SHORT : n < SEL_LONG ? SEL_SMEM_MID : SEL_SMEM_LONG;
+    const int min_cand = small ? 1024 : 2048;
+    p.nw = small ? 8 : n < SEL_LONG ? 16 : 32;
+    p.L = sel::plan_layout(n, false, budget, min_cand, p.nw);
+    if (!p.L.keyed) p.L = sel::plan_layout(n, true, budget, min_cand, p.nw);       // the general path stages the images
+    return p;
 }
 
 static vector_status launch_pool_select(const Dims& dm, const vector_budget* budget, const float* scores, int32_t* pool,
@@ -208,13 +256,11 @@ static vector_status launch_pool_select(const Dims& dm, const vector_budget* bud
     vector_status rc = select_kernels_setup();
     if (rc != VECTOR_OK) return rc;
     const int64_t n = budget->n_tokens;
-    if (n <= SEL_SHORT) {
-        const Layout L = sel::plan_layout(n, false, SEL_SMEM_SHORT, 1024);
-        pool_select_kernel<8><<<dm.U, 256, L.bytes(), st>>>(scores, n, (int)budget->n_pool, pool, L);
-    } else {
-        const Layout L = sel::plan_layout(n, false, SEL_SMEM_LONG, 2048);
-        pool_select_kernel<32><<<dm.U, 1024, L.bytes(), st>>>(scores, n, (int)budget->n_pool, pool, L);
-    }
+    const SelPlan p = plan_selection(n, dm.U);
+    const Layout L = p.L;
+    if (p.nw == 8) pool_select_kernel<8><<<dm.U, 256, L.bytes(), st>>>(scores, n, (int)budget->n_pool, pool, L);
+    else if (p.nw == 16) pool_select_kernel<16><<<dm.U, 512, L.bytes(), st>>>(scores, n, (int)budget->n_pool, pool, L);
+    else pool_select_kernel<32><<<dm.U, 1024, L.bytes(), st>>>(scores, n, (int)budget->n_pool, pool, L);
     VEC_LAUNCH_CHECK();
     return VECTOR_OK;
 }
@@ -224,19 +270,17 @@ static vector_status launch_truncate(const Dims& dm, const vector_budget* budget
                                      bool dependent = false) {
     vector_status rc = select_kernels_setup();
     if (rc != VECTOR_OK) return rc;
-    const int64_t n = budget->n_pool;
+    const SelPlan p = plan_selection(budget->n_pool, dm.U);
+    const Layout L = p.L;
     // dependent: may start (and clear the tier map) while the kernel before it in the stream drains
-    if (n <= SEL_SHORT) {
-        const Layout L = sel::plan_layout(n, true, SEL_SMEM_SHORT, 1024);
-        VEC_CUDA_CHECK(launch_maybe_dependent(dependent, truncate_kernel<8>, dim3(dm.U), dim3(256), L.bytes(), st, eps, pool,
-                                              (int64_t)budget->n_tokens, (int)budget->n_pool, (int)budget->n_apx, tier, ret_idx,
-                                              apx_idx, L));
-    } else {
-        const Layout L = sel::plan_layout(n, true, SEL_SMEM_LONG, 2048);
-        VEC_CUDA_CHECK(launch_maybe_dependent(dependent, truncate_kernel<32>, dim3(dm.U), dim3(1024), L.bytes(), st, eps, pool,
-                                              (int64_t)budget->n_tokens, (int)budget->n_pool, (int)budget->n_apx, tier, ret_idx,
-                                              apx_idx, L));
-    }
+#define VEC_TRUNC(NW)                                                                                                   \
+    VEC_CUDA_CHECK(launch_maybe_dependent(dependent, truncate_kernel<NW>, dim3(dm.U), dim3(32 * NW), L.bytes(), st, eps, \
+                                          pool, (int64_t)budget->n_tokens, (int)budget->n_pool, (int)budget->n_apx, tier, \
+                                          ret_idx, apx_idx, L))
+    if (p.nw == 8) VEC_TRUNC(8);
+    else if (p.nw == 16) VEC_TRUNC(16);
+    else VEC_TRUNC(32);
+#undef VEC_TRUNC
     return VECTOR_OK;
 }
 
