@@ -277,12 +277,13 @@ static vector_status launch_decode_bf16_d128(const Dims& dm, const void* q, cons
     const int apply_w = mode == 1 ? 0 : 1;
     const int cw = mode == 1 ? dpt::CONSUMERS : dbf::CONSUMER_WARPS;      // records a block leaves per unit
     const T* Wp = (const T*)W;
-    if (out_dtype == VECTOR_F32)
-        VEC_CUDA_CHECK(launch_maybe_dependent(true, dbf::decode_merge_bf16_d128<float>, dim3(dm.U), dim3(128 * dm.g), 0, st, rec,
-                                              Wp, dm.LH, dm.g, pl, apply_w, cw, (float*)out));
-    else
-        VEC_CUDA_CHECK(launch_maybe_dependent(true, dbf::decode_merge_bf16_d128<T>, dim3(dm.U), dim3(128 * dm.g), 0, st, rec, Wp,
-                                              dm.LH, dm.g, pl, apply_w, cw, (T*)out));
+    // blocks of 128 g threads; up to four heads leave the merge 128 registers a thread
+#define VEC_MERGE(TO, MAXT)                                                                                                  \
+    VEC_CUDA_CHECK(launch_maybe_dependent(true, dbf::decode_merge_bf16_d128<TO, MAXT>, dim3(dm.U), dim3(128 * dm.g), 0, st, rec, \
+                                          Wp, dm.LH, dm.g, pl, apply_w, cw, (TO*)out))
+    if (out_dtype == VECTOR_F32) { if (dm.g <= 4) VEC_MERGE(float, 512); else VEC_MERGE(float, 1024); }
+    else { if (dm.g <= 4) VEC_MERGE(T, 512); else VEC_MERGE(T, 1024); }
+#undef VEC_MERGE
     return VECTOR_OK;
 }
 

@@ -513,22 +513,35 @@ decode_stream_bf16_d128(const __nv_bfloat16* __restrict__ q, const __grid_consta
 // Combines the records of a unit, applies the unit's map to the p-weighted key sum and normalises:
 //   o = (sum_j f_j s_j acc_v_j + W sum_j f_j acc_k_j) / sum_j f_j l_j,   f_j = exp(m_j - max m).
 // Every load of a phase is independent of the others, so a phase costs one memory latency.
-template <typename TO>
-__global__ void __launch_bounds__(1024)
+// The product W (sum f acc_k) runs on warp-level MMAs, M = 128 output channels (warp w takes rows 16 w ..),
+// N = the unit's g query heads (padded to 8), K = 128: the A fragments are read straight from the map in
+// global memory, 16 bytes a load -- thread (row r, quarter t) of a warp holds columns 8 (t + 4 jj) .. + 7 of
+// rows r and r + 8, and the k slots of MMA step 2 jj + h stand for columns 8 (t + 4 jj) + 4 h .. + 3, which the
+// B fragments follow; the key sum enters as bf16 hi + lo (sixteen mantissa bits), the map's elements are bf16
+// as stored.
+template <typename TO, int MAXT>
+__global__ void __launch_bounds__(MAXT, 1024 / MAXT)
 decode_merge_bf16_d128(const float* __restrict__ partial, const __nv_bfloat16* __restrict__ W, int LH, int g,
                        Plan pl, int apply_w, int cw, TO* __restrict__ out) {
-    __shared__ uint32_t Ws[128 * 65];          // W rows as bf16 pairs, row stride 65 words (conflict-free)
-    __shared__ __align__(8) float aks[8][128];
+    __shared__ __align__(16) __nv_bfloat16 akh[8][128], akl[8][128];      // key sums per head, hi and lo halves
+    __shared__ float pw[8][128];               // W times the key sum
     __shared__ float fv[8][48], fk[8][48];     // per head, per record: factor for the value part / the key part
     __shared__ float Ls[8];
     const int u = blockIdx.x, tid = threadIdx.x, a = tid >> 7, c = tid & 127, lane = tid & 31;
-    const int nthr = blockDim.x;
-    // W tile into shared memory (overlaps the tail of the streaming kernel): 2048 16-byte pieces
-    const uint4* Wu = reinterpret_cast<const uint4*>(W + (size_t)(u % LH) * 128 * 128);
-    for (int i = tid; i < (apply_w ? 2048 : 0); i += nthr) {
-        const uint4 v = Wu[i];
-        uint32_t* dst = Ws + (i >> 4) * 65 + (i & 15) * 4;      // 16 pieces per 256-byte row
-        dst[0] = v.x; dst[1] = v.y; dst[2] = v.z; dst[3] = v.w;
+    const int wid = tid >> 5, nwarps = blockDim.x >> 5, row = lane >> 2, quarter = lane & 3;
+    // A fragments of 16 rows of W (the maps of a layer stay in L2: every sequence of the batch reads them)
+    const uint4* Wu = reinterpret_cast<const uint4*>(W + (size_t)(u % LH) * 128 * 128);       // 16 pieces per 256-byte row
+    uint4 A[8];
+    auto load_rows = [&](int mt) {
+#pragma unroll
+        for (int jj = 0; jj < 4; ++jj) {
+            A[2 * jj + 0] = Wu[(16 * mt + row) * 16 + quarter + 4 * jj];
+            A[2 * jj + 1] = Wu[(16 * mt + row + 8) * 16 + quarter + 4 * jj];
+        }
+    };
+    for (int i = tid; i < (8 - g) * 128; i += blockDim.x) {       // columns of B beyond the unit's heads
+        akh[g + i / 128][i % 128] = __float2bfloat16_rn(0.f);
+        akl[g + i / 128][i % 128] = __float2bfloat16_rn(0.f);
     }
     // everything above reads only W, which the streaming kernel does not write; its records from here on
     asm volatile("griddepcontrol.wait;\n" ::: "memory");
@@ -593,17 +606,32 @@ decode_merge_bf16_d128(const float* __restrict__ partial, const __nv_bfloat16* _
         store_out(out + ((size_t)u * g + a) * 128 + c, (av + ak) / Ls[a]);
         return;
     }
-    aks[a][c] = ak;
-    __syncthreads();
-    float p0 = 0.f, p1 = 0.f;
-#pragma unroll 8
-    for (int c2 = 0; c2 < 64; ++c2) {
-        const uint32_t w2 = Ws[c * 65 + c2];
-        const float2 k2 = *reinterpret_cast<const float2*>(&aks[a][2 * c2]);
-        p0 = fmaf(__uint_as_float(w2 << 16), k2.x, p0);
-        p1 = fmaf(__uint_as_float(w2 & 0xffff0000u), k2.y, p1);
+    {
+        const __nv_bfloat16 hi = __float2bfloat16_rn(ak);
+        akh[a][c] = hi;
+        akl[a][c] = __float2bfloat16_rn(ak - __bfloat162float(hi));
     }
-    store_out(out + ((size_t)u * g + a) * 128 + c, (av + p0 + p1) / Ls[a]);
+    __syncthreads();
+    for (int mt = wid; mt < 8; mt += nwarps) {
+        load_rows(mt);
+        float d[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+        for (int jj = 0; jj < 4; ++jj) {
+            const uint4 r0 = A[2 * jj], r1 = A[2 * jj + 1];
+            const int col = 8 * (quarter + 4 * jj);
+            const uint4 bh = *reinterpret_cast<const uint4*>(&akh[row][col]);      // B column = head `row`
+            const uint4 bl = *reinterpret_cast<const uint4*>(&akl[row][col]);
+            mma_16(d, r0.x, r1.x, r0.y, r1.y, bh.x, bh.y);
+            mma_16(d, r0.x, r1.x, r0.y, r1.y, bl.x, bl.y);
+            mma_16(d, r0.z, r1.z, r0.w, r1.w, bh.z, bh.w);
+            mma_16(d, r0.z, r1.z, r0.w, r1.w, bl.z, bl.w);
+        }
+        // d[0], d[1]: row `row`, heads 2 quarter and 2 quarter + 1; d[2], d[3]: row `row` + 8
+        if (2 * quarter < g) { pw[2 * quarter][16 * mt + row] = d[0]; pw[2 * quarter][16 * mt + row + 8] = d[2]; }
+        if (2 * quarter + 1 < g) { pw[2 * quarter + 1][16 * mt + row] = d[1]; pw[2 * quarter + 1][16 * mt + row + 8] = d[3]; }
+    }
+    __syncthreads();
+    store_out(out + ((size_t)u * g + a) * 128 + c, (av + pw[a][c]) / Ls[a]);
 }
 
 }  // namespace dbf
