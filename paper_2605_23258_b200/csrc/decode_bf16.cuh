@@ -520,7 +520,7 @@ decode_stream_bf16_d128(const __nv_bfloat16* __restrict__ q, const __grid_consta
 // B fragments follow; the key sum enters as bf16 hi + lo (sixteen mantissa bits), the map's elements are bf16
 // as stored.
 template <typename TO, int MAXT>
-__global__ void __launch_bounds__(MAXT, 1024 / MAXT)
+__global__ void __launch_bounds__(MAXT, MAXT == 512 ? 3 : 1)
 decode_merge_bf16_d128(const float* __restrict__ partial, const __nv_bfloat16* __restrict__ W, int LH, int g,
                        Plan pl, int apply_w, int cw, TO* __restrict__ out) {
     __shared__ __align__(16) __nv_bfloat16 akh[8][128], akl[8][128];      // key sums per head, hi and lo halves
@@ -548,11 +548,13 @@ decode_merge_bf16_d128(const float* __restrict__ partial, const __nv_bfloat16* _
     const int first = block_of_tile((long long)u * pl.n_tiles, pl);
     const int n_rec = (block_of_tile((long long)(u + 1) * pl.n_tiles - 1, pl) - first + 1) * cw;   // <= 36; cw records per block
     const float* base = partial + (size_t)u * pl.s_max * cw * g * REC;
-    // The first twelve records' sums are requested before the headers are looked at, so that the
-    // two loads share one memory latency (a unit has at most a dozen records unless it is very long).
-    float rv[12], rk[12];
+    // The first six records' sums are requested before the headers are looked at, so that the two loads
+    // share one memory latency (a unit lies in one or two blocks of the streaming kernel, three records
+    // each, unless it is very long).
+    constexpr int NPRE = 6;
+    float rv[NPRE], rk[NPRE];
 #pragma unroll
-    for (int k = 0; k < 12; ++k) {
+    for (int k = 0; k < NPRE; ++k) {
         const int j = min(k, n_rec - 1);
         const float* r = base + ((size_t)j * g + a) * REC + 4;
         rv[k] = r[c];
@@ -584,10 +586,10 @@ decode_merge_bf16_d128(const float* __restrict__ partial, const __nv_bfloat16* _
     }
     __syncthreads();
     float av = 0.f, ak = 0.f;
-    for (int j0 = 0; j0 < n_rec; j0 += 12) {
+    for (int j0 = 0; j0 < n_rec; j0 += NPRE) {
         if (j0 > 0) {
 #pragma unroll
-            for (int k = 0; k < 12; ++k) {
+            for (int k = 0; k < NPRE; ++k) {
                 const int j = min(j0 + k, n_rec - 1);
                 const float* r = base + ((size_t)j * g + a) * REC + 4;
                 rv[k] = r[c];
@@ -595,7 +597,7 @@ decode_merge_bf16_d128(const float* __restrict__ partial, const __nv_bfloat16* _
             }
         }
 #pragma unroll
-        for (int k = 0; k < 12; ++k) {
+        for (int k = 0; k < NPRE; ++k) {
             if (j0 + k < n_rec) {
                 av = fmaf(fv[a][j0 + k], rv[k], av);
                 ak = fmaf(fk[a][j0 + k], rk[k], ak);
