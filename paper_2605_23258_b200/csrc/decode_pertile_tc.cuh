@@ -5,8 +5,9 @@
 // is rebuilt as W k).  For every tile of 128 key-only keys the reconstructed values are
 // materialised as  V^T = W K_tile^T  (128 dims x 128 keys x 128) by tcgen05.mma with the accumulator
 // in tensor memory -- W and K are bf16 data, so the products are exact -- brought back to shared
-// memory as a bf16 pair hi + lo (sixteen mantissa bits) over the keys they came from, and then
-// weighted exactly like stored values.
+// memory as fp16 (eleven mantissa bits: a reconstructed value of size 25 is off by at most 0.006, a
+// bf16 rounding would cost four times that) over the keys they came from, and then weighted like
+// stored values, with the probabilities as an fp16 pair hi + lo.
 //
 // The mixed cache is streamed once, as in the factored kernel: 32 KB tiles (64 retained keys + their
 // 64 values, or 128 key-only keys) dealt in equal contiguous ranges to one persistent block per
@@ -14,12 +15,12 @@
 //   warps 0-1  consumers: tile i belongs to warp i % 2.  Scores S = Q K^T with warp-level MMAs (the g
 //              query heads padded to the MMA rows), online softmax, O += P V with P as bf16 hi + lo.
 //              For a key-only tile V is the reconstructed tile: the warp says when it has read the
-//              keys for the last time, waits for the conversion, and adds P V_hi + P_hi V_lo
+//              keys for the last time, waits for the conversion, and adds P V
 //   warp  2    producer: TMA loads of the tiles into four 32 KB slots
 //   warp  3    MMA issuer, owner of tensor memory; TMA-loads the unit's W when the range enters a unit
 //   warps 4-7  conversion: thread = output dim (its TMEM lane).  Per key-only tile: reads its row of
-//              V^T from tensor memory, splits it into bf16 hi and lo, and writes hi over the tile's keys
-//              (the slot is a [128 dims][128 keys] tile from then on) and lo into the consumer's side buffer
+//              V^T from tensor memory and writes it as fp16 over the tile's keys (the slot is a
+//              [128 dims][128 keys] tile from then on)
 // Per unit every consumer warp leaves one partial record (m, l, sum p v + sum p (W k)); the merge
 // kernel combines the records without applying W.
 // All hand-offs are mbarriers; every wait is bounded and records a fault code.
@@ -44,8 +45,7 @@ constexpr int SLOTS = 4;                     // a multiple of CONSUMERS: a slot 
 constexpr int SLOT_BYTES = 32768;
 constexpr int HALF_BYTES = 16384;
 constexpr int W_BYTES = 32768;
-constexpr int LO_BYTES = 32768;              // low halves of one reconstructed tile: [128 dims][128 keys] bf16
-constexpr int SMEM_BYTES = SLOTS * SLOT_BYTES + W_BYTES + CONSUMERS * LO_BYTES + 1024;
+constexpr int SMEM_BYTES = SLOTS * SLOT_BYTES + W_BYTES + 1024;
 constexpr int NB = 3;                        // V^T accumulators in tensor memory (128 columns each)
 constexpr int TMEM_COLS = 512;
 constexpr int THREADS = 256;
@@ -62,8 +62,7 @@ struct Sync {
     uint64_t full[SLOTS], empty[SLOTS];
     uint64_t vhat_full[NB], vhat_empty[NB];
     uint64_t keys_read[SLOTS];           // the consumer has formed its scores: the slot's keys may be overwritten
-    uint64_t vt_ready[SLOTS];            // the slot holds V^T hi, the consumer's side buffer V^T lo
-    uint64_t lo_free[CONSUMERS];         // the consumer has finished with its side buffer
+    uint64_t vt_ready[SLOTS];            // the slot holds V^T
     uint64_t w_full, w_empty;
     uint32_t tmem_base;
 };
@@ -77,7 +76,6 @@ decode_stream_pertile_tc(const __nv_bfloat16* __restrict__ q, const __grid_const
     __shared__ Sync sy;
     unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     unsigned char* Ws = smem + SLOTS * SLOT_BYTES;
-    unsigned char* Lo = smem + SLOTS * SLOT_BYTES + W_BYTES;                            // [consumer][128 dims][128 keys] bf16
     const int b = blockIdx.x;
     const int tid = threadIdx.x, lane = tid & 31, wq = tid >> 5;
     const long long gt_lo = dbf::tile_begin(b, pl), gt_hi = dbf::tile_begin(b + 1, pl);
@@ -94,8 +92,6 @@ decode_stream_pertile_tc(const __nv_bfloat16* __restrict__ q, const __grid_const
         for (int k = 0; k < NB; ++k) { tma::mbar_init(&sy.vhat_full[k], 1); tma::mbar_init(&sy.vhat_empty[k], RECON_WARPS); }
 #pragma unroll
         for (int s = 0; s < SLOTS; ++s) { tma::mbar_init(&sy.keys_read[s], 1); tma::mbar_init(&sy.vt_ready[s], RECON_WARPS); }
-#pragma unroll
-        for (int w = 0; w < CONSUMERS; ++w) tma::mbar_init(&sy.lo_free[w], 1);
         tma::mbar_init(&sy.w_full, 1);
         tma::mbar_init(&sy.w_empty, 1);
         tma::mbar_fence_init();
@@ -181,36 +177,29 @@ decode_stream_pertile_tc(const __nv_bfloat16* __restrict__ q, const __grid_const
         const int quarter = wq & 3, c = quarter * 32 + lane;          // this thread's output dim = its TMEM lane = its row of V^T
         const uint32_t lane_addr = sy.tmem_base + ((uint32_t)(quarter * 32) << 16);
         const uint32_t row_off = (uint32_t)c * 128u;                   // rows of 128 bytes, 16-byte chunk index XOR (row & 7)
-        uint32_t j = 0, kcount[SLOTS] = {0u, 0u, 0u, 0u}, lcount[CONSUMERS] = {0u, 0u};
+        uint32_t j = 0, kcount[SLOTS] = {};
         bool ok = n_my > 0;
         int t = n_my > 0 ? (int)(gt_lo - (long long)u0 * pl.n_tiles) : 0;
         for (int i = 0; i < n_my && ok; ++i) {
             if (t >= pl.n_rt) {
-                const int w = i % CONSUMERS, s = i % SLOTS;
+                const int s = i % SLOTS;
                 const uint32_t vb = j % NB, use = j / NB;
-                // the MMA has read the keys and left V^T; the consumer has formed its scores; its side buffer is free
+                // the MMA has read the keys and left V^T; the consumer has formed its scores
                 if (!tma::mbar_wait_warp(&sy.vhat_full[vb], use & 1, fault, 72)) { ok = false; break; }
                 if (!tma::mbar_wait_warp(&sy.keys_read[s], kcount[s] & 1, fault, 71)) { ok = false; break; }
-                if (lcount[w] > 0 && !tma::mbar_wait_warp(&sy.lo_free[w], (lcount[w] - 1) & 1, fault, 73)) { ok = false; break; }
                 tc::fence_after_sync();
                 const uint32_t hi_base = tma::smem_u32(smem + s * SLOT_BYTES) + row_off;
-                const uint32_t lo_base = tma::smem_u32(Lo + w * LO_BYTES) + row_off;
                 const uint32_t taddr = lane_addr + vb * 128;
                 // 16 keys = two 16-byte chunks of this row at a time, in a loop that stays rolled
                 auto split16 = [&](const uint32_t (&v16)[16], int chunk0) {
-                    uint32_t hi[8], lo[8];
+                    uint32_t hi[8];
 #pragma unroll
-                    for (int e = 0; e < 8; ++e) {
-                        const float x0 = __uint_as_float(v16[2 * e]), x1 = __uint_as_float(v16[2 * e + 1]);
-                        hi[e] = dbf::pack_bf16(x0, x1);
-                        lo[e] = dbf::pack_bf16(x0 - __uint_as_float(hi[e] << 16), x1 - __uint_as_float(hi[e] & 0xffff0000u));
-                    }
+                    for (int e = 0; e < 8; ++e) hi[e] = dbf::pack_f16(__uint_as_float(v16[2 * e]), __uint_as_float(v16[2 * e + 1]));
 #pragma unroll
                     for (int h = 0; h < 2; ++h) {
                         const int chunk = chunk0 + h;                  // keys 8 chunk .. 8 chunk + 7: box chunk / 8, chunk % 8 inside the row
                         const uint32_t off = (uint32_t)(chunk >> 3) * HALF_BYTES + (uint32_t)(((chunk & 7) ^ (c & 7)) << 4);
                         asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};\n" ::"r"(hi_base + off), "r"(hi[4 * h]), "r"(hi[4 * h + 1]), "r"(hi[4 * h + 2]), "r"(hi[4 * h + 3]) : "memory");
-                        asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};\n" ::"r"(lo_base + off), "r"(lo[4 * h]), "r"(lo[4 * h + 1]), "r"(lo[4 * h + 2]), "r"(lo[4 * h + 3]) : "memory");
                     }
                 };
                 uint32_t ra[16], rb[16];
@@ -234,7 +223,6 @@ decode_stream_pertile_tc(const __nv_bfloat16* __restrict__ q, const __grid_const
                 }
                 ++j;
                 ++kcount[s];
-                ++lcount[w];
             }
             if (++t == pl.n_tiles) t = 0;
         }
@@ -310,26 +298,21 @@ decode_stream_pertile_tc(const __nv_bfloat16* __restrict__ q, const __grid_const
                 }
             }
         };
-        // The same for 64 keys of a reconstructed tile: V^T hi at hibase, V^T lo at lobase, both [128 dims][keys]
-        // in boxes of 128 rows; `kc0` = first 16-byte chunk of these keys inside the row (0 or 8 -> box 0 or 1).
-        auto weigh64_rebuilt = [&](uint32_t hibase, uint32_t lobase, const float (&sc)[8][2]) {
+        // The same for 64 keys of a reconstructed tile: V^T as fp16 at vbase, [128 dims][keys] in boxes of 128
+        // rows; the probabilities as fp16 hi (MMA rows 0-7) + lo (rows 8-15).
+        auto weigh64_rebuilt = [&](uint32_t vbase, const float (&sc)[8][2]) {
 #pragma unroll
             for (int kk = 0; kk < 4; ++kk) {
                 const float p00 = sc[2 * kk][0], p01 = sc[2 * kk][1], p10 = sc[2 * kk + 1][0], p11 = sc[2 * kk + 1][1];
-                const float h00 = __bfloat162float(__float2bfloat16_rn(p00)), h01 = __bfloat162float(__float2bfloat16_rn(p01));
-                const float h10 = __bfloat162float(__float2bfloat16_rn(p10)), h11 = __bfloat162float(__float2bfloat16_rn(p11));
-                const uint32_t a0 = dbf::pack_bf16(h00, h01), a2 = dbf::pack_bf16(h10, h11);
-                const uint32_t a1 = dbf::pack_bf16(p00 - h00, p01 - h01), a3 = dbf::pack_bf16(p10 - h10, p11 - h11);
+                const uint32_t a0 = dbf::pack_f16(p00, p01), a2 = dbf::pack_f16(p10, p11);
+                const uint32_t a1 = dbf::pack_f16(p00 - dbf::f16_lo(a0), p01 - dbf::f16_hi(a0));
+                const uint32_t a3 = dbf::pack_f16(p10 - dbf::f16_lo(a2), p11 - dbf::f16_hi(a2));
 #pragma unroll
                 for (int jj = 0; jj < 8; ++jj) {        // 16 dims per ldmatrix: rows 16 jj .. of V^T, keys 16 kk .. along the row
                     uint32_t b0, b1, b2, b3;
-                    const uint32_t off = jj * 16 * 128 + qk_row + ((((2 * kk) & 7) << 4) ^ qk_x);
-                    dbf::ldsm_x4(hibase + off, b0, b1, b2, b3);
-                    dbf::mma_16(acc[2 * jj], a0, a1, a2, a3, b0, b1);
-                    dbf::mma_16(acc[2 * jj + 1], a0, a1, a2, a3, b2, b3);
-                    dbf::ldsm_x4(lobase + off, b0, b1, b2, b3);
-                    dbf::mma_16(acc[2 * jj], a0, 0u, a2, 0u, b0, b1);          // P_hi V_lo: the product of the two remainders is dropped
-                    dbf::mma_16(acc[2 * jj + 1], a0, 0u, a2, 0u, b2, b3);
+                    dbf::ldsm_x4(vbase + jj * 16 * 128 + qk_row + ((((2 * kk) & 7) << 4) ^ qk_x), b0, b1, b2, b3);
+                    dbf::mma_16_f16(acc[2 * jj], a0, a1, a2, a3, b0, b1);
+                    dbf::mma_16_f16(acc[2 * jj + 1], a0, a1, a2, a3, b2, b3);
                 }
             }
         };
@@ -433,17 +416,16 @@ decode_stream_pertile_tc(const __nv_bfloat16* __restrict__ q, const __grid_const
 #pragma unroll
                         for (int n = 0; n < 16; ++n) { acc[n][0] *= alpha; acc[n][1] *= alpha; acc[n][2] *= alpha; acc[n][3] *= alpha; }
                     }
-                    // the reconstructed values: hi where the keys were, lo in this warp's side buffer
+                    // the reconstructed values, where the keys were
                     const int sl = (i / CONSUMERS) % (SLOTS / CONSUMERS);
                     ok = tma::mbar_wait_warp(&sy.vt_ready[s], vcount[sl] & 1, fault, 68);
                     ++vcount[sl];
                     if (ok) {
-                        const uint32_t lob = tma::smem_u32(Lo + wq * LO_BYTES);
-                        weigh64_rebuilt(base, lob, sa);
-                        weigh64_rebuilt(base + HALF_BYTES, lob + HALF_BYTES, sb);
+                        weigh64_rebuilt(base, sa);
+                        weigh64_rebuilt(base + HALF_BYTES, sb);
                     }
                     __syncwarp();
-                    if (lane == 0) { tma::mbar_arrive(&sy.lo_free[wq]); tma::mbar_arrive(&sy.empty[s]); }
+                    if (lane == 0) tma::mbar_arrive(&sy.empty[s]);
                 }
             }
             flush(u);
