@@ -14,6 +14,7 @@
 // CUDA-core kernels (any supported dtype and head size): a first device path of this variant, bound
 // by the re-reading of the approximated keys (each of them enters the sums of all Hkv units of its layer).
 #include "common.cuh"
+#include "decode_layer_mma.cuh"
 #include "internal.h"
 
 namespace vec {
@@ -228,6 +229,34 @@ static vector_status launch_layer(const Dims& dm, int Hkv, int L, const void* q,
     return VECTOR_OK;
 }
 
+// bf16, head_dim 128, 8 KV heads, at most 32 query heads per layer: the split kernel on warp-level MMAs,
+// a block per (slice of the tokens, sequence, layer), and a merge kernel that applies the map the same way.
+static vector_status launch_layer_mma(const Dims& dm, int L, const void* q, const vector_cache* ch, const void* W, void* out,
+                                      int out_dtype, float* partial, cudaStream_t st) {
+    using T = __nv_bfloat16;
+    static PerDeviceOnce once;
+    if (once.first()) {
+        const cudaError_t e = cudaFuncSetAttribute(dlm::decode_layer_mma, cudaFuncAttributeMaxDynamicSharedMemorySize, dlm::SMEM_BYTES);
+        if (e != cudaSuccess) { once.undo(); VEC_CUDA_CHECK(e); }
+    }
+    const int UL = dm.U / dlm::HKV;
+    const int64_t tiles = (ch->n_ret + dlm::RT - 1) / dlm::RT + (ch->n_apx + dlm::AT - 1) / dlm::AT;
+    int64_t n_splits = (2 * (int64_t)sm_count() + UL - 1) / UL;       // two rounds of blocks
+    if (n_splits > tiles) n_splits = tiles;
+    if (n_splits > 32) n_splits = 32;
+    if (n_splits < 1) n_splits = 1;
+    dlm::decode_layer_mma<<<dim3((unsigned)n_splits, UL), dlm::THREADS, dlm::SMEM_BYTES, st>>>(
+        (const T*)q, (const T*)ch->ret_k, (const T*)ch->ret_v, (const T*)ch->apx_k, (long long)ch->cap_ret, (long long)ch->cap_apx,
+        (int)ch->n_ret, (int)ch->n_apx, dm.g, dm.scale * 1.4426950408889634f, partial);
+    VEC_LAUNCH_CHECK();
+    if (out_dtype == VECTOR_F32)
+        dlm::decode_layer_merge_mma<float><<<dm.U, 256, 0, st>>>(partial, (const T*)W, L, dm.g, (int)n_splits, (float*)out);
+    else
+        dlm::decode_layer_merge_mma<T><<<dm.U, 256, 0, st>>>(partial, (const T*)W, L, dm.g, (int)n_splits, (T*)out);
+    VEC_LAUNCH_CHECK();
+    return VECTOR_OK;
+}
+
 template <typename T, int D>
 static vector_status launch_layer_g(const Dims& dm, int Hkv, int L, const void* q, const vector_cache* ch, const void* W,
                                     void* out, int out_dtype, float* partial, cudaStream_t st) {
@@ -267,11 +296,13 @@ extern "C" vector_status vector_decode_attn_layer(const vector_shape* shape, con
     if (cache->n_ret > 0 && (!cache->ret_k || !cache->ret_v)) return VECTOR_ERR_NULL;
     if (cache->n_apx > 0 && !cache->apx_k) return VECTOR_ERR_NULL;
     const int Hkv = shape->n_kv_heads, L = shape->n_layers;
-    const int n_splits = layer_decode_splits(dm.U, cache->n_ret + cache->n_apx);
+    const bool mma = dm.dtype == VECTOR_BF16 && dm.d == 128 && Hkv == dlm::HKV && Hkv * dm.g <= dlm::MQ;
+    const int n_splits = mma ? 32 : layer_decode_splits(dm.U, cache->n_ret + cache->n_apx);      // the MMA path takes up to 32
     const size_t need = (size_t)dm.U * n_splits * dm.g * layer_rec_floats(dm.d, Hkv) * sizeof(float);
     if (!ws || ((uintptr_t)ws & 255) || ws_bytes < need) return VECTOR_ERR_WORKSPACE;
     cudaStream_t st = (cudaStream_t)stream;
     float* partial = (float*)ws;
+    if (mma) return launch_layer_mma(dm, L, q, cache, W_layer, out, out_dtype, partial, st);
     if (dm.dtype == VECTOR_F32)
         return dm.d == 64 ? launch_layer_g<float, 64>(dm, Hkv, L, q, cache, W_layer, out, out_dtype, partial, st)
                           : launch_layer_g<float, 128>(dm, Hkv, L, q, cache, W_layer, out, out_dtype, partial, st);
