@@ -489,13 +489,14 @@ def run_workload(env, cfg, wl, percent, steps, warmup, D, extras=True, want_e2e=
         ls_ms = timed(lambda: vec.vector_layer_scores(shape, comp.scores, N, lsc), 5)
         rl_ms = timed(lambda: vec.vector_route_layer(shape, budget, lsc, Kt, Vt, Wl, l_tier, l_ret, l_apx, None, None, lws), 5)
         cl_ms = timed(lambda: vec.vector_compact_layer(shape, budget, Kt, Vt, l_ret, l_apx, comp.cache), 5)
-        dl_ms = timed(lambda: vec.vector_decode_attn_layer(shape, qs[0], comp.cache, Wl, out, lws), 3)
+        dl_ms = timed(lambda: vec.vector_decode_attn_layer(shape, qs[0], comp.cache, Wl, out, lws), 10)
         rl_flop = 2.0 * UL * n_pool * DL * DL
         layer_map = {"layer_scores_ms": ls_ms, "route_layer_ms": rl_ms, "route_layer_tflops": rl_flop / (rl_ms * 1e-3) / 1e12,
                      "route_layer_frac_of_sustained_bf16": rl_flop / (rl_ms * 1e-3) / 1e12 / tf,
                      "compact_layer_ms": cl_ms, "decode_layer_us_per_step": dl_ms * 1e3,
                      "decode_layer_gbs": U * (2 * n_ret + n_apx) * d * es / (dl_ms * 1e-3) / 1e9,
-                     "note": "first device version: tcgen05 residual at the L2 rate, CUDA-core decode"}
+                     "decode_layer_frac_of_measured_copy": U * (2 * n_ret + n_apx) * d * es / (dl_ms * 1e-3) / 1e9 / hbm,
+                     "note": "tcgen05 residual at the L2 rate (a first version); decode split and merge on warp-level MMAs"}
         del Wl, lws, lsc, l_tier, l_ret, l_apx
         comp.compact(Kt, Vt)              # the per-head cache back in place for what follows
 

@@ -2,21 +2,20 @@
 // building block of Step 1 (the n_pool largest scores) and Step 3 (the n_apx smallest
 // residuals) of the routing (paper Section 3.2).  One thread block per unit.
 //
-// The k-th key is found by a most-significant-digit radix select on an order-preserving
-// 32-bit image of the fp32 value, digits of 11, 11 and 10 bits:
-//   pass 1  reads the whole input and counts the leading digit;
-//   pass 2  reads it once more, warp by contiguous piece, and on the way (a) notes per group
-//           of 32 elements, as a bit mask, those whose leading digit already beats the k-th
-//           key's and (b) lists the indices of those that share it (the candidates: a quarter
-//           of a binade of values) while counting their second digit;
-//   pass 3  and the classification of the candidates against the k-th key run over the list;
-//   the per-piece counts and the emission in index order (block-wide prefix sums) then need
-//           the masks only, not the values.
-// The masks, the candidate list and (for the residuals) the images kept by pass 1 live in
-// dynamic shared memory sized to the input, so a context of 131072 tokens keeps its masks.
-// Fallbacks that read the input again: more candidates than the list holds (pass 3 and the
-// classification walk the input), no room for the masks (inputs beyond a few hundred
-// thousand elements).
+// The k-th key is found on an order-preserving 32-bit image of the fp32 value.  Two paths:
+//
+// select_lean (the one that normally runs): a histogram of the leading 11 bits over the whole input;
+//   one more pass that writes, per 32 elements, a bit mask of the elements whose leading bits beat the
+//   k-th key's (chosen) and one of those that share them (candidates: a quarter of a binade of
+//   values); each warp lists its own candidates, their next 11 bits are counted, and the few that
+//   share those as well are ranked against each other directly; the emission in index order then
+//   needs the masks only.  It gives up when a warp's share of the candidate list overflows or many
+//   values are equal, and then
+// select_emit (the general one) runs: a most-significant-digit radix select with digits of 11, 11 and
+//   10 bits whose passes fall back to re-reading the input when the list or the masks do not fit.
+//
+// The masks, the candidate list, the warps' transposition tiles and (general path, residuals) the
+// images kept by pass 1 live in dynamic shared memory sized to the input.
 #ifndef VECTOR_SELECT_CUH_
 #define VECTOR_SELECT_CUH_
 
@@ -328,9 +327,8 @@ __device__ __forceinline__ void select_emit(const float* __restrict__ vals, int 
 // turn up than the list holds -- the caller then runs select_emit.
 
 // The bin search of pick_bin done by the first four warps only (16 bins a lane): a fortieth of the
-// instructions, the other warps wait at the barrier.  The bin and inner rank of rank_a go to bc[0], bc[1],
-// those of rank_b (if > 0) to bc[2], bc[3].
-__device__ __forceinline__ void pick_bins_few(const int* hist, int rank_a, int rank_b, int* bc, int* part) {
+// instructions, the other warps wait at the barrier.  Results go to bc[0] (bin) and bc[1] (rank inside it).
+__device__ __forceinline__ void pick_bin_few(const int* hist, int remaining, int* bc, int* part) {
     constexpr int NWP = 4, BW = SEL_BINS / NWP, BPL = BW / 32;
     const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
     const int r0 = wid * BW + lane * BPL;                    // rank from the top of this lane's first bin
@@ -347,26 +345,19 @@ __device__ __forceinline__ void pick_bins_few(const int* hist, int rank_a, int r
         int above = 0;
 #pragma unroll
         for (int w = 0; w < NWP; ++w) above += w < wid ? part[w] : 0;
-        const int s = lane_scan_incl(tot_l, lane);
-#pragma unroll
-        for (int which = 0; which < 2; ++which) {
-            const int remaining = which ? rank_b : rank_a;
-            if (remaining > 0 && above < remaining && above + tot >= remaining) {     // exactly one warp
-                const int r = remaining - above;
-                if (s - tot_l < r && s >= r) {                   // exactly one lane: walks its bins from the top
-                    int acc = s - tot_l;
-                    for (int j = 0; j < BPL; ++j) {
-                        const int c = hist[SEL_BINS - 1 - (r0 + j)];
-                        if (acc < r && acc + c >= r) { bc[2 * which] = SEL_BINS - 1 - (r0 + j); bc[2 * which + 1] = r - acc; }
-                        acc += c;
-                    }
+        if (above < remaining && above + tot >= remaining) {     // exactly one warp
+            const int r = remaining - above;
+            const int s = lane_scan_incl(tot_l, lane);
+            if (s - tot_l < r && s >= r) {                       // exactly one lane: walks its bins from the top
+                int acc = s - tot_l;
+                for (int j = 0; j < BPL; ++j) {
+                    const int c = hist[SEL_BINS - 1 - (r0 + j)];
+                    if (acc < r && acc + c >= r) { bc[0] = SEL_BINS - 1 - (r0 + j); bc[1] = r - acc; }
+                    acc += c;
                 }
             }
         }
     }
-}
-__device__ __forceinline__ void pick_bin_few(const int* hist, int remaining, int* bc, int* part) {
-    pick_bins_few(hist, remaining, 0, bc, part);
 }
 
 template <bool SMALLEST>

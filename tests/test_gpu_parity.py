@@ -520,6 +520,33 @@ def test_decode_long_block_ranges(oracle):
             assert np.max(np.abs(out1[u].cpu().double().numpy() - o_tok)) <= 2e-2, (base, u, "per tile")
 
 
+@pytest.mark.parametrize("g", [1, 2, 3, 6])
+def test_decode_every_group_size(oracle, g):
+    """Query heads per KV head other than the configurations' 4 and 8: the merge kernel's block is 128 g threads
+    and the MMA rows and columns beyond g are padding.  Both forms, three units, a ragged key-only tile."""
+    wl = synth.shrink(synth.WORKLOADS[1], N=2048, n_kv_heads=3, n_q_heads=3 * g, n_calib=1024)
+    K, V, _ = synth.context(wl, DEV)
+    W = calibrated_maps(wl).to(DEV)
+    sh = shape_of(wl)
+    _, sq, _ = synth.all_head_params(wl, DEV)
+    q = synth.decode_q(wl, 0, DEV, sq)
+    ws = vec.alloc_workspace(sh, budget_of(wl, 50))
+    ipos = torch.arange(wl.N, dtype=torch.int32, device=DEV).repeat(wl.units, 1).contiguous()
+    n_ret, n_apx = 700, 1100 + 13
+    cache = vec.Cache(K.clone(), V.clone(), K.flip(1).contiguous(), ipos, ipos.clone(), n_ret, n_apx)
+    out = torch.empty(wl.units, wl.group, wl.head_dim, dtype=torch.float32, device=DEV)
+    out1 = torch.empty_like(out)
+    vec.vector_decode_attn(sh, q, cache, W, out, 0, ws)
+    vec.vector_decode_attn(sh, q, cache, W, out1, 1, ws)
+    torch.cuda.synchronize()
+    assert vec.vector_device_fault() == 0
+    for u in range(wl.units):
+        o_tok, o = oracle.attend(q[u].cpu(), cache.ret_k[u, :n_ret].cpu(), cache.ret_v[u, :n_ret].cpu(),
+                                 cache.apx_k[u, :n_apx].cpu(), W[u].cpu(), 1.0 / np.sqrt(wl.head_dim))
+        assert np.max(np.abs(out[u].cpu().double().numpy() - o)) <= 2e-2, (g, u)
+        assert np.max(np.abs(out1[u].cpu().double().numpy() - o_tok)) <= 2e-2, (g, u, "per tile")
+
+
 @pytest.mark.parametrize("base,head_dim,N,Bp,n_a", [(0, 64, 777, 230, 100), (0, 128, 500, 61, 0), (1, 64, 900, 167, 167),
                                                     (1, 128, 1500, 514, 257)])
 def test_compact_bit_exact(oracle, base, head_dim, N, Bp, n_a):
