@@ -5,7 +5,8 @@
 // approximated key is read once for the key sums of all query heads of the layer.
 //
 // Split kernel: 8 warps, warp w = KV head w.  The slice is walked in tiles that fill one 64 KB stage (two
-// stages, cp.async, the next tile in flight while this one is worked on): 16 retained tokens (keys and
+// stages, cp.async, the next tile in flight while this one is worked on; a third stage would leave the
+// first-level cache, where the spilled registers live, a few KB): 16 retained tokens (keys and
 // values of the 8 heads) or 32 approximated tokens (keys of the 8 heads).  Per tile
 //   phase 1  warp h: logits of its g query heads against head h's keys (M = the heads padded to 16 rows),
 //            online softmax; for an approximated tile the probabilities go to shared memory as bf16
@@ -28,7 +29,8 @@ constexpr int HKV = 8, THREADS = 32 * HKV, MQ = 32;        // query heads per la
 constexpr int RT = 16, AT = 32;                            // tokens per retained / approximated tile
 constexpr int STAGE_BYTES = 65536, HEAD_RET = RT * 256, HEAD_APX = AT * 256;
 constexpr int PS_ROW = 80;                                 // bytes per row of P: 32 tokens + padding (conflict-free ldmatrix)
-constexpr int SMEM_BYTES = 2 * STAGE_BYTES + 2 * MQ * PS_ROW + MQ * 4 + 128;
+constexpr int STAGES = 2;
+constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 2 * MQ * PS_ROW + MQ * 4 + 128;
 constexpr int REC = 2 + 128 + HKV * 128;
 
 // grid (n_splits, U / 8), THREADS threads, SMEM_BYTES dynamic shared memory.
@@ -38,7 +40,7 @@ decode_layer_mma(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __res
                  long long cap_apx, int n_ret, int n_apx, int g, float scale_log2e, float* __restrict__ partial) {
     extern __shared__ __align__(128) unsigned char lsm[];
     unsigned char* stage0 = lsm;
-    unsigned char* ps_hi = lsm + 2 * STAGE_BYTES;
+    unsigned char* ps_hi = lsm + STAGES * STAGE_BYTES;
     unsigned char* ps_lo = ps_hi + MQ * PS_ROW;
     float* alpha_s = reinterpret_cast<float*>(ps_lo + MQ * PS_ROW);
     const int split = blockIdx.x, n_splits = gridDim.x, ul = blockIdx.y;
@@ -69,37 +71,48 @@ decode_layer_mma(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __res
     }
     float m = -INFINITY, l = 0.f;
 
-    // 4096 16-byte pieces per tile, 16 per thread; rows past the pool's end are filled with zeros
+    // 4096 16-byte pieces per tile, 16 per thread; rows past the pool's end are filled with zeros.  A thread's
+    // pieces share the 16-byte column (tid & 15) and the token row (tid >> 4, + 16 for every other piece of an
+    // approximated tile); they differ in the head (and, retained, in keys or values): fixed strides from one address.
+    const int p_tok = tid >> 4, p_ch = tid & 15;
+    const uint32_t p_dst = (uint32_t)(p_tok * 256 + ((p_ch ^ (p_tok & 7)) << 4));
+    const size_t ret_head = (size_t)cap_ret * 128, apx_head = (size_t)cap_apx * 128;      // elements from one head's pool to the next
     auto load_tile = [&](int t, unsigned char* st) {
-        const uint32_t sbase = tma::smem_u32(st);
+        const uint32_t dst = tma::smem_u32(st) + p_dst;
         if (t < n_rt) {
-            const int tok0 = t * RT;
+            const int tok = t * RT + p_tok;
+            const bool in = tok < n_ret;
+            const size_t off = ((size_t)ul * HKV * cap_ret + (in ? tok : 0)) * 128 + p_ch * 8;
+            const __nv_bfloat16* ks = ret_k + off;
+            const __nv_bfloat16* vs = ret_v + off;
 #pragma unroll
-            for (int j = 0; j < 16; ++j) {
-                const int e = tid + THREADS * j, isv = e >> 11, rem = e & 2047, hh = rem >> 8, tok = (rem >> 4) & 15, ch = rem & 15;
-                const bool in = tok0 + tok < n_ret;
-                const __nv_bfloat16* src = (isv ? ret_v : ret_k) + (((size_t)ul * HKV + hh) * cap_ret + (in ? tok0 + tok : 0)) * 128 + ch * 8;
-                rtc::cp_async16(sbase + isv * 32768 + hh * HEAD_RET + tok * 256 + ((ch ^ (tok & 7)) << 4), src, in ? 16u : 0u);
+            for (int hh = 0; hh < HKV; ++hh) {
+                rtc::cp_async16(dst + hh * HEAD_RET, ks + hh * ret_head, in ? 16u : 0u);
+                rtc::cp_async16(dst + 32768 + hh * HEAD_RET, vs + hh * ret_head, in ? 16u : 0u);
             }
         } else {
-            const int tok0 = (t - n_rt) * AT;
+            const int tok = (t - n_rt) * AT + p_tok;
+            const bool in0 = tok < n_apx, in1 = tok + 16 < n_apx;
+            const __nv_bfloat16* k0 = apx_k + ((size_t)ul * HKV * cap_apx + (in0 ? tok : 0)) * 128 + p_ch * 8;
+            const __nv_bfloat16* k1 = apx_k + ((size_t)ul * HKV * cap_apx + (in1 ? tok + 16 : 0)) * 128 + p_ch * 8;
 #pragma unroll
-            for (int j = 0; j < 16; ++j) {
-                const int e = tid + THREADS * j, hh = e >> 9, tok = (e >> 4) & 31, ch = e & 15;
-                const bool in = tok0 + tok < n_apx;
-                const __nv_bfloat16* src = apx_k + (((size_t)ul * HKV + hh) * cap_apx + (in ? tok0 + tok : 0)) * 128 + ch * 8;
-                rtc::cp_async16(sbase + hh * HEAD_APX + tok * 256 + ((ch ^ (tok & 7)) << 4), src, in ? 16u : 0u);
+            for (int hh = 0; hh < HKV; ++hh) {
+                rtc::cp_async16(dst + hh * HEAD_APX, k0 + hh * apx_head, in0 ? 16u : 0u);
+                rtc::cp_async16(dst + hh * HEAD_APX + 16 * 256, k1 + hh * apx_head, in1 ? 16u : 0u);
             }
         }
+    };
+    auto prefetch = [&](int t) {
+        if (t < t_hi) load_tile(t, stage0 + ((t - t_lo) % STAGES) * STAGE_BYTES);
         rtc::cp_async_commit();
     };
 
-    if (t_lo < t_hi) load_tile(t_lo, stage0);
+    prefetch(t_lo);
     for (int t = t_lo; t < t_hi; ++t) {
-        unsigned char* st = stage0 + ((t - t_lo) & 1) * STAGE_BYTES;
+        unsigned char* st = stage0 + ((t - t_lo) % STAGES) * STAGE_BYTES;
         rtc::cp_async_wait<0>();
-        __syncthreads();                       // the tile has landed; everyone is done with the other stage, P and the factors
-        if (t + 1 < t_hi) load_tile(t + 1, stage0 + ((t + 1 - t_lo) & 1) * STAGE_BYTES);
+        __syncthreads();                       // the tile has landed; everyone is done with the stage of tile t - 1, P and the factors
+        prefetch(t + 1);                       // into the stage of tile t - 1
         const bool retained = t < n_rt;
         const int ntok = retained ? min(RT, n_ret - t * RT) : min(AT, n_apx - (t - n_rt) * AT);
         const uint32_t kbase = tma::smem_u32(st) + h * (retained ? HEAD_RET : HEAD_APX);
@@ -170,14 +183,18 @@ decode_layer_mma(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __res
             const uint32_t a0 = dbf::pack_bf16(sc[0][0], sc[0][1]), a2 = dbf::pack_bf16(sc[1][0], sc[1][1]);
             const uint32_t l0 = dbf::pack_bf16(sc[0][0] - __uint_as_float(a0 << 16), sc[0][1] - __uint_as_float(a0 & 0xffff0000u));
             const uint32_t l2 = dbf::pack_bf16(sc[1][0] - __uint_as_float(a2 << 16), sc[1][1] - __uint_as_float(a2 & 0xffff0000u));
+            // the hi and the lo product of an accumulator are kept a whole sweep apart: back to back the second
+            // would wait for the first
 #pragma unroll
-            for (int np = 0; np < 8; ++np) {
-                uint32_t b0, b1, b2, b3;
-                dbf::ldsm_x4_t(vbase + (r8 + (mat & 1) * 8) * 256 + (((2 * np + (mat >> 1)) ^ r8) << 4), b0, b1, b2, b3);
-                dbf::mma_lo8(acc_v[2 * np][0], acc_v[2 * np][1], zz[0], zz[1], a0, a2, b0, b1);
-                dbf::mma_lo8(acc_v[2 * np][0], acc_v[2 * np][1], zz[0], zz[1], l0, l2, b0, b1);
-                dbf::mma_lo8(acc_v[2 * np + 1][0], acc_v[2 * np + 1][1], zz[0], zz[1], a0, a2, b2, b3);
-                dbf::mma_lo8(acc_v[2 * np + 1][0], acc_v[2 * np + 1][1], zz[0], zz[1], l0, l2, b2, b3);
+            for (int part = 0; part < 2; ++part) {
+                const uint32_t x0 = part ? l0 : a0, x2 = part ? l2 : a2;
+#pragma unroll
+                for (int np = 0; np < 8; ++np) {
+                    uint32_t b0, b1, b2, b3;
+                    dbf::ldsm_x4_t(vbase + (r8 + (mat & 1) * 8) * 256 + (((2 * np + (mat >> 1)) ^ r8) << 4), b0, b1, b2, b3);
+                    dbf::mma_lo8(acc_v[2 * np][0], acc_v[2 * np][1], zz[0], zz[1], x0, x2, b0, b1);
+                    dbf::mma_lo8(acc_v[2 * np + 1][0], acc_v[2 * np + 1][1], zz[0], zz[1], x0, x2, b2, b3);
+                }
             }
         } else {
             // key sums over head h (= this warp) for all query heads of the layer: P[32 x 32] K_h[32 x 128]
@@ -192,15 +209,17 @@ decode_layer_mma(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __res
                     dbf::ldsm_x4(pl + mt * 16 * PS_ROW + kk * 32, al[mt][0], al[mt][1], al[mt][2], al[mt][3]);
                 }
 #pragma unroll
-                for (int np = 0; np < 8; ++np) {
-                    uint32_t b0, b1, b2, b3;
-                    dbf::ldsm_x4_t(kbase + (kk * 16 + r8 + (mat & 1) * 8) * 256 + (((2 * np + (mat >> 1)) ^ r8) << 4), b0, b1, b2, b3);
+                for (int part = 0; part < 2; ++part) {             // hi sweep, then lo sweep (see above)
 #pragma unroll
-                    for (int mt = 0; mt < 2; ++mt) {
-                        dbf::mma_16(acc_k[mt][2 * np], ah[mt][0], ah[mt][1], ah[mt][2], ah[mt][3], b0, b1);
-                        dbf::mma_16(acc_k[mt][2 * np], al[mt][0], al[mt][1], al[mt][2], al[mt][3], b0, b1);
-                        dbf::mma_16(acc_k[mt][2 * np + 1], ah[mt][0], ah[mt][1], ah[mt][2], ah[mt][3], b2, b3);
-                        dbf::mma_16(acc_k[mt][2 * np + 1], al[mt][0], al[mt][1], al[mt][2], al[mt][3], b2, b3);
+                    for (int np = 0; np < 8; ++np) {
+                        uint32_t b0, b1, b2, b3;
+                        dbf::ldsm_x4_t(kbase + (kk * 16 + r8 + (mat & 1) * 8) * 256 + (((2 * np + (mat >> 1)) ^ r8) << 4), b0, b1, b2, b3);
+#pragma unroll
+                        for (int mt = 0; mt < 2; ++mt) {
+                            const uint32_t* a = part ? al[mt] : ah[mt];
+                            dbf::mma_16(acc_k[mt][2 * np], a[0], a[1], a[2], a[3], b0, b1);
+                            dbf::mma_16(acc_k[mt][2 * np + 1], a[0], a[1], a[2], a[3], b2, b3);
+                        }
                     }
                 }
             }
@@ -265,13 +284,18 @@ decode_layer_merge_mma(const float* __restrict__ partial, const __nv_bfloat16* _
         akl[g + i / KD][i % KD] = __float2bfloat16_rn(0.f);
     }
     __syncthreads();
-    // merged sums: element e of a record's 128 + 1024 values, coalesced over the threads
+    // merged sums: element e of a record's 128 + 1024 values, coalesced over the threads; eight splits' loads
+    // in flight at a time
     for (int a = 0; a < g; ++a) {
         for (int e = tid; e < 128 + KD; e += 256) {
+            const float* src = rec0 + (size_t)a * REC + 2 + e;
             float v = 0.f;
-            for (int s = 0; s < n_splits; ++s) {
-                const float f = fs[a][s];
-                if (f != 0.f) v = fmaf(f, rec0[((size_t)s * g + a) * REC + 2 + e], v);
+            for (int s0 = 0; s0 < n_splits; s0 += 8) {
+                float x[8];
+#pragma unroll
+                for (int k = 0; k < 8; ++k) x[k] = src[(size_t)min(s0 + k, n_splits - 1) * g * REC];      // always a valid record
+#pragma unroll
+                for (int k = 0; k < 8; ++k) v = fmaf(s0 + k < n_splits ? fs[a][s0 + k] : 0.f, x[k], v);
             }
             if (e < 128) accv[a][e] = v;
             else {
